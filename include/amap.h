@@ -1,0 +1,237 @@
+/*
+ * amap.h -- composed affine copies: C ABI.
+ *
+ * A chain of layout operators (reshape, transpose, strided slice, concat, pad,
+ * im2col-style window gather, ...) is a sequence of loop nests, each holding
+ * one element-wise load  v = t_l[C_l i + b_l]  feeding one store
+ * t_s[C_s i + b_s] = v  (the paper's Section 2, equations (load) and (store),
+ * and the pair pattern of Section 2.1).  amap_compose() removes every
+ * intermediate tensor by composing the access maps on the host (Section 2.1,
+ * equations (1) and (2), repeated until no pair is left); amap_plan() chooses
+ * a CUDA kernel family for what remains; amap_execute() runs the single
+ * remaining copy on a caller-supplied stream.
+ *
+ * Conventions
+ *  - Tensors are dense, row-major; elements are opaque patterns of elem_size
+ *    bytes (1, 2, 4, 8 or 16).  No floating-point arithmetic happens anywhere.
+ *  - Every function returns AMAP_OK (0) or a negative amap_status.  Out-handles
+ *    are written only on success.  Nothing throws, exits or prints (unless the
+ *    environment variable AMAP_LOG is set, which prints composed pieces).
+ *  - Host arrays passed in are read during the call and copied; the caller
+ *    keeps ownership.  Handles returned are owned by the library until the
+ *    matching *_destroy call.  Device buffers are always the caller's.
+ *  - "host" / "device" is stated for every pointer argument.
+ */
+#ifndef AMAP_H_
+#define AMAP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum amap_status {
+  AMAP_OK = 0,
+  AMAP_EINVAL = -1,               /* null pointer, bad rank / bounds / ids / elem_size             */
+  AMAP_ESTORE_NOT_INJECTIVE = -2, /* a store map writes one element twice: it has no reverse       */
+  AMAP_EOOB = -3,                 /* an unguarded access can leave its tensor                      */
+  AMAP_EUNDEFINED = -4,           /* an element that is read (or an output element) is never written*/
+  AMAP_EOVERLAP = -5,             /* two statements write the same element                         */
+  AMAP_EOVERFLOW = -6,            /* an offset or element count does not fit the integer width used*/
+  AMAP_EALIGN = -7,               /* a device pointer is less aligned than the plan requires       */
+  AMAP_ECUDA = -8,                /* a CUDA runtime call failed; see amap_last_cuda_error()        */
+  AMAP_EUNSUPPORTED = -9,         /* valid input the host algebra cannot compose affinely          */
+  AMAP_ENOMEM = -10
+} amap_status;
+
+#define AMAP_CONST (-1) /* amap_access.tensor of a load that yields the statement's fill_bits */
+#define AMAP_MAX_LOOPS 12
+#define AMAP_MAX_RANK 8
+
+/* One access t[C i + b] (Section 2, equations (load)/(store)).  host pointers. */
+typedef struct amap_access {
+  int32_t tensor;   /* id of the tensor accessed, or AMAP_CONST (loads only)       */
+  int32_t rank;     /* m, the tensor's rank                                         */
+  const int64_t *C; /* m x n_loops, row-major                                       */
+  const int64_t *b; /* m                                                            */
+} amap_access;
+
+/* One loop nest = one load/store pair (Section 2.1).  For every i in the box
+ * 0 <= i_j < bounds[j]:  store.tensor[C_s i + b_s] = load.tensor[C_l i + b_l]. */
+typedef struct amap_stmt {
+  int32_t n_loops;       /* n, 0..AMAP_MAX_LOOPS                                    */
+  const int64_t *bounds; /* n extents, each >= 0 (host)                             */
+  amap_access load;
+  amap_access store;
+  int32_t guarded;    /* 1: a load index outside load.tensor's shape yields fill_bits instead of being an error */
+  uint64_t fill_bits; /* low elem_size bytes (elements wider than 8 bytes: zero-extended) */
+} amap_stmt;
+
+typedef struct amap_tensor {
+  int32_t rank;         /* 1..AMAP_MAX_RANK                                          */
+  const int64_t *shape; /* rank extents (host)                                       */
+} amap_tensor;
+
+/* A whole chain: external inputs, intermediates and one output tensor; the
+ * statements in an order in which every tensor is written before it is read. */
+typedef struct amap_chain {
+  int32_t n_tensors;
+  const amap_tensor *tensors;
+  int32_t n_stmts;
+  const amap_stmt *stmts;
+  int32_t n_inputs;
+  const int32_t *inputs; /* tensor ids bound to device pointers at execute time, in this order */
+  int32_t output;        /* tensor id of the result                                            */
+  int32_t elem_size;     /* 1, 2, 4, 8 or 16 bytes                                             */
+} amap_chain;
+
+typedef struct amap_builder amap_builder;
+typedef struct amap_map amap_map;
+typedef struct amap_plan_t amap_plan_t;
+
+/* ---------------------------------------------------------------------------
+ * Chain builder: emits the statements of the common operators in the paper's
+ * form (Section 2.1 names the families).  Each call appends one tensor and the
+ * statement(s) that define it and returns the new tensor's id in *out.
+ * All array arguments are host pointers with `rank` entries unless stated.
+ * ------------------------------------------------------------------------- */
+int amap_builder_create(int32_t elem_size, amap_builder **out);
+void amap_builder_destroy(amap_builder *b);
+/* an external input of the given shape */
+int amap_builder_input(amap_builder *b, int32_t rank, const int64_t *shape, int32_t *out);
+/* same flat order, new shape (element counts must agree) */
+int amap_builder_reshape(amap_builder *b, int32_t src, int32_t rank, const int64_t *shape, int32_t *out);
+/* out.shape[d] = in.shape[perm[d]] */
+int amap_builder_transpose(amap_builder *b, int32_t src, int32_t rank, const int32_t *perm, int32_t *out);
+/* out[o] = in[start + step*o], step >= 1, 0 <= start <= stop <= in.shape */
+int amap_builder_slice(amap_builder *b, int32_t src, int32_t rank, const int64_t *start, const int64_t *stop,
+                       const int64_t *step, int32_t *out);
+/* join n tensors (ids in srcs) on `axis` */
+int amap_builder_concat(amap_builder *b, int32_t n, const int32_t *srcs, int32_t axis, int32_t *out);
+/* lo/hi elements of fill_bits before/after every axis (one guarded statement) */
+int amap_builder_pad(amap_builder *b, int32_t src, int32_t rank, const int64_t *lo, const int64_t *hi,
+                     uint64_t fill_bits, int32_t *out);
+/* NHWC [N,H,W,C] -> [N*Ho*Wo, kh*kw*C] with column (r*kw+s)*C+c reading
+ * in[n, ho*stride+r-pad, wo*stride+s-pad, c], zero outside (one guarded, non-injective load) */
+int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                        int32_t *out);
+/* broadcast: out[o] = in[o mod in.shape] with out.shape[d] = reps[d]*in.shape[d] (the paper's repeat/tile family) */
+int amap_builder_tile(amap_builder *b, int32_t src, int32_t rank, const int64_t *reps, int32_t *out);
+/* declare a tensor that raw statements will define */
+int amap_builder_tensor(amap_builder *b, int32_t rank, const int64_t *shape, int32_t *out);
+/* append one raw statement (deep-copied) */
+int amap_builder_stmt(amap_builder *b, const amap_stmt *stmt);
+/* a view of everything built so far with `output` as the result; valid until the next builder call */
+int amap_builder_chain(amap_builder *b, int32_t output, const amap_chain **out);
+
+/* ---------------------------------------------------------------------------
+ * amap_compose: Section 2.1, equations (1) and (2), to the fixpoint.
+ * Host only, no CUDA.  The result is a list of PIECES, each one loop nest in
+ * the paper's form over the FLAT (rank-1, row-major) views of an external
+ * input and of the output:
+ *     out.flat[C_s i + b_s] = in[input].flat[C_l i + b_l]      for i in the box,
+ * so C_l and C_s are 1 x n_loops (element strides) and b_l, b_s scalars.
+ * Pieces write pairwise disjoint sets that together cover the output.
+ * Errors: EINVAL, ESTORE_NOT_INJECTIVE, EOOB, EUNDEFINED, EOVERLAP,
+ * EOVERFLOW, EUNSUPPORTED (e.g. a reshape whose factors do not line up with
+ * the loops that read it), ENOMEM.
+ * ------------------------------------------------------------------------- */
+int amap_compose(const amap_chain *chain, amap_map **out_map);
+void amap_map_destroy(amap_map *map);
+
+/* a constraint  0 <= offset + sum_k coef[k] * i_k < extent  on the loop indices */
+typedef struct amap_constraint {
+  const int64_t *coef; /* n_loops (host, owned by the map) */
+  int64_t offset;
+  int64_t extent;
+} amap_constraint;
+
+typedef struct amap_piece {
+  int32_t n_loops;
+  const int64_t *bounds; /* n_loops (host, owned by the map)                                   */
+  int32_t input;         /* position in amap_chain.inputs of the tensor read, or AMAP_CONST    */
+  const int64_t *C_l;    /* n_loops source strides in elements (NULL for AMAP_CONST)           */
+  int64_t b_l;
+  const int64_t *C_s; /* n_loops destination strides in elements                               */
+  int64_t b_s;
+  int32_t n_guards; /* where any guard fails the piece stores fill_bits instead of loading     */
+  const amap_constraint *guards;
+  int32_t n_domain; /* where any of these fails the loop point is not part of the piece        */
+  const amap_constraint *domain;
+  uint64_t fill_bits;
+} amap_piece;
+
+int amap_map_num_pieces(const amap_map *map, int32_t *n);
+/* *out receives views into the map, valid until amap_map_destroy */
+int amap_map_get_piece(const amap_map *map, int32_t k, amap_piece *out);
+/* element counts of the external inputs (n_inputs entries written to in_numel) and of the output */
+int amap_map_sizes(const amap_map *map, int32_t *n_inputs, int64_t *in_numel /* may be NULL */, int64_t *out_numel,
+                   int32_t *elem_size);
+
+/* ---------------------------------------------------------------------------
+ * amap_plan: choose a kernel family per piece and build the launch table.
+ * Needs a CUDA device: `device` is a CUDA ordinal; the call makes it current,
+ * uploads a small descriptor table to device memory owned by the plan, and
+ * restores the previous device.  A plan is immutable and may be executed any
+ * number of times, on any stream of that device, concurrently.
+ * ------------------------------------------------------------------------- */
+typedef enum amap_kernel_kind {
+  AMAP_KERNEL_AUTO = 0,
+  AMAP_KERNEL_GATHER = 1,    /* one element per thread, full index arithmetic, guards; handles every piece */
+  AMAP_KERNEL_COPY = 2,      /* innermost loop contiguous on both sides: 16-byte vector runs               */
+  AMAP_KERNEL_TRANSPOSE = 3, /* the fastest source loop differs from the fastest destination loop: smem tile */
+  AMAP_KERNEL_FILL = 4       /* no source: vector stores of the constant                                   */
+} amap_kernel_kind;
+
+typedef struct amap_plan_opts {
+  int32_t force_kernel;     /* amap_kernel_kind; AUTO picks per piece; a family that cannot run a piece falls back to GATHER */
+  int32_t pointer_align;    /* bytes every src/dst base pointer is promised to be aligned to (0 = elem_size; 16 enables vectors) */
+  int32_t reserved[6];      /* must be zero */
+} amap_plan_opts;
+
+typedef struct amap_stats {
+  int64_t bytes_read;    /* unique source bytes the composed copy must read   */
+  int64_t bytes_written; /* output bytes written (copied + filled)            */
+  int64_t bytes_filled;  /* the part of bytes_written that has no source      */
+  int32_t n_pieces;
+  int32_t n_launches;     /* kernels one amap_execute enqueues                 */
+  int32_t kernel_kind[4]; /* pieces planned per family: [0] gather [1] copy [2] transpose [3] fill */
+  int32_t reserved[2];
+} amap_stats;
+
+int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts /* host, may be NULL */,
+              amap_plan_t **out_plan);
+void amap_plan_destroy(amap_plan_t *plan);
+int amap_plan_stats(const amap_plan_t *plan, amap_stats *out /* host */);
+/* kernel family chosen for piece k (an amap_kernel_kind) */
+int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
+
+/* ---------------------------------------------------------------------------
+ * amap_execute: the surviving copy (the data movement Section 2.1 cannot
+ * remove and Section 2.2 wants run at full memory bandwidth).
+ *   src_dev_ptrs  host array of n_inputs DEVICE pointers, in amap_chain.inputs order
+ *   dst_dev_ptr   DEVICE pointer to the output (out_numel * elem_size bytes)
+ *   cuda_stream   a cudaStream_t (NULL = the legacy default stream)
+ * Enqueues the plan's kernel(s) and returns without synchronising or
+ * allocating.  Source and destination must not overlap.  Pointers must be
+ * aligned to the plan's pointer_align, else AMAP_EALIGN and nothing is
+ * enqueued.  Launch failures give AMAP_ECUDA.
+ * ------------------------------------------------------------------------- */
+int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, void *cuda_stream);
+
+/* Same copy with HOST buffers: uploads the inputs, runs the plan, downloads
+ * the output and waits.  Uses device staging memory owned by the plan
+ * (allocated on first use).  src_host_ptrs: host array of n_inputs HOST
+ * pointers; dst_host_ptr: HOST.  Pinned host memory makes the copies faster
+ * but is not required. */
+int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr, void *cuda_stream);
+
+const char *amap_strerror(int code);
+/* text of the last CUDA error seen by this thread in this library ("" if none) */
+const char *amap_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMAP_H_ */

@@ -1,0 +1,350 @@
+"""Thin ctypes binding of libamap.so (include/amap.h): argument marshalling only.
+
+Every step of the path -- building statements, composing the affine maps,
+planning and the copy itself -- runs inside the C/CUDA library.  PyTorch is
+used only for device memory (`Tensor.data_ptr()`) and streams.  There is no
+CPU fallback: if the library cannot be built or loaded, importing this module
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_int, c_int32, c_int64, c_uint64, c_void_p
+
+from . import build as _build
+
+AMAP_CONST = -1
+KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2, 3, 4
+KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
+
+EXPORTS = [
+    "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",
+    "amap_builder_transpose", "amap_builder_slice", "amap_builder_concat", "amap_builder_pad",
+    "amap_builder_window", "amap_builder_tile", "amap_builder_tensor", "amap_builder_stmt",
+    "amap_builder_chain", "amap_compose", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
+    "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
+    "amap_execute", "amap_execute_host", "amap_strerror", "amap_last_cuda_error",
+]
+
+
+class AmapError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = _lib.amap_strerror(code).decode()
+        if code == -8:
+            msg += " (" + _lib.amap_last_cuda_error().decode() + ")"
+        super().__init__("%s: %s [%d]" % (where, msg, code))
+
+
+class _Access(Structure):
+    _fields_ = [("tensor", c_int32), ("rank", c_int32), ("C", POINTER(c_int64)), ("b", POINTER(c_int64))]
+
+
+class _Stmt(Structure):
+    _fields_ = [
+        ("n_loops", c_int32), ("bounds", POINTER(c_int64)), ("load", _Access), ("store", _Access),
+        ("guarded", c_int32), ("fill_bits", c_uint64),
+    ]
+
+
+class _Constraint(Structure):
+    _fields_ = [("coef", POINTER(c_int64)), ("offset", c_int64), ("extent", c_int64)]
+
+
+class _Piece(Structure):
+    _fields_ = [
+        ("n_loops", c_int32), ("bounds", POINTER(c_int64)), ("input", c_int32), ("C_l", POINTER(c_int64)),
+        ("b_l", c_int64), ("C_s", POINTER(c_int64)), ("b_s", c_int64), ("n_guards", c_int32),
+        ("guards", POINTER(_Constraint)), ("n_domain", c_int32), ("domain", POINTER(_Constraint)),
+        ("fill_bits", c_uint64),
+    ]
+
+
+class _PlanOpts(Structure):
+    _fields_ = [("force_kernel", c_int32), ("pointer_align", c_int32), ("reserved", c_int32 * 6)]
+
+
+class _Stats(Structure):
+    _fields_ = [
+        ("bytes_read", c_int64), ("bytes_written", c_int64), ("bytes_filled", c_int64), ("n_pieces", c_int32),
+        ("n_launches", c_int32), ("kernel_kind", c_int32 * 4), ("reserved", c_int32 * 2),
+    ]
+
+
+def _load():
+    path = _build.build_library()
+    lib = ctypes.CDLL(path)
+    lib.amap_strerror.restype = c_char_p
+    lib.amap_strerror.argtypes = [c_int]
+    lib.amap_last_cuda_error.restype = c_char_p
+    lib.amap_builder_destroy.restype = None
+    lib.amap_builder_destroy.argtypes = [c_void_p]
+    lib.amap_map_destroy.restype = None
+    lib.amap_map_destroy.argtypes = [c_void_p]
+    lib.amap_plan_destroy.restype = None
+    lib.amap_plan_destroy.argtypes = [c_void_p]
+    lib.amap_builder_pad.argtypes = [c_void_p, c_int32, c_int32, POINTER(c_int64), POINTER(c_int64), c_uint64, POINTER(c_int32)]
+    lib.amap_execute.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
+    lib.amap_execute_host.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+
+
+def _check(rc, where):
+    if rc != 0:
+        raise AmapError(rc, where)
+
+
+def _i64(a):
+    return (c_int64 * max(len(a), 1))(*[int(v) for v in a])
+
+
+def _i32(a):
+    return (c_int32 * max(len(a), 1))(*[int(v) for v in a])
+
+
+class Builder:
+    """amap_builder_*: emits the load/store statements of layout operators."""
+
+    def __init__(self, elem_size: int):
+        self._h = c_void_p()
+        _check(_lib.amap_builder_create(c_int32(elem_size), byref(self._h)), "amap_builder_create")
+        self.elem_size = elem_size
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.amap_builder_destroy(self._h)
+            self._h = None
+
+    def _out(self, rc, where, out):
+        _check(rc, where)
+        return out.value
+
+    def input(self, shape):
+        o = c_int32()
+        return self._out(_lib.amap_builder_input(self._h, len(shape), _i64(shape), byref(o)), "amap_builder_input", o)
+
+    def tensor(self, shape):
+        o = c_int32()
+        return self._out(_lib.amap_builder_tensor(self._h, len(shape), _i64(shape), byref(o)), "amap_builder_tensor", o)
+
+    def reshape(self, src, shape):
+        o = c_int32()
+        return self._out(_lib.amap_builder_reshape(self._h, src, len(shape), _i64(shape), byref(o)), "amap_builder_reshape", o)
+
+    def transpose(self, src, perm):
+        o = c_int32()
+        return self._out(_lib.amap_builder_transpose(self._h, src, len(perm), _i32(perm), byref(o)), "amap_builder_transpose", o)
+
+    def slice(self, src, start, stop, step):
+        o = c_int32()
+        return self._out(
+            _lib.amap_builder_slice(self._h, src, len(start), _i64(start), _i64(stop), _i64(step), byref(o)),
+            "amap_builder_slice", o,
+        )
+
+    def concat(self, srcs, axis):
+        o = c_int32()
+        return self._out(_lib.amap_builder_concat(self._h, len(srcs), _i32(srcs), axis, byref(o)), "amap_builder_concat", o)
+
+    def pad(self, src, lo, hi, fill_bits=0):
+        o = c_int32()
+        return self._out(
+            _lib.amap_builder_pad(self._h, src, len(lo), _i64(lo), _i64(hi), c_uint64(fill_bits), byref(o)),
+            "amap_builder_pad", o,
+        )
+
+    def window(self, src, kh, kw, stride, pad):
+        o = c_int32()
+        return self._out(_lib.amap_builder_window(self._h, src, kh, kw, stride, pad, byref(o)), "amap_builder_window", o)
+
+    def tile(self, src, reps):
+        o = c_int32()
+        return self._out(_lib.amap_builder_tile(self._h, src, len(reps), _i64(reps), byref(o)), "amap_builder_tile", o)
+
+    def stmt(self, bounds, load, store, guarded=False, fill_bits=0):
+        """One raw statement.  load = None | (tensor, C rows, b); store = (tensor, C rows, b)."""
+        n = len(bounds)
+        st = _Stmt()
+        st.n_loops = n
+        keep = [_i64(bounds)]
+        st.bounds = keep[0]
+
+        def acc(a):
+            t, C, b = a
+            flat = [v for row in C for v in row]
+            Cb, bb = _i64(flat), _i64(b)
+            keep.extend([Cb, bb])
+            return _Access(int(t), len(b), Cb, bb)
+
+        if load is None:
+            st.load = _Access(AMAP_CONST, 0, None, None)
+        else:
+            st.load = acc(load)
+        st.store = acc(store)
+        st.guarded = int(bool(guarded))
+        st.fill_bits = int(fill_bits)
+        _check(_lib.amap_builder_stmt(self._h, byref(st)), "amap_builder_stmt")
+
+    def compose(self, output) -> "Map":
+        chain = c_void_p()
+        _check(_lib.amap_builder_chain(self._h, output, byref(chain)), "amap_builder_chain")
+        h = c_void_p()
+        _check(_lib.amap_compose(chain, byref(h)), "amap_compose")
+        return Map(h)
+
+
+class Map:
+    """A composed map: amap_compose's result."""
+
+    def __init__(self, handle):
+        self._h = handle
+        n_in, out_numel, es = c_int32(), c_int64(), c_int32()
+        _check(_lib.amap_map_sizes(self._h, byref(n_in), None, byref(out_numel), byref(es)), "amap_map_sizes")
+        ins = (c_int64 * max(n_in.value, 1))()
+        _check(_lib.amap_map_sizes(self._h, None, ins, None, None), "amap_map_sizes")
+        self.in_numel = [ins[q] for q in range(n_in.value)]
+        self.out_numel = out_numel.value
+        self.elem_size = es.value
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.amap_map_destroy(self._h)
+            self._h = None
+
+    def pieces(self):
+        n = c_int32()
+        _check(_lib.amap_map_num_pieces(self._h, byref(n)), "amap_map_num_pieces")
+        out = []
+        for k in range(n.value):
+            p = _Piece()
+            _check(_lib.amap_map_get_piece(self._h, k, byref(p)), "amap_map_get_piece")
+            nl = p.n_loops
+
+            def cons(ptr, cnt):
+                return [([ptr[c].coef[j] for j in range(nl)], ptr[c].offset, ptr[c].extent) for c in range(cnt)]
+
+            out.append(
+                {
+                    "bounds": [p.bounds[j] for j in range(nl)],
+                    "input": p.input,
+                    "C_l": [p.C_l[j] for j in range(nl)] if p.input >= 0 else None,
+                    "b_l": p.b_l,
+                    "C_s": [p.C_s[j] for j in range(nl)],
+                    "b_s": p.b_s,
+                    "guards": cons(p.guards, p.n_guards),
+                    "domain": cons(p.domain, p.n_domain),
+                    "fill_bits": p.fill_bits,
+                }
+            )
+        return out
+
+    def plan(self, device=0, force_kernel=KERNEL_AUTO, pointer_align=16) -> "Plan":
+        opts = _PlanOpts()
+        opts.force_kernel = force_kernel
+        opts.pointer_align = pointer_align
+        h = c_void_p()
+        _check(_lib.amap_plan(self._h, device, byref(opts), byref(h)), "amap_plan")
+        return Plan(h, self)
+
+
+class Plan:
+    """amap_plan's result; execute() enqueues the copy on a CUDA stream."""
+
+    def __init__(self, handle, amap: Map):
+        self._h = handle
+        self.map = amap
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.amap_plan_destroy(self._h)
+            self._h = None
+
+    def stats(self) -> dict:
+        s = _Stats()
+        _check(_lib.amap_plan_stats(self._h, byref(s)), "amap_plan_stats")
+        return {
+            "bytes_read": s.bytes_read, "bytes_written": s.bytes_written, "bytes_filled": s.bytes_filled,
+            "n_pieces": s.n_pieces, "n_launches": s.n_launches,
+            "kernels": {"gather": s.kernel_kind[0], "copy": s.kernel_kind[1], "transpose": s.kernel_kind[2], "fill": s.kernel_kind[3]},
+        }
+
+    def piece_kernels(self):
+        out = []
+        for k in range(self.stats()["n_pieces"]):
+            kind = c_int32()
+            _check(_lib.amap_plan_piece_kernel(self._h, k, byref(kind)), "amap_plan_piece_kernel")
+            out.append(KERNEL_NAMES[kind.value])
+        return out
+
+    def execute_ptrs(self, src_ptrs, dst_ptr, stream=0):
+        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        _check(_lib.amap_execute(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute")
+
+    def execute(self, srcs, dst, stream=None):
+        """srcs: CUDA tensors (contiguous), dst: CUDA tensor; stream: torch.cuda.Stream or None (current)."""
+        import torch
+
+        for t in list(srcs) + [dst]:
+            if not t.is_cuda or not t.is_contiguous():
+                raise ValueError("amap_execute wants contiguous CUDA tensors")
+        for t, n in zip(srcs, self.map.in_numel):
+            if t.numel() * t.element_size() != n * self.map.elem_size:
+                raise ValueError("input size differs from the composed map's")
+        if dst.numel() * dst.element_size() != self.map.out_numel * self.map.elem_size:
+            raise ValueError("output size differs from the composed map's")
+        s = (stream or torch.cuda.current_stream(dst.device)).cuda_stream
+        self.execute_ptrs([t.data_ptr() for t in srcs], dst.data_ptr(), s)
+
+    def execute_host(self, srcs, dst, stream=0):
+        """srcs / dst: host numpy arrays (or anything with .ctypes.data / .data_ptr())."""
+
+        def ptr(a):
+            return a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data
+
+        arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(ptr(a)) for a in srcs])
+        _check(_lib.amap_execute_host(self._h, arr, c_void_p(ptr(dst)), c_void_p(stream)), "amap_execute_host")
+
+
+def build_chain(chain) -> tuple:
+    """Feed a workloads.Chain to the library's builder.  Returns (builder, output tensor id)."""
+    b = Builder(chain.elem_size)
+    ids = [b.input(s) for s in chain.inputs]
+    for op in chain.ops:
+        k = op["kind"]
+        if k == "reshape":
+            t = b.reshape(ids[op["src"]], op["shape"])
+        elif k == "transpose":
+            t = b.transpose(ids[op["src"]], op["perm"])
+        elif k == "slice":
+            t = b.slice(ids[op["src"]], op["start"], op["stop"], op["step"])
+        elif k == "concat":
+            t = b.concat([ids[s] for s in op["srcs"]], op["axis"])
+        elif k == "pad":
+            t = b.pad(ids[op["src"]], op["lo"], op["hi"], 0)
+        elif k == "window":
+            t = b.window(ids[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"])
+        elif k == "tile":
+            t = b.tile(ids[op["src"]], op["reps"])
+        elif k == "stmts":
+            t = b.tensor(op["shape"])
+            for st in op["stmts"]:
+                load = None
+                if st["load"] is not None:
+                    lt, Cl, bl = st["load"]
+                    load = (ids[lt], Cl, bl)
+                Cs, bs = st["store"]
+                b.stmt(st["bounds"], load, (t, Cs, bs), st.get("guarded", False), st.get("fill", 0))
+        else:
+            raise ValueError("unknown operator kind %r" % k)
+        ids.append(t)
+    return b, ids[-1]
+
+
+def compose_chain(chain) -> Map:
+    b, out = build_chain(chain)
+    return b.compose(out)

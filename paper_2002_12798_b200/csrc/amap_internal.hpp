@@ -1,0 +1,78 @@
+// Internal data model of the host algebra (not part of the C ABI).
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "amap.h"
+
+namespace amap {
+
+// c0 + sum_k c[k] * i_k over a piece's loops
+struct Aff {
+  int64_t c0 = 0;
+  std::vector<int64_t> c;
+};
+
+// 0 <= e < extent
+struct Con {
+  Aff e;
+  int64_t extent = 0;
+};
+
+// One loop nest of the composed form: for i in the box (and where `domain`
+// holds) dst.flat[dst(i)] = guards hold ? src.flat[srcoff(i)] : fill.
+struct Piece {
+  std::vector<int64_t> ext;
+  Aff dst;
+  int src = AMAP_CONST;  // tensor id while composing; input slot in a finished map
+  Aff srcoff;
+  std::vector<Con> guards;
+  std::vector<Con> domain;
+  uint64_t fill = 0;
+  int n() const { return (int)ext.size(); }
+};
+
+struct TensorInfo {
+  std::vector<int64_t> shape;
+  std::vector<int64_t> stride;  // row-major, elements
+  int64_t numel = 0;
+  int input_slot = -1;  // >= 0 for external inputs
+};
+
+struct Status {
+  int code = AMAP_OK;
+  std::string msg;
+  bool ok() const { return code == AMAP_OK; }
+};
+
+// ---- simplify.cpp --------------------------------------------------------
+// interval of an affine expression over the box [0,ext)
+void aff_range(const Aff &a, const std::vector<int64_t> &ext, int64_t *lo, int64_t *hi);
+// Drops constraints that always hold, clips single-loop domain constraints
+// into the box.  Returns false when the piece has no points left.
+bool tighten(Piece &p);
+// number of loop points of the piece (box and domain); -1 if it cannot be counted cheaply
+int64_t count_points(const Piece &p);
+void reverse_loop(Piece &p, int k);
+void permute_loops(Piece &p, const std::vector<int> &order);
+void drop_unit_loops(Piece &p);
+// final canonical form of a composed map's pieces (splits single-loop guards
+// into copy + fill pieces, sorts by destination stride, merges loops)
+Status canonicalise(std::vector<Piece> &pieces);
+
+// ---- compose.cpp ---------------------------------------------------------
+struct Map {
+  int elem_size = 0;
+  std::vector<int64_t> in_numel;
+  int64_t out_numel = 0;
+  std::vector<Piece> pieces;
+  // storage for the C views handed out by amap_map_get_piece
+  std::vector<std::vector<amap_constraint>> guard_views, domain_views;
+};
+
+}  // namespace amap
+
+struct amap_map {
+  amap::Map m;
+};

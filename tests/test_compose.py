@@ -1,0 +1,289 @@
+"""Host algebra (amap_compose) on the CPU: the composed pieces, evaluated point
+by point with a few lines of numpy, must reproduce the oracle's sequential
+chain; plus the error paths and the C ABI's export list."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2002_12798_b200 import binding as B
+from paper_2002_12798_b200 import workloads as W
+from chain_gen import random_chain
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def eval_map(m, inputs):
+    """out.flat[C_s i + b_s] = in.flat[C_l i + b_l] for every loop point of every piece."""
+    out = np.zeros(m.out_numel, dtype=inputs[0].dtype)
+    cnt = np.zeros(m.out_numel, dtype=np.int32)
+    flat = [x.reshape(-1) for x in inputs]
+    for p in m.pieces():
+        nl = len(p["bounds"])
+        idx = np.indices(p["bounds"], dtype=np.int64).reshape(nl, -1) if nl else np.zeros((0, 1), dtype=np.int64)
+
+        def aff(c, c0):
+            v = np.full(idx.shape[1], c0, dtype=np.int64)
+            for k, ck in enumerate(c):
+                v += ck * idx[k]
+            return v
+
+        dom = np.ones(idx.shape[1], bool)
+        for c, o, e in p["domain"]:
+            v = aff(c, o)
+            dom &= (v >= 0) & (v < e)
+        g = np.ones(idx.shape[1], bool)
+        for c, o, e in p["guards"]:
+            v = aff(c, o)
+            g &= (v >= 0) & (v < e)
+        d = aff(p["C_s"], p["b_s"])[dom]
+        if p["input"] >= 0:
+            s = aff(p["C_l"], p["b_l"])[dom]
+            gg = g[dom]
+            vals = np.where(gg, flat[p["input"]][np.where(gg, s, 0)], p["fill_bits"]).astype(out.dtype)
+        else:
+            vals = np.full(d.shape, p["fill_bits"], dtype=out.dtype)
+        out[d] = vals
+        np.add.at(cnt, d, 1)
+    assert (cnt == 1).all(), "pieces must write every output element exactly once"
+    return out
+
+
+@pytest.mark.parametrize("name", sorted(W.reduced_configs()))
+def test_composed_map_equals_sequential_chain(name):
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    m = B.compose_chain(chain)
+    want = oracle.run_chain(chain, xs)
+    assert m.out_numel == want.size and m.elem_size == chain.elem_size
+    assert np.array_equal(eval_map(m, xs), want.reshape(-1))
+
+
+def test_c1_composes_to_the_closed_form():
+    (p,) = B.compose_chain(W.c1_small_chain()).pieces()
+    # loops (a, j, k) < (64, 8, 6): load X.flat[2a + 1024j + 128k + 128], store Y.flat[48a + 6j + k]
+    assert p["bounds"] == [64, 8, 6]
+    assert p["C_l"] == [2, 1024, 128] and p["b_l"] == 128
+    assert p["C_s"] == [48, 6, 1] and p["b_s"] == 0
+    assert not p["guards"] and not p["domain"]
+
+
+def test_full_size_maps_have_the_expected_shape():
+    full = W.full_configs()
+    (p,) = B.compose_chain(full["c2_fwd"]).pieces()
+    assert (p["bounds"], p["C_l"], p["C_s"]) == ([32, 3136, 256], [802816, 1, 3136], [802816, 256, 1])
+    (p,) = B.compose_chain(full["c2_inv"]).pieces()
+    assert (p["bounds"], p["C_l"], p["C_s"]) == ([32, 256, 3136], [802816, 1, 256], [802816, 3136, 1])
+    p0, p1 = B.compose_chain(full["c3"]).pieces()
+    assert p0["bounds"] == p1["bounds"] == [16, 32, 1536, 128]
+    assert p0["C_l"] == [8388608, 128, 4096, 1] and p0["C_s"] == [12582912, 393216, 128, 1]
+    assert (p0["b_s"], p1["b_s"], p0["input"], p1["input"]) == (0, 196608, 0, 1)
+    (p,) = B.compose_chain(full["c5"]).pieces()
+    assert p["bounds"] == [64, 56, 56, 3, 3, 128]
+    assert p["C_l"] == [401408, 7168, 128, 7168, 128, 1] and p["b_l"] == -7296
+    assert p["C_s"] == [3612672, 64512, 1152, 384, 128, 1]
+    assert len(p["guards"]) == 2 and not p["domain"]
+    c4 = B.compose_chain(full["c4"]).pieces()
+    copies = [p for p in c4 if p["input"] >= 0]
+    assert sorted(p["bounds"][-1] for p in copies) == [32, 64, 96, 128]
+    for p in copies:
+        cq = p["bounds"][-1]
+        assert p["bounds"] == [64, 28, 28, cq] and p["C_l"] == [784 * cq, 28, 1, 784] and p["C_s"] == [288000, 9600, 320, 1]
+    filled = sum(int(np.prod(p["bounds"])) for p in c4 if p["input"] < 0)
+    assert filled == 2375680
+
+
+def test_random_tiny_chains():
+    r = np.random.default_rng(12798)
+    done = unsupported = 0
+    for trial in range(300):
+        chain = random_chain(r)
+        xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
+        try:
+            m = B.compose_chain(chain)
+        except B.AmapError as e:
+            assert e.code == -9, (trial, chain.ops, str(e))  # only "cannot compose affinely" is acceptable
+            unsupported += 1
+            continue
+        want = oracle.run_chain(chain, xs)
+        assert np.array_equal(eval_map(m, xs), want.reshape(-1)), (trial, chain.ops)
+        done += 1
+    assert done >= 200, (done, unsupported)
+
+
+def test_pad_written_as_explicit_fill_statements():
+    """The other encoding of padding: border boxes of constant stores plus an interior copy."""
+    b = B.Builder(2)
+    x = b.input([4, 5])
+    t = b.tensor([6, 8])  # pad 1 on axis 0, (1, 2) on axis 1
+    eye = [[1, 0], [0, 1]]
+    b.stmt([1, 8], None, (t, eye, [0, 0]), fill_bits=7)
+    b.stmt([1, 8], None, (t, eye, [5, 0]), fill_bits=7)
+    b.stmt([4, 1], None, (t, eye, [1, 0]), fill_bits=7)
+    b.stmt([4, 2], None, (t, eye, [1, 6]), fill_bits=7)
+    b.stmt([4, 5], (x, eye, [0, 0]), (t, eye, [1, 1]))
+    y = b.transpose(t, [1, 0])
+    m = b.compose(y)
+    xin = np.arange(1, 21, dtype=np.uint16).reshape(4, 5)
+    want = np.pad(xin, [(1, 1), (1, 2)], constant_values=7).T
+    assert np.array_equal(eval_map(m, [xin]).reshape(8, 6), want)
+
+
+def test_window_over_a_transposed_input_stays_one_guarded_piece():
+    b = B.Builder(2)
+    x = b.input([2, 3, 6, 5])  # NCHW
+    nhwc = b.transpose(x, [0, 2, 3, 1])
+    y = b.window(nhwc, 3, 3, 1, 1)
+    m = b.compose(y)
+    ps = m.pieces()
+    assert len(ps) == 1 and len(ps[0]["guards"]) == 2
+    xin = np.random.default_rng(3).integers(1, 60000, size=(2, 3, 6, 5)).astype(np.uint16)
+    want = oracle.window(oracle.transpose(xin, [0, 2, 3, 1]), 3, 3, 1, 1)
+    assert np.array_equal(eval_map(m, [xin]), want.reshape(-1))
+
+
+def test_tile_is_a_broadcast_load():
+    b = B.Builder(4)
+    x = b.input([2, 3])
+    y = b.tile(x, [2, 3])
+    m = b.compose(b.transpose(y, [1, 0]))
+    xin = np.arange(6, dtype=np.uint32).reshape(2, 3) + 1
+    assert np.array_equal(eval_map(m, [xin]).reshape(9, 4), np.tile(xin, (2, 3)).T)
+
+
+# ---------------------------------------------------------------------------
+# error paths (all on the host)
+# ---------------------------------------------------------------------------
+def _code(fn):
+    with pytest.raises(B.AmapError) as e:
+        fn()
+    return e.value.code
+
+
+def test_error_codes():
+    eye = [[1, 0], [0, 1]]
+
+    def non_injective():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, [[1, 0]], [0]))  # the second loop never moves the store
+        b.compose(t)
+
+    assert _code(non_injective) == -2
+
+    def interleaved_collision():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([16])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, [[2, 3]], [0]))  # 2a + 3b collides (a,b) = (3,0) and (0,2)
+        b.compose(t)
+
+    assert _code(interleaved_collision) == -2
+
+    def load_escapes():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4, 4])
+        b.stmt([4, 4], (x, eye, [1, 0]), (t, eye, [0, 0]))
+        b.compose(t)
+
+    assert _code(load_escapes) == -3
+
+    def store_escapes():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4, 4])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, eye, [0, 1]))
+        b.compose(t)
+
+    assert _code(store_escapes) == -3
+
+    def output_partly_written():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4, 5])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, eye, [0, 0]))
+        b.compose(t)
+
+    assert _code(output_partly_written) == -4
+
+    def reads_unwritten_intermediate():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4, 5])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, eye, [0, 0]))
+        b.compose(b.transpose(t, [1, 0]))
+
+    assert _code(reads_unwritten_intermediate) == -4
+
+    def overlap():
+        b = B.Builder(4)
+        x = b.input([4, 4])
+        t = b.tensor([4, 6])
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, eye, [0, 0]))
+        b.stmt([4, 4], (x, eye, [0, 0]), (t, eye, [0, 2]))
+        b.compose(t)
+
+    assert _code(overlap) == -5
+
+    assert _code(lambda: B.Builder(3)) == -1
+    assert _code(lambda: B.Builder(4).reshape(0, [2])) == -1  # no such tensor
+
+    def reshape_that_does_not_factor():
+        b = B.Builder(4)
+        x = b.input([2, 3])
+        b.reshape(x, [3, 2])
+
+    assert _code(reshape_that_does_not_factor) == -9
+
+
+def test_interleaved_stores_are_told_apart_from_overlap():
+    b = B.Builder(2)
+    x0, x1 = b.input([8]), b.input([8])
+    t = b.tensor([16])
+    b.stmt([8], (x0, [[1]], [0]), (t, [[2]], [0]))
+    b.stmt([8], (x1, [[1]], [0]), (t, [[2]], [1]))
+    m = b.compose(b.reshape(t, [4, 4]))
+    a, c = np.arange(8, dtype=np.uint16) + 100, np.arange(8, dtype=np.uint16) + 200
+    want = np.empty(16, np.uint16)
+    want[0::2], want[1::2] = a, c
+    assert np.array_equal(eval_map(m, [a, c]), want)
+
+
+def test_empty_and_scalar_shapes():
+    b = B.Builder(2)
+    x = b.input([1, 1])
+    m = b.compose(b.transpose(x, [1, 0]))
+    assert np.array_equal(eval_map(m, [np.array([[9]], np.uint16)]), [9])
+    b = B.Builder(2)
+    x = b.input([0, 3])
+    m = b.compose(b.transpose(x, [1, 0]))
+    assert m.out_numel == 0 and m.pieces() == []
+
+
+# ---------------------------------------------------------------------------
+# the C ABI
+# ---------------------------------------------------------------------------
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "amap.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(amap_[a-z_]+)\s*\(", header))
+    assert declared and declared == set(B.EXPORTS), declared ^ set(B.EXPORTS)
+    import ctypes
+
+    lib = ctypes.CDLL(B.LIBRARY_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert lib.amap_strerror  # loads without a GPU
+
+
+def test_strerror_is_distinct_per_code():
+    import ctypes
+
+    lib = ctypes.CDLL(B.LIBRARY_PATH)
+    lib.amap_strerror.restype = ctypes.c_char_p
+    msgs = {lib.amap_strerror(c) for c in range(0, -11, -1)}
+    assert len(msgs) == 11

@@ -1,0 +1,158 @@
+"""Parity of the CUDA path with the CPU oracle, bit for bit, through the C ABI."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import oracle
+from paper_2002_12798_b200 import workloads as W
+from chain_gen import random_chain
+
+pytestmark = pytest.mark.gpu
+
+SIGNED = {1: np.int8, 2: np.int16, 4: np.int32, 8: np.int64}
+CANARY = 64  # elements of guard band on both sides of the output
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2002_12798_b200 import binding
+
+    return binding
+
+
+def run_gpu(B, chain, xs, force=0, align=16):
+    """compose -> plan -> execute on cuda:0; returns the output as a flat numpy array of raw bits."""
+    import torch
+
+    m = B.compose_chain(chain)
+    plan = m.plan(device=0, force_kernel=force, pointer_align=align)
+    es = chain.elem_size
+    dev = [torch.from_numpy(np.ascontiguousarray(x).view(SIGNED[es])).cuda() for x in xs]
+    band = torch.full(((m.out_numel + 2 * CANARY) * es,), 0x5A, dtype=torch.uint8, device="cuda")
+    out = band[CANARY * es : (CANARY + m.out_numel) * es]
+    assert out.data_ptr() % 16 == 0 or align < 16
+    plan.execute_ptrs([d.data_ptr() for d in dev], out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    host = band.cpu().numpy()
+    assert (host[: CANARY * es] == 0x5A).all() and (host[(CANARY + m.out_numel) * es :] == 0x5A).all(), "wrote outside the output"
+    return host[CANARY * es : (CANARY + m.out_numel) * es].view(xs[0].dtype), plan
+
+
+@pytest.mark.parametrize("force", [0, 1], ids=["auto", "gather"])
+@pytest.mark.parametrize("name", sorted(W.reduced_configs()))
+def test_reduced_configs_bit_exact(B, name, force):
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, _ = run_gpu(B, chain, xs, force=force)
+    assert np.array_equal(got, want.reshape(-1))
+
+
+@pytest.mark.parametrize("name", ["c1", "c2_fwd", "c3_odd", "c4_odd", "c5_odd"])
+def test_index_tagged_inputs(B, name):
+    """With inputs that hold their own index the output IS the composed source-index map."""
+    chain = W.reduced_configs()[name]
+    for part in (0, 1):
+        xs = W.make_index_tagged_inputs(chain, part)
+        want = oracle.run_chain(chain, xs)
+        got, _ = run_gpu(B, chain, xs)
+        assert np.array_equal(got, want.reshape(-1))
+
+
+def test_c1_closed_form_on_the_gpu(B):
+    chain = W.c1_small_chain()
+    got, _ = run_gpu(B, chain, W.make_index_tagged_inputs(chain))
+    a, j, k = np.meshgrid(np.arange(64), np.arange(8), np.arange(6), indexing="ij")
+    want = np.zeros((64, 48), dtype=np.int64)
+    want[a, 6 * j + k] = 1024 * j + 128 * k + 128 + 2 * a
+    assert np.array_equal(got.astype(np.int64).reshape(64, 48), want)
+
+
+def test_random_tiny_chains(B):
+    r = np.random.default_rng(20021279)
+    done = 0
+    for trial in range(120):
+        chain = random_chain(r)
+        xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
+        try:
+            B.compose_chain(chain)
+        except B.AmapError as e:
+            assert e.code == -9
+            continue
+        want = oracle.run_chain(chain, xs)
+        for force in (0, 1):
+            got, _ = run_gpu(B, chain, xs, force=force)
+            assert np.array_equal(got, want.reshape(-1)), (trial, force, chain.ops)
+        done += 1
+    assert done >= 60
+
+
+@pytest.mark.parametrize("dtype,es", [("u8", 1), ("u64", 8)])
+def test_other_element_sizes(B, dtype, es):
+    chain = W.c3_head_split(B=2, S=20, heads=3, D=16, keep=11, dtype=dtype)
+    chain.values = "raw"
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, _ = run_gpu(B, chain, xs)
+    assert np.array_equal(got, want.reshape(-1))
+
+
+def test_execute_host_matches(B):
+    chain = W.reduced_configs()["c4_odd"]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    m = B.compose_chain(chain)
+    plan = m.plan(0)
+    out = np.empty(m.out_numel, dtype=xs[0].dtype)
+    plan.execute_host([np.ascontiguousarray(x) for x in xs], out)
+    assert np.array_equal(out, want.reshape(-1))
+    out[:] = 0
+    plan.execute_host([np.ascontiguousarray(x) for x in xs], out)  # staging buffers are reused
+    assert np.array_equal(out, want.reshape(-1))
+
+
+def test_misaligned_pointer_is_refused(B):
+    import torch
+
+    chain = W.reduced_configs()["c3"]
+    m = B.compose_chain(chain)
+    plan = m.plan(0, pointer_align=16)
+    buf = torch.zeros(m.out_numel * 2 + 64, dtype=torch.uint8, device="cuda")
+    srcs = [torch.zeros(n * 2, dtype=torch.uint8, device="cuda") for n in m.in_numel]
+    with pytest.raises(B.AmapError) as e:
+        plan.execute_ptrs([s.data_ptr() for s in srcs], buf.data_ptr() + 2, 0)
+    assert e.value.code == -7
+    # a plan that promises only element alignment accepts it and still copies exactly
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    plan2 = m.plan(0, pointer_align=2)
+    dev = [torch.from_numpy(x.view(np.int16)).cuda() for x in xs]
+    plan2.execute_ptrs([d.data_ptr() for d in dev], buf.data_ptr() + 2, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    got = buf.cpu().numpy()[2 : 2 + m.out_numel * 2].view(np.uint16)
+    assert np.array_equal(got, want.reshape(-1))
+
+
+def test_plan_stats_count_algorithmic_bytes(B):
+    full = W.full_configs()
+    want = {
+        "c2_fwd": (51380224, 51380224, 0),
+        "c3": (402653184, 402653184, 0),
+        "c4": (32112640, 36864000, 2375680 * 2),
+        "c5": (51380224, 462422016, 0),
+    }
+    for name, (rd, wr, fl) in want.items():
+        st = B.compose_chain(full[name]).plan(0).stats()
+        assert (st["bytes_read"], st["bytes_written"], st["bytes_filled"]) == (rd, wr, fl), (name, st)
+
+
+@pytest.mark.parametrize("name", ["c2_fwd", "c2_inv", "c3", "c3_merge", "c4", "c5"])
+def test_full_size_configs_bit_exact(B, name):
+    """The sizes and launch configuration the benchmark times."""
+    chain = W.full_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs, nt=min(os.cpu_count() or 1, 32))
+    got, plan = run_gpu(B, chain, xs)
+    assert np.array_equal(got, want.reshape(-1))
+    del want, got

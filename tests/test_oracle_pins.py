@@ -9,6 +9,7 @@ import pytest
 
 from oracle import oracle
 from paper_2002_12798_b200 import workloads as W
+from chain_gen import random_chain
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 rng = np.random.default_rng(7)
@@ -309,59 +310,6 @@ def _python_chain(chain, inputs):
             t = np.pad(ts[op["src"]], list(zip(op["lo"], op["hi"])))
         ts.append(np.ascontiguousarray(t))
     return ts[-1]
-
-
-def random_chain(r, n_ops=4, max_extent=5, max_rank=4):
-    """A random chain of <= n_ops operators over one or two tiny inputs."""
-    rank = int(r.integers(1, max_rank + 1))
-    shape = [int(r.integers(1, max_extent + 1)) for _ in range(rank)]
-    inputs = [shape]
-    ops = []
-    cur, cur_shape = 0, list(shape)
-    for _ in range(n_ops):
-        kind = r.choice(["reshape", "transpose", "slice", "pad", "concat"])
-        tid = len(inputs) + len(ops)
-        if kind == "reshape":
-            n = int(np.prod(cur_shape))
-            facs = []
-            rem = n
-            for _ in range(int(r.integers(1, 4))):
-                divs = [d for d in range(1, rem + 1) if rem % d == 0]
-                f = int(r.choice(divs))
-                facs.append(f)
-                rem //= f
-            facs.append(rem)
-            r.shuffle(facs)
-            ops.append({"kind": "reshape", "src": cur, "shape": [int(f) for f in facs]})
-            cur_shape = [int(f) for f in facs]
-        elif kind == "transpose":
-            perm = [int(p) for p in r.permutation(len(cur_shape))]
-            ops.append({"kind": "transpose", "src": cur, "perm": perm})
-            cur_shape = [cur_shape[p] for p in perm]
-        elif kind == "slice":
-            start, stop, step = [], [], []
-            for n in cur_shape:
-                a = int(r.integers(0, n))
-                b = int(r.integers(a + 1, n + 1))
-                s = int(r.integers(1, 3))
-                start.append(a), stop.append(b), step.append(s)
-            ops.append({"kind": "slice", "src": cur, "start": start, "stop": stop, "step": step})
-            cur_shape = [-(-(b - a) // s) for a, b, s in zip(start, stop, step)]
-        elif kind == "pad":
-            lo = [int(r.integers(0, 2)) for _ in cur_shape]
-            hi = [int(r.integers(0, 2)) for _ in cur_shape]
-            ops.append({"kind": "pad", "src": cur, "lo": lo, "hi": hi})
-            cur_shape = [a + n + b for a, n, b in zip(lo, cur_shape, hi)]
-        else:  # concat the current tensor with itself or with the first input when shapes allow
-            axis = int(r.integers(0, len(cur_shape)))
-            other = cur
-            ops.append({"kind": "concat", "srcs": [cur, other], "axis": axis})
-            cur_shape = list(cur_shape)
-            cur_shape[axis] *= 2
-        cur = tid
-        if int(np.prod(cur_shape)) > 4000:
-            break
-    return W.Chain(name="random", dtype="fp32", inputs=inputs, ops=ops, values="raw")
 
 
 def test_random_tiny_chains_against_numpy():
