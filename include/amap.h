@@ -171,10 +171,15 @@ int amap_map_sizes(const amap_map *map, int32_t *n_inputs, int64_t *in_numel /* 
 
 /* ---------------------------------------------------------------------------
  * amap_plan: choose a kernel family per piece and build the launch table.
- * Needs a CUDA device: `device` is a CUDA ordinal; the call makes it current,
- * uploads a small descriptor table to device memory owned by the plan, and
- * restores the previous device.  A plan is immutable and may be executed any
- * number of times, on any stream of that device, concurrently.
+ * `device` is a CUDA ordinal: the call makes it current, uploads a small
+ * descriptor table to device memory owned by the plan, and restores the
+ * previous device.  device = -1 gives a dry plan (no CUDA call at all) whose
+ * statistics and kernel choices can be read but which amap_execute refuses
+ * with AMAP_EINVAL.  Before anything is uploaded the planner walks the table
+ * on the host with the kernel's own index arithmetic and checks that every
+ * address stays inside its buffer and is aligned to the access width; a
+ * violation gives AMAP_EOVERFLOW.  A plan is immutable and may be executed
+ * any number of times, on any stream of its device, concurrently.
  * ------------------------------------------------------------------------- */
 typedef enum amap_kernel_kind {
   AMAP_KERNEL_AUTO = 0,

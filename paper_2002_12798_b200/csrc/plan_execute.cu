@@ -128,8 +128,9 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
     if (k == p.n() - 1) e /= q;
     d->ext[j] = (uint32_t)e;
     d->fd[j] = make_fastdiv((uint32_t)e);
-    d->sstride[j] = (p.src == AMAP_CONST) ? 0 : p.srcoff.c[k] * es;
-    d->dstride[j] = p.dst.c[k] * es;
+    const int64_t unit = (k == p.n() - 1) ? V : es;  // the innermost loop steps by whole units
+    d->sstride[j] = (p.src == AMAP_CONST) ? 0 : p.srcoff.c[k] * unit;
+    d->dstride[j] = p.dst.c[k] * unit;
     items *= (uint64_t)e;
   }
   if (items >= (1ull << 32) - (uint64_t)kAffineThreads * kUnroll) return AMAP_EUNSUPPORTED;
@@ -157,6 +158,66 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
   return AMAP_OK;
 }
 
+// Walks a device descriptor on the HOST with the kernel's own arithmetic and
+// checks every address it would form: inside its buffer and aligned to the
+// unit.  Small pieces are walked completely, large ones at their first and
+// last items and a pseudo-random sample.  A failure here is a planner bug and
+// is reported instead of being launched.
+static uint32_t host_fast_div(uint32_t n, const FastDiv &f) {
+  const uint32_t t = (uint32_t)(((uint64_t)f.mul * n) >> 32);
+  return (t + ((n - t) >> f.sh1)) >> f.sh2;
+}
+
+static bool check_affine_item(const DevPiece &d, uint64_t L, int64_t in_bytes, int64_t out_bytes) {
+  uint32_t rem = (uint32_t)L;
+  int64_t s = d.soff, o = d.doff;
+  int64_t acc[kDevMaxCons] = {0};
+  const int nc = d.n_guards + d.n_domain;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    const uint32_t q = host_fast_div(rem, d.fd[k]);
+    if (q != rem / d.ext[k]) return false;
+    const uint32_t i = rem - q * d.ext[k];
+    rem = q;
+    s += (int64_t)i * d.sstride[k];
+    o += (int64_t)i * d.dstride[k];
+    for (int c = 0; c < nc; ++c) acc[c] += (int64_t)d.cons[c].coef[k] * i;
+  }
+  if (rem != 0) return false;
+  bool load = d.input >= 0, live = true;
+  for (int c = 0; c < nc; ++c) {
+    const int64_t v = acc[c] + d.cons[c].off;
+    const bool ok = v >= 0 && v < d.cons[c].extent;
+    if (c < d.n_guards) load = load && ok; else live = live && ok;
+  }
+  if (!live) return true;
+  const int V = d.unit_bytes;
+  if (o % V || o < 0 || o + V > out_bytes) return false;
+  if (load && (s % V || s < 0 || s + V > in_bytes)) return false;
+  return true;
+}
+
+static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_bytes) {
+  if (d.n_items == 0) return true;
+  if (d.n_items <= (1u << 18)) {
+    for (uint64_t L = 0; L < d.n_items; ++L)
+      if (!check_affine_item(d, L, in_bytes, out_bytes)) return false;
+    return true;
+  }
+  uint64_t x = 0x9E3779B97F4A7C15ull;
+  for (int t = 0; t < (1 << 16); ++t) {
+    x ^= x << 13; x ^= x >> 7; x ^= x << 17;  // xorshift64
+    uint64_t L = (t == 0) ? 0 : (t == 1) ? d.n_items - 1 : x % d.n_items;
+    if (!check_affine_item(d, L, in_bytes, out_bytes)) return false;
+  }
+  // the far corner of every loop on its own
+  uint64_t mult = 1;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    if (!check_affine_item(d, mult * (d.ext[k] - 1), in_bytes, out_bytes)) return false;
+    mult *= d.ext[k];
+  }
+  return true;
+}
+
 extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts, amap_plan_t **out_plan) {
   if (!map || !out_plan) return AMAP_EINVAL;
   amap_plan_opts o;
@@ -171,9 +232,12 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   if (align < es || (align & (align - 1))) return AMAP_EINVAL;
   if ((int)m.in_numel.size() > kMaxInputs) return AMAP_EUNSUPPORTED;
 
-  int n_dev = 0;
-  CUDA_TRY(cudaGetDeviceCount(&n_dev));
-  if (device < 0 || device >= n_dev) return AMAP_EINVAL;
+  if (device < -1) return AMAP_EINVAL;
+  if (device >= 0) {
+    int n_dev = 0;
+    CUDA_TRY(cudaGetDeviceCount(&n_dev));
+    if (device >= n_dev) return AMAP_EINVAL;
+  }
 
   amap_plan_t *pl = new (std::nothrow) amap_plan_t();
   if (!pl) return AMAP_ENOMEM;
@@ -218,6 +282,12 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
         return rc;
       }
       if (d.n_items == 0) continue;
+      const int64_t in_bytes = (d.input >= 0) ? m.in_numel[d.input] * es : 0;
+      if (!check_affine_piece(d, in_bytes, m.out_numel * es)) {
+        if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] plan self-check failed on piece %zu\n", q);
+        delete pl;
+        return AMAP_EOVERFLOW;
+      }
       if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) {
         delete pl;
         return AMAP_EUNSUPPORTED;
@@ -235,6 +305,10 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
 
+  if (device < 0) {  // a dry plan: can be inspected, not executed
+    *out_plan = pl;
+    return AMAP_OK;
+  }
   int prev = 0;
   cudaError_t e = cudaGetDevice(&prev);
   if (e == cudaSuccess) e = cudaSetDevice(device);
@@ -255,6 +329,10 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
 
 extern "C" void amap_plan_destroy(amap_plan_t *plan) {
   if (!plan) return;
+  if (plan->device < 0) {
+    delete plan;
+    return;
+  }
   int prev = 0;
   cudaGetDevice(&prev);
   cudaSetDevice(plan->device);
@@ -286,7 +364,7 @@ static cudaError_t launch_affine(const amap_plan_t *pl, const Launch &L, const P
 
 extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
                             void *cuda_stream) {
-  if (!plan || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
+  if (!plan || plan->device < 0 || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
   if (plan->out_numel == 0) return AMAP_OK;
   if (!dst_dev_ptr) return AMAP_EINVAL;
   PtrTable pt;
@@ -324,7 +402,8 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
 
 extern "C" int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr,
                                  void *cuda_stream) {
-  if (!plan || (!src_host_ptrs && !plan->in_numel.empty()) || (!dst_host_ptr && plan->out_numel > 0)) return AMAP_EINVAL;
+  if (!plan || plan->device < 0 || (!src_host_ptrs && !plan->in_numel.empty()) || (!dst_host_ptr && plan->out_numel > 0))
+    return AMAP_EINVAL;
   int prev = 0;
   CUDA_TRY(cudaGetDevice(&prev));
   CUDA_TRY(cudaSetDevice(plan->device));
