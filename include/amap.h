@@ -42,7 +42,8 @@ typedef enum amap_status {
   AMAP_EALIGN = -7,               /* a device pointer is less aligned than the plan requires       */
   AMAP_ECUDA = -8,                /* a CUDA runtime call failed; see amap_last_cuda_error()        */
   AMAP_EUNSUPPORTED = -9,         /* valid input the host algebra cannot compose affinely          */
-  AMAP_ENOMEM = -10
+  AMAP_ENOMEM = -10,
+  AMAP_ETOOLARGE = -11            /* the plan does not fit the fixed table of amap_execute_static   */
 } amap_status;
 
 #define AMAP_CONST (-1) /* amap_access.tensor of a load that yields the statement's fill_bits */
@@ -231,6 +232,39 @@ int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void 
  * pointers; dst_host_ptr: HOST.  Pinned host memory makes the copies faster
  * but is not required. */
 int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * amap_execute_static: amap_execute for callers that are not allowed to
+ * allocate device memory.  (The paper has no counterpart; this is a service of
+ * the library.)  Typical callers: a plug-in running inside a framework that
+ * owns all device memory, a real-time or serving loop in which cudaMalloc's
+ * implicit device-wide synchronisation is not acceptable, code that runs after
+ * the memory budget has been handed out.  Such a caller makes a DRY plan
+ * (amap_plan with device = -1, which touches no CUDA API) and passes it here;
+ * a plan made for the current device is accepted too.
+ *
+ * Instead of the plan's own table in cudaMalloc'ed memory, the kernels read
+ * their descriptors from a fixed array that is part of the library image
+ * (64 descriptors, about 70 KB; every GPU on which the library is loaded
+ * holds it until the process exits).  The call copies the plan's descriptors
+ * into that array on `cuda_stream` and enqueues the same kernels as
+ * amap_execute behind the copy.  It calls no cudaMalloc / cudaFree and no
+ * allocating library routine, and does not synchronise.
+ *
+ *  - Runs on the CURRENT device; src/dst pointers and the stream must belong
+ *    to it.  Arguments and alignment rules are those of amap_execute.
+ *  - A plan with more than 64 descriptors is refused with AMAP_ETOOLARGE and
+ *    nothing is enqueued (compose fewer operators per call, or use amap_execute).
+ *  - The first call on each device looks up the array's device address
+ *    (cudaGetSymbolAddress); make that first call before starting any stream
+ *    capture on that device.
+ *  - All calls on one device share the one array, which still holds the
+ *    previous call's descriptors until the next copy overwrites them.  Calls
+ *    are safe back to back on ONE stream.  Two calls that can overlap on the
+ *    GPU (different streams without an ordering between them) race on the
+ *    array: order them with events or use amap_execute for one of them.
+ * ------------------------------------------------------------------------- */
+int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, void *cuda_stream);
 
 const char *amap_strerror(int code);
 /* text of the last CUDA error seen by this thread in this library ("" if none) */

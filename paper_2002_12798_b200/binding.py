@@ -24,7 +24,7 @@ EXPORTS = [
     "amap_builder_window", "amap_builder_tile", "amap_builder_tensor", "amap_builder_stmt",
     "amap_builder_chain", "amap_compose", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
-    "amap_execute", "amap_execute_host", "amap_strerror", "amap_last_cuda_error",
+    "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
 
 
@@ -87,6 +87,7 @@ def _load():
     lib.amap_builder_pad.argtypes = [c_void_p, c_int32, c_int32, POINTER(c_int64), POINTER(c_int64), c_uint64, POINTER(c_int32)]
     lib.amap_execute.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
     lib.amap_execute_host.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
+    lib.amap_execute_static.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
     return lib
 
 
@@ -284,6 +285,11 @@ class Plan:
     def execute_ptrs(self, src_ptrs, dst_ptr, stream=0):
         arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
         _check(_lib.amap_execute(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute")
+
+    def execute_static_ptrs(self, src_ptrs, dst_ptr, stream=0):
+        """amap_execute_static: no device allocation; the descriptors go through the library's fixed table."""
+        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        _check(_lib.amap_execute_static(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute_static")
 
     def execute(self, srcs, dst, stream=None):
         """srcs: CUDA tensors (contiguous), dst: CUDA tensor; stream: torch.cuda.Stream or None (current)."""

@@ -738,6 +738,7 @@ extern "C" const char *amap_strerror(int code) {
     case AMAP_ECUDA: return "a CUDA call failed";
     case AMAP_EUNSUPPORTED: return "the maps cannot be composed affinely by this library";
     case AMAP_ENOMEM: return "out of memory";
+    case AMAP_ETOOLARGE: return "the plan has more descriptors than the fixed table of amap_execute_static holds";
   }
   return "unknown amap status";
 }

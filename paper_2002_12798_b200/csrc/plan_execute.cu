@@ -428,3 +428,76 @@ extern "C" int amap_execute_host(amap_plan_t *plan, const void *const *src_host_
   if (e != cudaSuccess) return cuda_fail(e, "amap_execute_host");
   return rc;
 }
+
+// ---------------------------------------------------------------------------
+// amap_execute_static: the same copy for callers that must not allocate.
+// The descriptor table, which amap_plan normally places in memory it gets from
+// cudaMalloc, is kept in a fixed array inside the library image instead.
+// ---------------------------------------------------------------------------
+static const int kStaticMaxPieces = 64;
+static __device__ __align__(256) unsigned char g_static_table[kStaticMaxPieces * sizeof(DevPiece)];
+
+static const int kStaticMaxDevices = 64;
+static void *g_static_table_addr[kStaticMaxDevices];  // device address of g_static_table, per device, 0 = not set up
+
+// In host code `g_static_table` is only a handle for the runtime; the address the
+// kernels need comes from cudaGetSymbolAddress, once per device, with that device current.
+static int static_table_address(int device, void **out) {
+  if (device < 0 || device >= kStaticMaxDevices) return AMAP_EINVAL;
+  void *p = __atomic_load_n(&g_static_table_addr[device], __ATOMIC_ACQUIRE);
+  if (!p) {
+    cudaError_t e = cudaGetSymbolAddress(&p, g_static_table);
+    if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: cudaGetSymbolAddress");
+    if (!p) return AMAP_ECUDA;
+    __atomic_store_n(&g_static_table_addr[device], p, __ATOMIC_RELEASE);
+  }
+  *out = p;
+  return AMAP_OK;
+}
+
+template <int V>
+static cudaError_t launch_affine_at(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
+  amap_affine_kernel<V, kUnroll><<<L.n_blocks, kAffineThreads, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  return cudaGetLastError();
+}
+
+extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
+                                   void *cuda_stream) {
+  if (!plan || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
+  if (plan->table.size() > (size_t)kStaticMaxPieces) return AMAP_ETOOLARGE;
+  if (plan->out_numel == 0) return AMAP_OK;
+  if (!dst_dev_ptr) return AMAP_EINVAL;
+  PtrTable pt;
+  memset(&pt, 0, sizeof pt);
+  const uintptr_t mask = (uintptr_t)plan->pointer_align - 1;
+  for (size_t q = 0; q < plan->in_numel.size(); ++q) {
+    if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
+    if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
+    if (src_dev_ptrs[q] == dst_dev_ptr) return AMAP_EINVAL;
+    pt.src[q] = (const char *)src_dev_ptrs[q];
+  }
+  if ((uintptr_t)dst_dev_ptr & mask) return AMAP_EALIGN;
+  pt.dst = (char *)dst_dev_ptr;
+  int device = 0;
+  CUDA_TRY(cudaGetDevice(&device));
+  if (plan->device >= 0 && plan->device != device) return AMAP_EINVAL;
+  void *table = nullptr;
+  const int rc = static_table_address(device, &table);
+  if (rc != AMAP_OK) return rc;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  // the part of the array this plan uses is overwritten in full; nothing in it needs to start at zero
+  CUDA_TRY(cudaMemcpyAsync(table, plan->table.data(), plan->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice, s));
+  for (const Launch &L : plan->launches) {
+    cudaError_t e = cudaSuccess;
+    const DevPiece *t = (const DevPiece *)table;
+    switch (L.unit) {
+      case 16: e = launch_affine_at<16>(t, L, pt, s); break;
+      case 8: e = launch_affine_at<8>(t, L, pt, s); break;
+      case 4: e = launch_affine_at<4>(t, L, pt, s); break;
+      case 2: e = launch_affine_at<2>(t, L, pt, s); break;
+      default: e = launch_affine_at<1>(t, L, pt, s); break;
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: kernel launch");
+  }
+  return AMAP_OK;
+}

@@ -1,0 +1,67 @@
+"""amap_execute_static: the entry point for callers that may not allocate device memory
+(a plug-in inside a framework that owns the GPU's memory, a serving loop that cannot
+afford cudaMalloc's device-wide synchronisation).  It must produce exactly what
+amap_execute produces, call after call, although every call reuses one fixed descriptor
+table inside the library.  Collected last on purpose (file name)."""
+import numpy as np
+import pytest
+
+from paper_2002_12798_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+SIGNED = {1: np.int8, 2: np.int16, 4: np.int32, 8: np.int64}
+
+
+def _both_ways(B, torch, chain):
+    xs = W.make_inputs(chain)
+    m = B.compose_chain(chain)
+    es = chain.elem_size
+    dev = [torch.from_numpy(np.ascontiguousarray(x).view(SIGNED[es])).cuda() for x in xs]
+    ptrs = [d.data_ptr() for d in dev]
+    stream = torch.cuda.current_stream().cuda_stream
+    ref = torch.full((m.out_numel,), 0x11, dtype=dev[0].dtype, device="cuda")
+    m.plan(device=0).execute_ptrs(ptrs, ref.data_ptr(), stream)  # the existing entry point
+    out = torch.full((m.out_numel,), 0x22, dtype=dev[0].dtype, device="cuda")
+    dry = m.plan(device=-1)  # a plan made without touching CUDA
+    dry.execute_static_ptrs(ptrs, out.data_ptr(), stream)
+    torch.cuda.synchronize()
+    return ref, out, dry, dev, stream  # dev is returned so that the inputs stay allocated
+
+
+def test_static_table_matches_amap_execute_on_calls_in_a_row():
+    import torch
+
+    from paper_2002_12798_b200 import binding as B
+
+    cfg = W.reduced_configs()
+    # different maps one after the other: each call finds the previous call's descriptors in the table
+    for name in ("c3", "c4_odd", "c5", "c1", "c3"):
+        ref, out, dry, dev, stream = _both_ways(B, torch, cfg[name])
+        ptrs = [d.data_ptr() for d in dev]
+        assert torch.equal(ref, out), name  # pure copies: bit-exact
+        # and the same plan twice in a row into a fresh buffer
+        again = torch.zeros_like(out)
+        dry.execute_static_ptrs(ptrs, again.data_ptr(), stream)
+        dry.execute_static_ptrs(ptrs, again.data_ptr(), stream)
+        torch.cuda.synchronize()
+        assert torch.equal(ref, again), name
+
+
+def test_static_table_refuses_a_plan_that_does_not_fit():
+    import torch
+
+    from paper_2002_12798_b200 import binding as B
+
+    # 14 inputs, each padded on both axes (1 copy + 4 border pieces), joined: 70 pieces > the table's 64 descriptors
+    n_in = 14
+    b = B.Builder(2)
+    ids = [b.input([4, 8]) for _ in range(n_in)]
+    m = b.compose(b.concat([b.pad(t, [1, 1], [1, 1]) for t in ids], 0))
+    dry = m.plan(device=-1)
+    assert dry.stats()["n_pieces"] > 64
+    srcs = [torch.zeros(32, dtype=torch.int16, device="cuda") for _ in range(n_in)]
+    out = torch.zeros(m.out_numel, dtype=torch.int16, device="cuda")
+    with pytest.raises(B.AmapError) as e:
+        dry.execute_static_ptrs([s.data_ptr() for s in srcs], out.data_ptr(), 0)
+    assert e.value.code == -11
