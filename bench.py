@@ -304,7 +304,12 @@ def cpu_baseline(oracle, fwd_c, inv_c, x, bytes_per_step, budget_s=20.0):
 def all_configs(torch, B, device, stream, l2, peak):
     """Every large configuration, each timed the same way (device time per launch, rotating buffers)."""
     out = {}
-    for name, chain in W.full_configs().items():
+    configs = dict(W.full_configs())
+    # the practical ceiling: a same-kernel plain copy (a reshape composes to one contiguous piece)
+    configs["plain_copy_512MB"] = W.Chain(
+        name="plain_copy", dtype="bf16", inputs=[[1 << 28]], ops=[{"kind": "reshape", "src": 0, "shape": [1 << 14, 1 << 14]}]
+    )
+    for name, chain in configs.items():
         if name == "c1":
             continue
         xs = W.make_inputs(chain)

@@ -16,18 +16,32 @@ struct FastDiv {
   uint32_t mul, sh1, sh2, d;
 };
 
-struct DevCon {  // 0 <= off + sum coef[k] * i_k < extent
-  int64_t off;
-  int64_t extent;
+struct DevCon {  // 0 <= off + sum coef[k] * i_k < extent   (all values fit 32 bits; the planner checks)
+  int32_t off;
+  int32_t extent;
   int32_t coef[kDevMaxLoops];
 };
 
 enum DevKind : int32_t { kDevAffine = 0, kDevTranspose = 1 };
 
+// Transpose tiles: 8 chunks of 16 bytes of the destination-contiguous index a
+// (128 bytes) by kTileB elements of the source-contiguous index b.
+constexpr int kTileB = 128;
+constexpr int kTileBytes = 16384;
+constexpr int kTransposeThreads = 256;
+
 // One piece of a composed map, ready to run.  Loops are in canonical order
-// (destination stride descending).  For the affine kernel one "item" is one
-// unit of `unit_bytes` bytes; the innermost loop counts units and all strides
-// and offsets are in BYTES.
+// (destination stride descending).  All strides and offsets are in BYTES.
+//
+// Affine kernel: one item = one unit of `unit_bytes` bytes; the innermost loop
+// counts units; ext/fd/sstride/dstride describe all loops.
+//
+// Transpose kernel: ext/fd/sstride/dstride describe the BATCH loops only.  The
+// tile indices are a (contiguous in the destination) and b (contiguous in the
+// source); each may merge two loops of the piece: a = a_hi * a_in + a_lo with
+// source offset a_lo * sa[0] + a_hi * sa[1] and destination offset a * es;
+// b = b_hi * b_in + b_lo with destination offset b_lo * db[0] + b_hi * db[1]
+// and source offset b * es.
 struct DevPiece {
   int32_t kind;
   int32_t n_loops;
@@ -46,12 +60,12 @@ struct DevPiece {
   int64_t dstride[kDevMaxLoops];
   DevCon cons[kDevMaxCons];  // guards first, then domain constraints
   // --- transpose kernel only -------------------------------------------
-  // Tile = TA elements of loop `la` (destination-contiguous) x TB elements of
-  // loop `lb` (source-contiguous); the remaining loops are the batch.
-  int32_t la, lb;
-  uint32_t tiles_a, tiles_b;  // tiles along la / lb
+  uint32_t ext_a, ext_b;      // merged extents, in elements
+  uint32_t tiles_a, tiles_b;  // tiles along a / b
   FastDiv fd_tiles_a, fd_tiles_b;
-  int32_t pad_[2];
+  FastDiv fd_a_in, fd_b_in;  // inner extents of the merged indices
+  int64_t sa[2];             // source byte strides of (a_lo, a_hi)
+  int64_t db[2];             // destination byte strides of (b_lo, b_hi)
 };
 
 struct PtrTable {

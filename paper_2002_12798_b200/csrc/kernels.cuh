@@ -61,68 +61,210 @@ __device__ __forceinline__ void fetch_piece(const DevPiece *__restrict__ table, 
 // destination byte offsets  b + sum_k stride_k * i_k  of the composed map.
 // With V = 16 and a contiguous innermost loop this is the coalesced streaming
 // copy; with V = elem_size and arbitrary strides it is the gather that handles
-// every piece, including non-injective loads (overlapping windows).  All U
-// loads are issued before the first store so that each thread keeps U
-// independent requests in flight.
+// every piece, including non-injective loads (overlapping windows) and guards
+// (out-of-range loads give the fill value).  All U loads are issued before the
+// first store so that each thread keeps U independent requests in flight; the
+// loop over the nest is outermost so that each descriptor field is fetched
+// once for the U units.
+//   NC   : 0 = the piece has no constraints; otherwise the table's guards and
+//          domain constraints (at most kDevMaxCons) are evaluated per unit.
+//   OffT : uint32_t when every byte offset is below 4 GiB (wrap-around
+//          arithmetic keeps intermediate negative values exact), else int64_t.
 // ---------------------------------------------------------------------------
 constexpr int kAffineThreads = 256;
 
-template <int V, int U>
+template <int V, int U, int NC, typename OffT>
 __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPiece *__restrict__ table, int first_piece,
                                                                       int n_pieces, PtrTable ptrs) {
   __shared__ DevPiece sp;
   fetch_piece(table, first_piece, n_pieces, &sp);
   using T = typename Unit<V>::T;
   const int n = sp.n_loops;
-  const int n_cons = sp.n_guards + sp.n_domain;
   const uint64_t item0 = (uint64_t)(blockIdx.x - sp.first_block) * (uint64_t)(kAffineThreads * U) + threadIdx.x;
   const char *src = (sp.input >= 0) ? ptrs.src[sp.input] : nullptr;
   char *dst = ptrs.dst;
 
-  int64_t so[U], doff[U];
-  bool live[U], load[U];
+  uint32_t rem[U];
+  OffT so[U], doff[U];
+  bool live[U];
+  int32_t acc[U][NC > 0 ? NC : 1];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     const uint64_t L = item0 + (uint64_t)u * kAffineThreads;
     live[u] = L < sp.n_items;
-    load[u] = live[u] && (src != nullptr);
-    uint32_t rem = live[u] ? (uint32_t)L : 0u;
-    int64_t s = sp.soff, d = sp.doff;
-    int64_t acc[kDevMaxCons];
+    rem[u] = live[u] ? (uint32_t)L : 0u;
+    so[u] = (OffT)sp.soff;
+    doff[u] = (OffT)sp.doff;
+    if constexpr (NC > 0) {
 #pragma unroll
-    for (int c = 0; c < kDevMaxCons; ++c) acc[c] = 0;
-    for (int k = n - 1; k >= 0; --k) {
-      const uint32_t q = fast_div(rem, sp.fd[k]);
-      const uint32_t i = rem - q * sp.ext[k];
-      rem = q;
-      s += (int64_t)i * sp.sstride[k];
-      d += (int64_t)i * sp.dstride[k];
-      if (n_cons > 0) {
+      for (int c = 0; c < NC; ++c) acc[u][c] = sp.cons[c].off;
+    }
+  }
+  for (int k = n - 1; k >= 0; --k) {
+    const FastDiv fd = sp.fd[k];
+    const uint32_t ext = sp.ext[k];
+    const OffT ss = (OffT)sp.sstride[k], ds = (OffT)sp.dstride[k];
 #pragma unroll
-        for (int c = 0; c < kDevMaxCons; ++c)
-          if (c < n_cons) acc[c] += (int64_t)sp.cons[c].coef[k] * (int64_t)i;
+    for (int u = 0; u < U; ++u) {
+      const uint32_t q = fast_div(rem[u], fd);
+      const uint32_t i = rem[u] - q * ext;
+      rem[u] = q;
+      so[u] += (OffT)i * ss;
+      doff[u] += (OffT)i * ds;
+      if constexpr (NC > 0) {
+#pragma unroll
+        for (int c = 0; c < NC; ++c) acc[u][c] += sp.cons[c].coef[k] * (int32_t)i;
       }
     }
-    if (n_cons > 0) {
+  }
+  bool load[U];
 #pragma unroll
-      for (int c = 0; c < kDevMaxCons; ++c)
-        if (c < n_cons) {
-          const int64_t v = acc[c] + sp.cons[c].off;
-          const bool ok = (v >= 0) && (v < sp.cons[c].extent);
-          if (c < sp.n_guards) load[u] = load[u] && ok;   // a failed guard stores the fill value
-          else live[u] = live[u] && ok;                    // outside the piece's domain: nothing to do
-        }
+  for (int u = 0; u < U; ++u) {
+    load[u] = live[u] && (src != nullptr);
+    if constexpr (NC > 0) {
+      const int ng = sp.n_guards, nc = sp.n_guards + sp.n_domain;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const bool ok = (c >= nc) || ((uint32_t)acc[u][c] < (uint32_t)sp.cons[c].extent);
+        if (c < ng) load[u] = load[u] && ok;  // a failed guard stores the fill value
+        else live[u] = live[u] && ok;         // outside the piece's domain: nothing to do
+      }
+      load[u] = load[u] && live[u];
     }
-    so[u] = s;
-    doff[u] = d;
   }
   T val[U];
   const T fill = fill_unit<V>(sp);
 #pragma unroll
-  for (int u = 0; u < U; ++u) val[u] = (load[u] && live[u]) ? load_unit<V>(src + so[u]) : fill;
+  for (int u = 0; u < U; ++u) val[u] = load[u] ? load_unit<V>(src + so[u]) : fill;
 #pragma unroll
   for (int u = 0; u < U; ++u)
     if (live[u]) store_unit<V>(dst + doff[u], val[u]);
+}
+
+// ---------------------------------------------------------------------------
+// Tiled transpose for pieces whose destination-contiguous index a is not the
+// source-contiguous index b.  A block moves a tile of (128 bytes of a) x
+// (kTileB elements of b) = 16 KiB through shared memory:
+//   phase 1  16-byte loads along b (full 128-byte lines of the source), stored
+//            as 16-byte chunks in the row of their a;
+//   phase 2  each thread gathers the 16/ES elements of 16/ES consecutive a at
+//            one b, packs them, and stores 16 bytes along a (full lines of the
+//            destination).
+// The 16-byte chunk index within a row is XOR-ed with (a / (16/ES)) & 7, which
+// makes both the vector stores of phase 1 and the element reads of phase 2
+// bank-conflict-free.  Tiles on the ragged edge are predicated per chunk (the
+// planner only selects this kernel when both extents are multiples of 16/ES).
+// ---------------------------------------------------------------------------
+template <int ES>
+__device__ __forceinline__ uint4 gather_column(const unsigned char *tile, int ca, int b_l) {
+  constexpr int EPU = 16 / ES;
+  constexpr int RB = kTileB * ES;
+  const int chunk = b_l / EPU;
+  const unsigned char *p = tile + (ca * EPU) * RB + ((chunk ^ ca) << 4) + (b_l % EPU) * ES;
+  uint4 out;
+  if constexpr (ES == 1) {
+    uint32_t w[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      w[g] = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[g] |= (uint32_t)p[(g * 4 + j) * RB] << (8 * j);
+    }
+    out = make_uint4(w[0], w[1], w[2], w[3]);
+  } else if constexpr (ES == 2) {
+    uint32_t w[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const uint32_t lo = *reinterpret_cast<const uint16_t *>(p + (2 * g) * RB);
+      const uint32_t hi = *reinterpret_cast<const uint16_t *>(p + (2 * g + 1) * RB);
+      w[g] = lo | (hi << 16);
+    }
+    out = make_uint4(w[0], w[1], w[2], w[3]);
+  } else if constexpr (ES == 4) {
+    out.x = *reinterpret_cast<const uint32_t *>(p);
+    out.y = *reinterpret_cast<const uint32_t *>(p + RB);
+    out.z = *reinterpret_cast<const uint32_t *>(p + 2 * RB);
+    out.w = *reinterpret_cast<const uint32_t *>(p + 3 * RB);
+  } else {
+    const uint2 lo = *reinterpret_cast<const uint2 *>(p);
+    const uint2 hi = *reinterpret_cast<const uint2 *>(p + RB);
+    out = make_uint4(lo.x, lo.y, hi.x, hi.y);
+  }
+  return out;
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const DevPiece *__restrict__ table,
+                                                                            int first_piece, int n_pieces, PtrTable ptrs) {
+  constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
+  constexpr int TA = 8 * EPU;      // rows of the tile: 128 bytes of destination run
+  constexpr int RB = kTileB * ES;  // bytes per row
+  constexpr int CB = RB / 16;      // chunks per row
+  constexpr int U = TA * CB / kTransposeThreads;
+  static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB, "tile geometry");
+  __shared__ DevPiece sp;
+  __shared__ __align__(128) unsigned char tile[kTileBytes];
+  fetch_piece(table, first_piece, n_pieces, &sp);
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_b);
+  const uint32_t b0 = (t - q * sp.tiles_b) * kTileB;
+  t = q;
+  q = fast_div(t, sp.fd_tiles_a);
+  const uint32_t a0 = (t - q * sp.tiles_a) * TA;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const char *src = ptrs.src[sp.input] + sbase;
+  char *dst = ptrs.dst + dbase;
+  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+
+  // phase 1: global -> shared, 16 bytes along b
+  uint4 v[U];
+  {
+    const FastDiv fa = sp.fd_a_in;
+    const int64_t sa0 = sp.sa[0], sa1 = sp.sa[1];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int a_l = idx / CB, cb = idx % CB;
+      const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
+      v[u] = make_uint4(0, 0, 0, 0);
+      if (a < ext_a && b < ext_b) {
+        const uint32_t a_hi = fast_div(a, fa), a_lo = a - a_hi * fa.d;
+        v[u] = __ldg(reinterpret_cast<const uint4 *>(src + (int64_t)a_lo * sa0 + (int64_t)a_hi * sa1 + (int64_t)b * ES));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int a_l = idx / CB, cb = idx % CB;
+      *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+    }
+  }
+  __syncthreads();
+  // phase 2: shared -> global, 16 bytes along a
+  {
+    const FastDiv fb = sp.fd_b_in;
+    const int64_t db0 = sp.db[0], db1 = sp.db[1];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int ca = idx & 7, b_l = idx >> 3;
+      const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
+      if (a < ext_a && b < ext_b) {
+        const uint4 o = gather_column<ES>(tile, ca, b_l);
+        const uint32_t b_hi = fast_div(b, fb), b_lo = b - b_hi * fb.d;
+        __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)b_lo * db0 + (int64_t)b_hi * db1 + (int64_t)a * ES), o);
+      }
+    }
+  }
 }
 
 }  // namespace amap

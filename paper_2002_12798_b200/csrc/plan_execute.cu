@@ -33,8 +33,10 @@ static int cuda_fail(cudaError_t e, const char *what) {
 extern "C" const char *amap_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
 struct Launch {
-  int kind;       // DevKind
-  int unit;       // bytes per item (affine kernel) / element size (transpose)
+  int kind;  // DevKind
+  int unit;  // bytes per item (affine kernel) / element size (transpose kernel)
+  int cons;  // affine kernel: constraint slots evaluated per unit (0, 2 or kDevMaxCons)
+  int wide;  // affine kernel: 1 when a byte offset can reach 4 GiB (64-bit offsets)
   int first_piece;
   int n_pieces;
   uint32_t n_blocks;
@@ -138,14 +140,18 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
   d->n_guards = (int)p.guards.size();
   d->n_domain = (int)p.domain.size();
   int c = 0;
+  // the kernel evaluates constraints in 32-bit arithmetic: every partial sum must fit
   auto put = [&](const Con &g) -> bool {
-    d->cons[c].off = g.e.c0;
-    d->cons[c].extent = g.extent;
+    int64_t span = std::llabs(g.e.c0);
     for (size_t j = 0; j < loops.size(); ++j) {
       const int64_t v = g.e.c[loops[j]];
-      if (v > INT32_MAX || v < INT32_MIN) return false;
+      if (std::llabs(v) > INT32_MAX) return false;
+      span += std::llabs(v) * (int64_t)(d->ext[j] - 1);
       d->cons[c].coef[j] = (int32_t)v;
     }
+    if (span >= INT32_MAX) return false;
+    d->cons[c].off = (int32_t)g.e.c0;
+    d->cons[c].extent = (int32_t)std::min<int64_t>(g.extent, INT32_MAX);
     ++c;
     return true;
   };
@@ -186,7 +192,8 @@ static bool check_affine_item(const DevPiece &d, uint64_t L, int64_t in_bytes, i
   bool load = d.input >= 0, live = true;
   for (int c = 0; c < nc; ++c) {
     const int64_t v = acc[c] + d.cons[c].off;
-    const bool ok = v >= 0 && v < d.cons[c].extent;
+    if (v > INT32_MAX || v < INT32_MIN) return false;
+    const bool ok = (uint32_t)(int32_t)v < (uint32_t)d.cons[c].extent;
     if (c < d.n_guards) load = load && ok; else live = live && ok;
   }
   if (!live) return true;
@@ -214,6 +221,153 @@ static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_
   for (int k = d.n_loops - 1; k >= 0; --k) {
     if (!check_affine_item(d, mult * (d.ext[k] - 1), in_bytes, out_bytes)) return false;
     mult *= d.ext[k];
+  }
+  return true;
+}
+
+// ---------------------------------------------------------------------------
+// Transpose family.  A piece qualifies when its destination-contiguous loop is
+// not its source-contiguous loop, it has no constraints, and all vector
+// addresses are 16-byte aligned.  The a index (destination-contiguous) and the
+// b index (source-contiguous) may each merge a second loop that is contiguous
+// on that one side only (e.g. (h, w) is one run in an NCHW source but two
+// strides in a padded NHWC destination).
+// ---------------------------------------------------------------------------
+static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiece *d) {
+  if (es > 8 || ptr_align < 16 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
+  const int n = p.n();
+  if (n < 2) return false;
+  const int epu = 16 / es;
+  const int ia = n - 1;
+  if (p.dst.c[ia] != 1 || p.srcoff.c[ia] == 1) return false;
+  int ib = -1;
+  for (int k = 0; k < n - 1; ++k)
+    if (p.srcoff.c[k] == 1) ib = k;
+  if (ib < 0) return false;
+  // second loop of a: next in destination order, contiguous with ia on the destination side
+  int ia_hi = -1;
+  if (ia - 1 >= 0 && ia - 1 != ib && p.dst.c[ia - 1] == p.ext[ia]) ia_hi = ia - 1;
+  // second loop of b: contiguous with ib on the source side
+  int ib_hi = -1;
+  for (int k = 0; k < n; ++k)
+    if (k != ia && k != ia_hi && k != ib && p.srcoff.c[k] == p.ext[ib]) ib_hi = k;
+  auto try_build = [&](int a_hi, int b_hi) -> bool {
+    const int64_t ext_a = p.ext[ia] * (a_hi >= 0 ? p.ext[a_hi] : 1);
+    const int64_t ext_b = p.ext[ib] * (b_hi >= 0 ? p.ext[b_hi] : 1);
+    if (ext_a % epu || ext_b % epu || ext_a > INT32_MAX || ext_b > INT32_MAX) return false;
+    memset(d, 0, sizeof *d);
+    d->kind = kDevTranspose;
+    d->input = p.src;
+    d->unit_bytes = es;
+    d->soff = p.srcoff.c0 * es;
+    d->doff = p.dst.c0 * es;
+    d->ext_a = (uint32_t)ext_a;
+    d->ext_b = (uint32_t)ext_b;
+    d->fd_a_in = make_fastdiv((uint32_t)p.ext[ia]);
+    d->fd_b_in = make_fastdiv((uint32_t)p.ext[ib]);
+    d->sa[0] = p.srcoff.c[ia] * es;
+    d->sa[1] = a_hi >= 0 ? p.srcoff.c[a_hi] * es : 0;
+    d->db[0] = p.dst.c[ib] * es;
+    d->db[1] = b_hi >= 0 ? p.dst.c[b_hi] * es : 0;
+    bool aligned = (d->soff % 16 == 0) && (d->doff % 16 == 0) && (d->sa[0] % 16 == 0) && (d->sa[1] % 16 == 0) &&
+                   (d->db[0] % 16 == 0) && (d->db[1] % 16 == 0);
+    int j = 0;
+    unsigned __int128 batch = 1;
+    for (int k = 0; k < n; ++k) {
+      if (k == ia || k == a_hi || k == ib || k == b_hi) continue;
+      if (j >= kDevMaxLoops) return false;
+      d->ext[j] = (uint32_t)p.ext[k];
+      d->fd[j] = make_fastdiv((uint32_t)p.ext[k]);
+      d->sstride[j] = p.srcoff.c[k] * es;
+      d->dstride[j] = p.dst.c[k] * es;
+      if (d->sstride[j] % 16 || d->dstride[j] % 16) aligned = false;
+      batch *= (uint64_t)p.ext[k];
+      ++j;
+    }
+    if (!aligned) return false;
+    d->n_loops = j;
+    const int ta = 8 * epu;
+    d->tiles_a = (uint32_t)((ext_a + ta - 1) / ta);
+    d->tiles_b = (uint32_t)((ext_b + kTileB - 1) / kTileB);
+    d->fd_tiles_a = make_fastdiv(d->tiles_a);
+    d->fd_tiles_b = make_fastdiv(d->tiles_b);
+    const unsigned __int128 blocks = batch * d->tiles_a * d->tiles_b;
+    if (blocks > 0x7FFFFFFFull) return false;
+    d->n_blocks = (uint32_t)blocks;
+    d->n_items = (uint64_t)blocks;
+    return true;
+  };
+  if (try_build(ia_hi, ib_hi)) return true;
+  if (ib_hi >= 0 && try_build(ia_hi, -1)) return true;
+  if (ia_hi >= 0 && try_build(-1, ib_hi)) return true;
+  if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1)) return true;
+  return false;
+}
+
+// the kernel's address arithmetic for one block, replayed on the host
+static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
+  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu, cb_n = kTileB * es / 16;
+  uint32_t t = blk;
+  uint32_t q = host_fast_div(t, d.fd_tiles_b);
+  if (q != t / d.tiles_b) return false;
+  const uint32_t b0 = (t - q * d.tiles_b) * kTileB;
+  t = q;
+  q = host_fast_div(t, d.fd_tiles_a);
+  if (q != t / d.tiles_a) return false;
+  const uint32_t a0 = (t - q * d.tiles_a) * ta;
+  t = q;
+  int64_t sbase = d.soff, dbase = d.doff;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    q = host_fast_div(t, d.fd[k]);
+    if (q != t / d.ext[k]) return false;
+    const uint32_t i = t - q * d.ext[k];
+    t = q;
+    sbase += (int64_t)i * d.sstride[k];
+    dbase += (int64_t)i * d.dstride[k];
+  }
+  if (t != 0) return false;
+  for (int idx = 0; idx < ta * cb_n; ++idx) {
+    {  // phase 1
+      const int a_l = idx / cb_n, cb = idx % cb_n;
+      const uint32_t a = a0 + a_l, b = b0 + cb * epu;
+      if (a < d.ext_a && b < d.ext_b) {
+        const uint32_t a_hi = host_fast_div(a, d.fd_a_in);
+        if (a_hi != a / d.fd_a_in.d) return false;
+        const uint32_t a_lo = a - a_hi * d.fd_a_in.d;
+        const int64_t s = sbase + (int64_t)a_lo * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
+        if (s % 16 || s < 0 || s + 16 > in_bytes) return false;
+        const int sm = a_l * (kTileB * es) + ((cb ^ ((a_l / epu) & 7)) << 4);
+        if (sm < 0 || sm + 16 > kTileBytes) return false;
+      }
+    }
+    {  // phase 2
+      const int ca = idx & 7, b_l = idx >> 3;
+      const uint32_t a = a0 + ca * epu, b = b0 + b_l;
+      if (a < d.ext_a && b < d.ext_b) {
+        const uint32_t b_hi = host_fast_div(b, d.fd_b_in);
+        if (b_hi != b / d.fd_b_in.d) return false;
+        const uint32_t b_lo = b - b_hi * d.fd_b_in.d;
+        const int64_t o = dbase + (int64_t)b_lo * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a * es;
+        if (o % 16 || o < 0 || o + 16 > out_bytes) return false;
+        const int sm = (ca * epu + epu - 1) * (kTileB * es) + (((b_l / epu) ^ ca) << 4) + (b_l % epu) * es;
+        if (sm + es > kTileBytes) return false;
+      }
+    }
+  }
+  return true;
+}
+
+static bool check_transpose_piece(const DevPiece &d, int64_t in_bytes, int64_t out_bytes) {
+  if (d.n_blocks <= 256) {
+    for (uint32_t b = 0; b < d.n_blocks; ++b)
+      if (!check_transpose_block(d, b, in_bytes, out_bytes)) return false;
+    return true;
+  }
+  uint64_t x = 0x9E3779B97F4A7C15ull;
+  for (int t = 0; t < 256; ++t) {
+    x ^= x << 13; x ^= x >> 7; x ^= x << 17;  // xorshift64
+    const uint32_t b = (t == 0) ? 0 : (t == 1) ? d.n_blocks - 1 : (uint32_t)(x % d.n_blocks);
+    if (!check_transpose_block(d, b, in_bytes, out_bytes)) return false;
   }
   return true;
 }
@@ -249,9 +403,12 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   memset(&pl->stats, 0, sizeof pl->stats);
   pl->stats.n_pieces = (int32_t)m.pieces.size();
 
-  // one launch of the affine kernel per unit width present (pieces grouped by width)
+  // Kernel family and unit width per piece
   std::vector<int> unit_of(m.pieces.size());
+  std::vector<DevPiece> tr(m.pieces.size());
+  std::vector<char> is_tr(m.pieces.size(), 0);
   std::vector<int64_t> reads(m.in_numel.size(), 0);
+  const bool allow_transpose = (o.force_kernel == AMAP_KERNEL_AUTO || o.force_kernel == AMAP_KERNEL_TRANSPOSE);
   for (size_t q = 0; q < m.pieces.size(); ++q) {
     const Piece &p = m.pieces[q];
     unit_of[q] = pick_unit(p, es, std::min(align, 16), o.force_kernel);
@@ -264,34 +421,31 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       kind = AMAP_KERNEL_FILL;
     } else {
       reads[p.src] += piece_unique_reads(p, m.in_numel[p.src]);
-      kind = (unit_of[q] > es || (p.n() > 0 && p.srcoff.c[p.n() - 1] == 1 && p.dst.c[p.n() - 1] == 1)) ? AMAP_KERNEL_COPY
-                                                                                                         : AMAP_KERNEL_GATHER;
+      const bool contiguous = p.n() > 0 && p.srcoff.c[p.n() - 1] == 1 && p.dst.c[p.n() - 1] == 1;
+      if (!contiguous && allow_transpose && build_transpose_piece(p, es, align, &tr[q])) {
+        is_tr[q] = 1;
+        kind = AMAP_KERNEL_TRANSPOSE;
+      } else {
+        kind = (unit_of[q] > es || contiguous) ? AMAP_KERNEL_COPY : AMAP_KERNEL_GATHER;
+      }
     }
     pl->piece_kernel.push_back(kind);
   }
   for (size_t q = 0; q < reads.size(); ++q) pl->stats.bytes_read += std::min(reads[q], m.in_numel[q]) * es;
 
-  for (int V = 16; V >= 1; V >>= 1) {
-    Launch L{kDevAffine, V, (int)pl->table.size(), 0, 0};
+  auto fail = [&](int rc, size_t q) {
+    if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", q, rc);
+    delete pl;
+    return rc;
+  };
+  // one launch of the transpose kernel for all its pieces
+  {
+    Launch L{kDevTranspose, es, 0, 0, (int)pl->table.size(), 0, 0};
     for (size_t q = 0; q < m.pieces.size(); ++q) {
-      if (unit_of[q] != V) continue;
-      DevPiece d;
-      const int rc = build_affine_piece(m.pieces[q], es, V, &d);
-      if (rc != AMAP_OK) {
-        delete pl;
-        return rc;
-      }
-      if (d.n_items == 0) continue;
-      const int64_t in_bytes = (d.input >= 0) ? m.in_numel[d.input] * es : 0;
-      if (!check_affine_piece(d, in_bytes, m.out_numel * es)) {
-        if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] plan self-check failed on piece %zu\n", q);
-        delete pl;
-        return AMAP_EOVERFLOW;
-      }
-      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) {
-        delete pl;
-        return AMAP_EUNSUPPORTED;
-      }
+      if (!is_tr[q]) continue;
+      DevPiece d = tr[q];
+      if (!check_transpose_piece(d, m.in_numel[d.input] * es, m.out_numel * es)) return fail(AMAP_EOVERFLOW, q);
+      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
       d.first_block = L.n_blocks;
       L.n_blocks += d.n_blocks;
       L.n_pieces++;
@@ -299,6 +453,32 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     }
     if (L.n_pieces > 0) pl->launches.push_back(L);
   }
+  // affine kernel: one launch per (unit width, constraints, offset width) present
+  for (int V = 16; V >= 1; V >>= 1)
+    for (int cons : {0, 2, kDevMaxCons})
+      for (int wide = 0; wide < 2; ++wide) {
+        Launch L{kDevAffine, V, cons, wide, (int)pl->table.size(), 0, 0};
+        for (size_t q = 0; q < m.pieces.size(); ++q) {
+          if (is_tr[q] || unit_of[q] != V) continue;
+          const Piece &p = m.pieces[q];
+          const int n_cons = (int)(p.guards.size() + p.domain.size());
+          if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
+          const int64_t in_bytes = (p.src >= 0) ? m.in_numel[p.src] * es : 0;
+          const int64_t out_bytes = m.out_numel * es;
+          if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
+          DevPiece d;
+          const int rc = build_affine_piece(p, es, V, &d);
+          if (rc != AMAP_OK) return fail(rc, q);
+          if (d.n_items == 0) continue;
+          if (!check_affine_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
+          if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
+          d.first_block = L.n_blocks;
+          L.n_blocks += d.n_blocks;
+          L.n_pieces++;
+          pl->table.push_back(d);
+        }
+        if (L.n_pieces > 0) pl->launches.push_back(L);
+      }
   for (int k : pl->piece_kernel) {
     const int slot = (k == AMAP_KERNEL_GATHER) ? 0 : (k == AMAP_KERNEL_COPY) ? 1 : (k == AMAP_KERNEL_TRANSPOSE) ? 2 : 3;
     pl->stats.kernel_kind[slot]++;
@@ -357,8 +537,38 @@ extern "C" int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_
 }
 
 template <int V>
-static cudaError_t launch_affine(const amap_plan_t *pl, const Launch &L, const PtrTable &pt, cudaStream_t s) {
-  amap_affine_kernel<V, kUnroll><<<L.n_blocks, kAffineThreads, 0, s>>>(pl->dev_table, L.first_piece, L.n_pieces, pt);
+static void launch_affine(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
+  const dim3 grid(L.n_blocks), block(kAffineThreads);
+  if (L.cons > 2) {
+    if (L.wide) amap_affine_kernel<V, kUnroll, kDevMaxCons, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_affine_kernel<V, kUnroll, kDevMaxCons, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  } else if (L.cons > 0) {
+    if (L.wide) amap_affine_kernel<V, kUnroll, 2, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_affine_kernel<V, kUnroll, 2, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  } else {
+    if (L.wide) amap_affine_kernel<V, kUnroll, 0, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_affine_kernel<V, kUnroll, 0, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  }
+}
+
+static cudaError_t enqueue(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
+  if (L.kind == kDevTranspose) {
+    const dim3 grid(L.n_blocks), block(kTransposeThreads);
+    switch (L.unit) {
+      case 8: amap_transpose_kernel<8><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
+      case 4: amap_transpose_kernel<4><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
+      case 2: amap_transpose_kernel<2><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
+      default: amap_transpose_kernel<1><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
+    }
+  } else {
+    switch (L.unit) {
+      case 16: launch_affine<16>(table, L, pt, s); break;
+      case 8: launch_affine<8>(table, L, pt, s); break;
+      case 4: launch_affine<4>(table, L, pt, s); break;
+      case 2: launch_affine<2>(table, L, pt, s); break;
+      default: launch_affine<1>(table, L, pt, s); break;
+    }
+  }
   return cudaGetLastError();
 }
 
@@ -387,14 +597,7 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
     ~Restore() { if (prev != cur) cudaSetDevice(prev); }
   } restore{prev, plan->device};
   for (const Launch &L : plan->launches) {
-    cudaError_t e = cudaSuccess;
-    switch (L.unit) {
-      case 16: e = launch_affine<16>(plan, L, pt, s); break;
-      case 8: e = launch_affine<8>(plan, L, pt, s); break;
-      case 4: e = launch_affine<4>(plan, L, pt, s); break;
-      case 2: e = launch_affine<2>(plan, L, pt, s); break;
-      default: e = launch_affine<1>(plan, L, pt, s); break;
-    }
+    const cudaError_t e = enqueue(plan->dev_table, L, pt, s);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
   }
   return AMAP_OK;
@@ -455,12 +658,6 @@ static int static_table_address(int device, void **out) {
   return AMAP_OK;
 }
 
-template <int V>
-static cudaError_t launch_affine_at(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
-  amap_affine_kernel<V, kUnroll><<<L.n_blocks, kAffineThreads, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-  return cudaGetLastError();
-}
-
 extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
                                    void *cuda_stream) {
   if (!plan || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
@@ -488,15 +685,7 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
   // the part of the array this plan uses is overwritten in full; nothing in it needs to start at zero
   CUDA_TRY(cudaMemcpyAsync(table, plan->table.data(), plan->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice, s));
   for (const Launch &L : plan->launches) {
-    cudaError_t e = cudaSuccess;
-    const DevPiece *t = (const DevPiece *)table;
-    switch (L.unit) {
-      case 16: e = launch_affine_at<16>(t, L, pt, s); break;
-      case 8: e = launch_affine_at<8>(t, L, pt, s); break;
-      case 4: e = launch_affine_at<4>(t, L, pt, s); break;
-      case 2: e = launch_affine_at<2>(t, L, pt, s); break;
-      default: e = launch_affine_at<1>(t, L, pt, s); break;
-    }
+    const cudaError_t e = enqueue((const DevPiece *)table, L, pt, s);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: kernel launch");
   }
   return AMAP_OK;

@@ -70,15 +70,15 @@ def _f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
 
 def make_values(n: int, dtype: str, values: str, rng: np.random.Generator) -> np.ndarray:
     """n seeded elements of `dtype` as raw unsigned integers of the same width."""
+    if values == "raw" or dtype in ("u8", "u64"):
+        es = ELEM_SIZE[dtype]
+        return rng.integers(0, 1 << (8 * min(es, 4)), size=n, dtype=np.uint64).astype(RAW_DTYPE[es])
     if values == "uniform_int20":
         f = rng.integers(0, 1 << 20, size=n, dtype=np.int64).astype(np.float32)
     elif values == "uniform_pm1":
         f = rng.random(size=n, dtype=np.float32) * np.float32(2.0) - np.float32(1.0)
     elif values == "normal":
         f = rng.standard_normal(size=n, dtype=np.float32)
-    elif values == "raw":
-        es = ELEM_SIZE[dtype]
-        return rng.integers(0, 1 << (8 * min(es, 4)), size=n, dtype=np.uint64).astype(RAW_DTYPE[es])
     else:
         raise ValueError(values)
     if dtype == "fp32":
@@ -258,6 +258,11 @@ def reduced_configs() -> dict:
         "c2_inv": c2_nhwc_to_nchw(N=3, C=72, H=13, W=11),
         "c2_fwd_mid": c2_nchw_to_nhwc(N=2, C=256, H=56, W=56),
         "c2_inv_mid": c2_nhwc_to_nchw(N=2, C=256, H=56, W=56),
+        "c2_fwd_rag": c2_nchw_to_nhwc(N=2, C=72, H=13, W=8),
+        "c2_inv_rag": c2_nhwc_to_nchw(N=2, C=72, H=13, W=8),
+        "c2_fwd_f32": c2_nchw_to_nhwc(N=2, C=36, H=13, W=12, dtype="fp32"),
+        "c2_inv_u8": c2_nhwc_to_nchw(N=2, C=80, H=14, W=8, dtype="u8"),
+        "c2_fwd_u64": c2_nchw_to_nhwc(N=2, C=34, H=5, W=6, dtype="u64"),
         "c3": c3_head_split(B=2, S=80, heads=3, D=128, keep=50),
         "c3_odd": c3_head_split(B=2, S=33, heads=5, D=24, keep=17),
         "c3_merge": c3_head_merge(B=2, S=70, heads=3, D=128),
