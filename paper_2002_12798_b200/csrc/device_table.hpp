@@ -7,6 +7,7 @@ namespace amap {
 constexpr int kDevMaxLoops = 12;
 constexpr int kDevMaxCons = 6;
 constexpr int kMaxInputs = 24;
+constexpr int kStrip = 8;  // units per thread in the affine and strip kernels
 
 // unsigned 32-bit division by an invariant divisor, multiply-and-shift form
 // (Granlund & Montgomery 1994, "Division by invariant integers using
@@ -22,7 +23,7 @@ struct DevCon {  // 0 <= off + sum coef[k] * i_k < extent   (all values fit 32 b
   int32_t coef[kDevMaxLoops];
 };
 
-enum DevKind : int32_t { kDevAffine = 0, kDevTranspose = 1 };
+enum DevKind : int32_t { kDevAffine = 0, kDevTranspose = 1, kDevStrip = 2 };
 
 // Transpose tiles: 8 chunks of 16 bytes of the destination-contiguous index a
 // (128 bytes) by kTileB elements of the source-contiguous index b.
@@ -35,6 +36,12 @@ constexpr int kTransposeThreads = 256;
 //
 // Affine kernel: one item = one unit of `unit_bytes` bytes; the innermost loop
 // counts units; ext/fd/sstride/dstride describe all loops.
+//
+// Strip kernel: as the affine kernel, but loop `ku` (not the innermost) is cut
+// into strips of kStrip iterations: ext[ku] counts strips, its strides and
+// constraint coefficients are per strip, and one item = one strip of up to
+// kStrip units that differ only in loop ku (ku_ext is that loop's true extent;
+// ku_ss, ku_ds, ku_coef are its per-iteration strides and coefficients).
 //
 // Transpose kernel: ext/fd/sstride/dstride describe the BATCH loops only.  The
 // tile indices are a (contiguous in the destination) and b (contiguous in the
@@ -59,6 +66,11 @@ struct DevPiece {
   int64_t sstride[kDevMaxLoops];
   int64_t dstride[kDevMaxLoops];
   DevCon cons[kDevMaxCons];  // guards first, then domain constraints
+  // --- strip kernel only -----------------------------------------------
+  int32_t ku;
+  uint32_t ku_ext;
+  int64_t ku_ss, ku_ds;
+  int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b

@@ -142,6 +142,73 @@ __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPi
 }
 
 // ---------------------------------------------------------------------------
+// Strip copy: the affine copy for nests of two or more loops.  A thread
+// decomposes ONE item index and then walks kStrip consecutive iterations of
+// loop ku by adding that loop's strides, so the index arithmetic is paid once
+// per kStrip units (a 3x3 window gather has six loops and two guards: per-unit
+// decomposition would make it issue-bound).  Consecutive threads still take
+// consecutive units of the innermost loop, so accesses stay coalesced, and all
+// loads of a strip are issued before its first store.
+// ---------------------------------------------------------------------------
+template <int V, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_strip_kernel(const DevPiece *__restrict__ table, int first_piece,
+                                                                     int n_pieces, PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  using T = typename Unit<V>::T;
+  const uint64_t item = (uint64_t)(blockIdx.x - sp.first_block) * kAffineThreads + threadIdx.x;
+  if (item >= sp.n_items) return;
+  const char *src = (sp.input >= 0) ? ptrs.src[sp.input] : nullptr;
+  char *dst = ptrs.dst;
+  uint32_t rem = (uint32_t)item;
+  OffT so = (OffT)sp.soff, dof = (OffT)sp.doff;
+  int32_t acc[NC > 0 ? NC : 1];
+  if constexpr (NC > 0) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) acc[c] = sp.cons[c].off;
+  }
+  uint32_t strip = 0;
+  const int ku = sp.ku;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    const uint32_t q = fast_div(rem, sp.fd[k]);
+    const uint32_t i = rem - q * sp.ext[k];
+    rem = q;
+    so += (OffT)i * (OffT)sp.sstride[k];
+    dof += (OffT)i * (OffT)sp.dstride[k];
+    if (k == ku) strip = i;
+    if constexpr (NC > 0) {
+#pragma unroll
+      for (int c = 0; c < NC; ++c) acc[c] += sp.cons[c].coef[k] * (int32_t)i;
+    }
+  }
+  const uint32_t left = sp.ku_ext - strip * kStrip;  // iterations of loop ku that remain, >= 1
+  const OffT ss = (OffT)sp.ku_ss, ds = (OffT)sp.ku_ds;
+  bool live[kStrip], load[kStrip];
+#pragma unroll
+  for (int u = 0; u < kStrip; ++u) {
+    live[u] = (uint32_t)u < left;
+    load[u] = live[u] && (src != nullptr);
+    if constexpr (NC > 0) {
+      const int ng = sp.n_guards, nc = sp.n_guards + sp.n_domain;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const bool ok = (c >= nc) || ((uint32_t)(acc[c] + u * sp.ku_coef[c]) < (uint32_t)sp.cons[c].extent);
+        if (c < ng) load[u] = load[u] && ok;
+        else live[u] = live[u] && ok;
+      }
+      load[u] = load[u] && live[u];
+    }
+  }
+  T val[kStrip];
+  const T fill = fill_unit<V>(sp);
+#pragma unroll
+  for (int u = 0; u < kStrip; ++u) val[u] = load[u] ? load_unit<V>(src + (OffT)(so + (OffT)u * ss)) : fill;
+#pragma unroll
+  for (int u = 0; u < kStrip; ++u)
+    if (live[u]) store_unit<V>(dst + (OffT)(dof + (OffT)u * ds), val[u]);
+}
+
+// ---------------------------------------------------------------------------
 // Tiled transpose for pieces whose destination-contiguous index a is not the
 // source-contiguous index b.  A block moves a tile of (128 bytes of a) x
 // (kTileB elements of b) = 16 KiB through shared memory:

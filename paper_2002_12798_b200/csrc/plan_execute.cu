@@ -69,7 +69,7 @@ static FastDiv make_fastdiv(uint32_t d) {
   return f;
 }
 
-static const int kUnroll = 8;  // units per thread in the affine kernel
+static const int kUnroll = kStrip;  // units per thread in the affine kernel
 
 // largest power-of-two unit (<= 16 bytes) in which the piece is still an affine loop nest
 static int pick_unit(const Piece &p, int es, int ptr_align, int force_kind) {
@@ -164,6 +164,48 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
   return AMAP_OK;
 }
 
+// Turns an affine descriptor with two or more loops into a strip descriptor:
+// picks the loop to walk (not the innermost; one whose extent is a multiple of
+// kStrip if there is one, else the longest; the innermost such candidate) and
+// rescales it to count strips.
+static bool make_strip(DevPiece *d) {
+  const int n = d->n_loops;
+  if (n < 2) return false;
+  int ku = -1;
+  for (int k = n - 2; k >= 0; --k)
+    if (d->ext[k] % kStrip == 0) {
+      ku = k;
+      break;
+    }
+  if (ku < 0) {
+    ku = n - 2;
+    for (int k = n - 3; k >= 0; --k)
+      if (d->ext[k] > d->ext[ku]) ku = k;
+  }
+  const int nc = d->n_guards + d->n_domain;
+  for (int c = 0; c < nc; ++c)
+    if (std::llabs((int64_t)d->cons[c].coef[ku]) * kStrip > INT32_MAX / 4) return false;
+  d->kind = kDevStrip;
+  d->ku = ku;
+  d->ku_ext = d->ext[ku];
+  d->ku_ss = d->sstride[ku];
+  d->ku_ds = d->dstride[ku];
+  for (int c = 0; c < nc; ++c) {
+    d->ku_coef[c] = d->cons[c].coef[ku];
+    d->cons[c].coef[ku] *= kStrip;
+  }
+  const uint32_t strips = (d->ext[ku] + kStrip - 1) / kStrip;
+  d->ext[ku] = strips;
+  d->fd[ku] = make_fastdiv(strips);
+  d->sstride[ku] *= kStrip;
+  d->dstride[ku] *= kStrip;
+  uint64_t items = 1;
+  for (int k = 0; k < n; ++k) items *= d->ext[k];
+  d->n_items = items;
+  d->n_blocks = (uint32_t)((items + kAffineThreads - 1) / kAffineThreads);
+  return true;
+}
+
 // Walks a device descriptor on the HOST with the kernel's own arithmetic and
 // checks every address it would form: inside its buffer and aligned to the
 // unit.  Small pieces are walked completely, large ones at their first and
@@ -189,6 +231,31 @@ static bool check_affine_item(const DevPiece &d, uint64_t L, int64_t in_bytes, i
     for (int c = 0; c < nc; ++c) acc[c] += (int64_t)d.cons[c].coef[k] * i;
   }
   if (rem != 0) return false;
+  if (d.kind == kDevStrip) {  // walk the strip as the kernel does
+    uint32_t r2 = (uint32_t)L, strip = 0;
+    for (int k = d.n_loops - 1; k >= 0; --k) {
+      const uint32_t q = r2 / d.ext[k];
+      if (k == d.ku) strip = r2 - q * d.ext[k];
+      r2 = q;
+    }
+    if ((uint64_t)strip * kStrip >= d.ku_ext) return false;
+    const uint32_t left = d.ku_ext - strip * kStrip;
+    const int V = d.unit_bytes;
+    for (uint32_t u = 0; u < (uint32_t)kStrip && u < left; ++u) {
+      bool load = d.input >= 0, live = true;
+      for (int c = 0; c < nc; ++c) {
+        const int64_t v = acc[c] + d.cons[c].off + (int64_t)u * d.ku_coef[c];
+        if (v > INT32_MAX || v < INT32_MIN) return false;
+        const bool ok = (uint32_t)(int32_t)v < (uint32_t)d.cons[c].extent;
+        if (c < d.n_guards) load = load && ok; else live = live && ok;
+      }
+      if (!live) continue;
+      const int64_t oo = o + (int64_t)u * d.ku_ds, sso = s + (int64_t)u * d.ku_ss;
+      if (oo % V || oo < 0 || oo + V > out_bytes) return false;
+      if (load && (sso % V || sso < 0 || sso + V > in_bytes)) return false;
+    }
+    return true;
+  }
   bool load = d.input >= 0, live = true;
   for (int c = 0; c < nc; ++c) {
     const int64_t v = acc[c] + d.cons[c].off;
@@ -456,8 +523,9 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   // affine kernel: one launch per (unit width, constraints, offset width) present
   for (int V = 16; V >= 1; V >>= 1)
     for (int cons : {0, 2, kDevMaxCons})
-      for (int wide = 0; wide < 2; ++wide) {
-        Launch L{kDevAffine, V, cons, wide, (int)pl->table.size(), 0, 0};
+      for (int wide = 0; wide < 2; ++wide)
+       for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
+        Launch L{kind, V, cons, wide, (int)pl->table.size(), 0, 0};
         for (size_t q = 0; q < m.pieces.size(); ++q) {
           if (is_tr[q] || unit_of[q] != V) continue;
           const Piece &p = m.pieces[q];
@@ -470,6 +538,8 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
           const int rc = build_affine_piece(p, es, V, &d);
           if (rc != AMAP_OK) return fail(rc, q);
           if (d.n_items == 0) continue;
+          if (o.force_kernel != AMAP_KERNEL_GATHER) make_strip(&d);
+          if (d.kind != kind) continue;
           if (!check_affine_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
           if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
           d.first_block = L.n_blocks;
@@ -551,8 +621,31 @@ static void launch_affine(const DevPiece *table, const Launch &L, const PtrTable
   }
 }
 
+template <int V>
+static void launch_strip(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
+  const dim3 grid(L.n_blocks), block(kAffineThreads);
+  if (L.cons > 2) {
+    if (L.wide) amap_strip_kernel<V, kDevMaxCons, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_strip_kernel<V, kDevMaxCons, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  } else if (L.cons > 0) {
+    if (L.wide) amap_strip_kernel<V, 2, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_strip_kernel<V, 2, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  } else {
+    if (L.wide) amap_strip_kernel<V, 0, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    else amap_strip_kernel<V, 0, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+  }
+}
+
 static cudaError_t enqueue(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
-  if (L.kind == kDevTranspose) {
+  if (L.kind == kDevStrip) {
+    switch (L.unit) {
+      case 16: launch_strip<16>(table, L, pt, s); break;
+      case 8: launch_strip<8>(table, L, pt, s); break;
+      case 4: launch_strip<4>(table, L, pt, s); break;
+      case 2: launch_strip<2>(table, L, pt, s); break;
+      default: launch_strip<1>(table, L, pt, s); break;
+    }
+  } else if (L.kind == kDevTranspose) {
     const dim3 grid(L.n_blocks), block(kTransposeThreads);
     switch (L.unit) {
       case 8: amap_transpose_kernel<8><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;

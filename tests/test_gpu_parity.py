@@ -39,7 +39,7 @@ def run_gpu(B, chain, xs, force=0, align=16):
     return host[CANARY * es : (CANARY + m.out_numel) * es].view(xs[0].dtype), plan
 
 
-@pytest.mark.parametrize("force", [0, 1], ids=["auto", "gather"])
+@pytest.mark.parametrize("force", [0, 1, 2], ids=["auto", "gather", "copy"])
 @pytest.mark.parametrize("name", sorted(W.reduced_configs()))
 def test_reduced_configs_bit_exact(B, name, force):
     chain = W.reduced_configs()[name]
@@ -81,7 +81,7 @@ def test_random_tiny_chains(B):
             assert e.code == -9
             continue
         want = oracle.run_chain(chain, xs)
-        for force in (0, 1):
+        for force in (0, 1, 2):
             got, _ = run_gpu(B, chain, xs, force=force)
             assert np.array_equal(got, want.reshape(-1)), (trial, force, chain.ops)
         done += 1
