@@ -190,10 +190,15 @@ typedef enum amap_kernel_kind {
   AMAP_KERNEL_FILL = 4       /* no source: vector stores of the constant                                   */
 } amap_kernel_kind;
 
+/* amap_plan_opts.flags: launch the kernels without programmatic dependent launch (by default a kernel's
+ * prologue may overlap the tail of the kernel before it on the stream; it touches no buffer until that one is done) */
+#define AMAP_PLAN_NO_PDL 1
+
 typedef struct amap_plan_opts {
   int32_t force_kernel;     /* amap_kernel_kind; AUTO picks per piece; a family that cannot run a piece falls back to GATHER */
   int32_t pointer_align;    /* bytes every src/dst base pointer is promised to be aligned to (0 = elem_size; 16 enables vectors) */
-  int32_t reserved[6];      /* must be zero */
+  int32_t flags;            /* AMAP_PLAN_* bits */
+  int32_t reserved[5];      /* must be zero */
 } amap_plan_opts;
 
 typedef struct amap_stats {

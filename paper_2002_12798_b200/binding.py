@@ -16,6 +16,7 @@ from . import build as _build
 
 AMAP_CONST = -1
 KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2, 3, 4
+PLAN_NO_PDL = 1
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
 
 EXPORTS = [
@@ -62,7 +63,7 @@ class _Piece(Structure):
 
 
 class _PlanOpts(Structure):
-    _fields_ = [("force_kernel", c_int32), ("pointer_align", c_int32), ("reserved", c_int32 * 6)]
+    _fields_ = [("force_kernel", c_int32), ("pointer_align", c_int32), ("flags", c_int32), ("reserved", c_int32 * 5)]
 
 
 class _Stats(Structure):
@@ -244,10 +245,11 @@ class Map:
             )
         return out
 
-    def plan(self, device=0, force_kernel=KERNEL_AUTO, pointer_align=16) -> "Plan":
+    def plan(self, device=0, force_kernel=KERNEL_AUTO, pointer_align=16, flags=0) -> "Plan":
         opts = _PlanOpts()
         opts.force_kernel = force_kernel
         opts.pointer_align = pointer_align
+        opts.flags = flags
         h = c_void_p()
         _check(_lib.amap_plan(self._h, device, byref(opts), byref(h)), "amap_plan")
         return Plan(h, self)

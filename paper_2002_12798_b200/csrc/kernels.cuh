@@ -15,6 +15,12 @@ template <> struct Unit<4> { using T = uint32_t; };
 template <> struct Unit<8> { using T = uint2; };
 template <> struct Unit<16> { using T = uint4; };
 
+// Programmatic dependent launch: let the next kernel on the stream start its
+// prologue now; wait (before touching any caller buffer) until the kernel
+// before this one has completed and its writes are visible.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f) {
   const uint32_t t = __umulhi(f.mul, n);
   return (t + ((n - t) >> f.sh1)) >> f.sh2;
@@ -77,6 +83,7 @@ template <int V, int U, int NC, typename OffT>
 __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPiece *__restrict__ table, int first_piece,
                                                                       int n_pieces, PtrTable ptrs) {
   __shared__ DevPiece sp;
+  pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
   using T = typename Unit<V>::T;
   const int n = sp.n_loops;
@@ -134,6 +141,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPi
   }
   T val[U];
   const T fill = fill_unit<V>(sp);
+  pdl_wait();
 #pragma unroll
   for (int u = 0; u < U; ++u) val[u] = load[u] ? load_unit<V>(src + so[u]) : fill;
 #pragma unroll
@@ -154,6 +162,7 @@ template <int V, int NC, typename OffT>
 __global__ void __launch_bounds__(kAffineThreads) amap_strip_kernel(const DevPiece *__restrict__ table, int first_piece,
                                                                      int n_pieces, PtrTable ptrs) {
   __shared__ DevPiece sp;
+  pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
   using T = typename Unit<V>::T;
   const uint64_t item = (uint64_t)(blockIdx.x - sp.first_block) * kAffineThreads + threadIdx.x;
@@ -201,6 +210,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_strip_kernel(const DevPie
   }
   T val[kStrip];
   const T fill = fill_unit<V>(sp);
+  pdl_wait();
 #pragma unroll
   for (int u = 0; u < kStrip; ++u) val[u] = load[u] ? load_unit<V>(src + (OffT)(so + (OffT)u * ss)) : fill;
 #pragma unroll
@@ -260,7 +270,46 @@ __device__ __forceinline__ uint4 gather_column(const unsigned char *tile, int ca
   return out;
 }
 
-template <int ES>
+// A block of a fill piece (a strip or affine descriptor with 16-byte units, no source
+// and no constraints) that rides in a transpose launch, so that a map made of
+// transposed copies plus constant borders (padding) is still ONE launch.
+__device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
+  const uint4 fill = fill_unit<16>(sp);
+  if (sp.kind == kDevStrip) {
+    const uint64_t item = (uint64_t)(blockIdx.x - sp.first_block) * kAffineThreads + threadIdx.x;
+    if (item >= sp.n_items) return;
+    uint32_t rem = (uint32_t)item, strip = 0;
+    int64_t dof = sp.doff;
+    for (int k = sp.n_loops - 1; k >= 0; --k) {
+      const uint32_t q = fast_div(rem, sp.fd[k]);
+      const uint32_t i = rem - q * sp.ext[k];
+      rem = q;
+      dof += (int64_t)i * sp.dstride[k];
+      if (k == sp.ku) strip = i;
+    }
+    const uint32_t left = sp.ku_ext - strip * kStrip;
+#pragma unroll
+    for (int u = 0; u < kStrip; ++u)
+      if ((uint32_t)u < left) store_unit<16>(dst + dof + (int64_t)u * sp.ku_ds, fill);
+  } else {
+    const uint64_t item0 = (uint64_t)(blockIdx.x - sp.first_block) * (uint64_t)(kAffineThreads * kStrip) + threadIdx.x;
+#pragma unroll
+    for (int u = 0; u < kStrip; ++u) {
+      const uint64_t L = item0 + (uint64_t)u * kAffineThreads;
+      if (L >= sp.n_items) continue;
+      uint32_t rem = (uint32_t)L;
+      int64_t dof = sp.doff;
+      for (int k = sp.n_loops - 1; k >= 0; --k) {
+        const uint32_t q = fast_div(rem, sp.fd[k]);
+        dof += (int64_t)(rem - q * sp.ext[k]) * sp.dstride[k];
+        rem = q;
+      }
+      store_unit<16>(dst + dof, fill);
+    }
+  }
+}
+
+template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const DevPiece *__restrict__ table,
                                                                             int first_piece, int n_pieces, PtrTable ptrs) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
@@ -271,7 +320,13 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
   static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB, "tile geometry");
   __shared__ DevPiece sp;
   __shared__ __align__(128) unsigned char tile[kTileBytes];
+  pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
+  if (sp.kind != kDevTranspose) {  // block-uniform
+    pdl_wait();
+    fill_block(sp, ptrs.dst);
+    return;
+  }
 
   uint32_t t = blockIdx.x - sp.first_block;
   uint32_t q = fast_div(t, sp.fd_tiles_b);
@@ -291,12 +346,14 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
   const char *src = ptrs.src[sp.input] + sbase;
   char *dst = ptrs.dst + dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  pdl_wait();
 
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];
   {
     const FastDiv fa = sp.fd_a_in;
-    const int64_t sa0 = sp.sa[0], sa1 = sp.sa[1];
+    const bool split = fa.d < ext_a;  // a merges two loops
+    const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
@@ -304,8 +361,14 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
       const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
       v[u] = make_uint4(0, 0, 0, 0);
       if (a < ext_a && b < ext_b) {
-        const uint32_t a_hi = fast_div(a, fa), a_lo = a - a_hi * fa.d;
-        v[u] = __ldg(reinterpret_cast<const uint4 *>(src + (int64_t)a_lo * sa0 + (int64_t)a_hi * sa1 + (int64_t)b * ES));
+        OffT off = (OffT)(b * ES);
+        if (split) {
+          const uint32_t a_hi = fast_div(a, fa);
+          off += (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1;
+        } else {
+          off += (OffT)a * sa0;
+        }
+        v[u] = __ldg(reinterpret_cast<const uint4 *>(src + off));
       }
     }
 #pragma unroll
@@ -317,19 +380,47 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
   }
   __syncthreads();
   // phase 2: shared -> global, 16 bytes along a
-  {
-    const FastDiv fb = sp.fd_b_in;
-    const int64_t db0 = sp.db[0], db1 = sp.db[1];
+  const FastDiv fb = sp.fd_b_in;
+  const bool split_b = fb.d < ext_b;  // b merges two loops
+  const OffT db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
+  auto dst_of = [&](uint32_t a, uint32_t b) -> char * {
+    OffT off = (OffT)(a * ES);
+    if (split_b) {
+      const uint32_t b_hi = fast_div(b, fb);
+      off += (OffT)(b - b_hi * fb.d) * db0 + (OffT)b_hi * db1;
+    } else {
+      off += (OffT)b * db0;
+    }
+    return dst + off;
+  };
+  if constexpr (ES == 2) {
+    // a thread takes two neighbouring b: the 8 words it reads hold both, so half as many shared loads
+#pragma unroll
+    for (int u = 0; u < U / 2; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int ca = idx & 7, b_l = (idx >> 3) * 2;
+      const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
+      if (a < ext_a && b < ext_b) {  // extents are even: b + 1 is inside too
+        const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ ca) << 4) + (b_l % EPU) * ES;
+        uint32_t r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * RB);
+        uint4 lo, hi;
+        lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
+        lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
+        lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
+        lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
+        __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), lo);
+        __stcs(reinterpret_cast<uint4 *>(dst_of(a, b + 1)), hi);
+      }
+    }
+  } else {
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
       const int ca = idx & 7, b_l = idx >> 3;
       const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
-      if (a < ext_a && b < ext_b) {
-        const uint4 o = gather_column<ES>(tile, ca, b_l);
-        const uint32_t b_hi = fast_div(b, fb), b_lo = b - b_hi * fb.d;
-        __stcs(reinterpret_cast<uint4 *>(dst + (int64_t)b_lo * db0 + (int64_t)b_hi * db1 + (int64_t)a * ES), o);
-      }
+      if (a < ext_a && b < ext_b) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), gather_column<ES>(tile, ca, b_l));
     }
   }
 }

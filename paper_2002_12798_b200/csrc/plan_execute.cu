@@ -46,6 +46,7 @@ struct amap_plan_t {
   int device = 0;
   int elem_size = 0;
   int pointer_align = 0;
+  bool pdl = true;  // launch with programmatic stream serialisation
   std::vector<int64_t> in_numel;
   int64_t out_numel = 0;
   std::vector<DevPiece> table;
@@ -446,6 +447,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   if (opts) o = *opts;
   for (int r : o.reserved)
     if (r != 0) return AMAP_EINVAL;
+  if (o.flags & ~AMAP_PLAN_NO_PDL) return AMAP_EINVAL;
   if (o.force_kernel < AMAP_KERNEL_AUTO || o.force_kernel > AMAP_KERNEL_FILL) return AMAP_EINVAL;
   const Map &m = map->m;
   const int es = m.elem_size;
@@ -465,6 +467,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   pl->device = device;
   pl->elem_size = es;
   pl->pointer_align = align;
+  pl->pdl = !(o.flags & AMAP_PLAN_NO_PDL);
   pl->in_numel = m.in_numel;
   pl->out_numel = m.out_numel;
   memset(&pl->stats, 0, sizeof pl->stats);
@@ -505,20 +508,40 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     delete pl;
     return rc;
   };
-  // one launch of the transpose kernel for all its pieces
-  {
-    Launch L{kDevTranspose, es, 0, 0, (int)pl->table.size(), 0, 0};
+  // one launch of the transpose kernel for all its pieces (per offset width); fill pieces with 16-byte units and
+  // no constraints ride in the first such launch, so that padding borders do not cost a launch of their own
+  std::vector<char> placed(m.pieces.size(), 0);
+  for (int wide = 0; wide < 2; ++wide) {
+    Launch L{kDevTranspose, es, 0, wide, (int)pl->table.size(), 0, 0};
     for (size_t q = 0; q < m.pieces.size(); ++q) {
       if (!is_tr[q]) continue;
       DevPiece d = tr[q];
-      if (!check_transpose_piece(d, m.in_numel[d.input] * es, m.out_numel * es)) return fail(AMAP_EOVERFLOW, q);
+      const int64_t in_bytes = m.in_numel[d.input] * es, out_bytes = m.out_numel * es;
+      if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
+      if (!check_transpose_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
       if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
       d.first_block = L.n_blocks;
       L.n_blocks += d.n_blocks;
       L.n_pieces++;
       pl->table.push_back(d);
+      placed[q] = 1;
     }
-    if (L.n_pieces > 0) pl->launches.push_back(L);
+    if (L.n_pieces == 0) continue;
+    for (size_t q = 0; q < m.pieces.size(); ++q) {
+      const Piece &p = m.pieces[q];
+      if (placed[q] || p.src != AMAP_CONST || unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
+      DevPiece d;
+      if (build_affine_piece(p, es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
+      make_strip(&d);
+      if (!check_affine_piece(d, 0, m.out_numel * es)) return fail(AMAP_EOVERFLOW, q);
+      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) continue;
+      d.first_block = L.n_blocks;
+      L.n_blocks += d.n_blocks;
+      L.n_pieces++;
+      pl->table.push_back(d);
+      placed[q] = 1;
+    }
+    pl->launches.push_back(L);
   }
   // affine kernel: one launch per (unit width, constraints, offset width) present
   for (int V = 16; V >= 1; V >>= 1)
@@ -527,7 +550,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
        for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
         Launch L{kind, V, cons, wide, (int)pl->table.size(), 0, 0};
         for (size_t q = 0; q < m.pieces.size(); ++q) {
-          if (is_tr[q] || unit_of[q] != V) continue;
+          if (placed[q] || unit_of[q] != V) continue;
           const Piece &p = m.pieces[q];
           const int n_cons = (int)(p.guards.size() + p.domain.size());
           if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
@@ -606,60 +629,89 @@ extern "C" int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_
   return AMAP_OK;
 }
 
+// One kernel launch.  With `pdl` the launch carries the programmatic-stream-serialisation attribute: the grid may
+// become resident while the kernel before it on the stream drains; the kernels wait (griddepcontrol.wait) for that
+// kernel's completion before they touch a caller buffer.
+template <typename... P, typename... A>
+static void launch(void (*kernel)(P...), uint32_t blocks, int threads, cudaStream_t s, bool pdl, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks);
+  cfg.blockDim = dim3(threads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <int V>
-static void launch_affine(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
-  const dim3 grid(L.n_blocks), block(kAffineThreads);
+static void launch_affine(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  const int fp = L.first_piece, np = L.n_pieces;
   if (L.cons > 2) {
-    if (L.wide) amap_affine_kernel<V, kUnroll, kDevMaxCons, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_affine_kernel<V, kUnroll, kDevMaxCons, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_affine_kernel<V, kUnroll, kDevMaxCons, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_affine_kernel<V, kUnroll, kDevMaxCons, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   } else if (L.cons > 0) {
-    if (L.wide) amap_affine_kernel<V, kUnroll, 2, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_affine_kernel<V, kUnroll, 2, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_affine_kernel<V, kUnroll, 2, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_affine_kernel<V, kUnroll, 2, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   } else {
-    if (L.wide) amap_affine_kernel<V, kUnroll, 0, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_affine_kernel<V, kUnroll, 0, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_affine_kernel<V, kUnroll, 0, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_affine_kernel<V, kUnroll, 0, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   }
 }
 
 template <int V>
-static void launch_strip(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
-  const dim3 grid(L.n_blocks), block(kAffineThreads);
+static void launch_strip(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  const int fp = L.first_piece, np = L.n_pieces;
   if (L.cons > 2) {
-    if (L.wide) amap_strip_kernel<V, kDevMaxCons, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_strip_kernel<V, kDevMaxCons, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_strip_kernel<V, kDevMaxCons, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_strip_kernel<V, kDevMaxCons, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   } else if (L.cons > 0) {
-    if (L.wide) amap_strip_kernel<V, 2, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_strip_kernel<V, 2, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_strip_kernel<V, 2, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_strip_kernel<V, 2, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   } else {
-    if (L.wide) amap_strip_kernel<V, 0, int64_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
-    else amap_strip_kernel<V, 0, uint32_t><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt);
+    if (L.wide) launch(amap_strip_kernel<V, 0, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    else launch(amap_strip_kernel<V, 0, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
   }
 }
 
-static cudaError_t enqueue(const DevPiece *table, const Launch &L, const PtrTable &pt, cudaStream_t s) {
+static cudaError_t enqueue(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  const int fp = L.first_piece, np = L.n_pieces;
   if (L.kind == kDevStrip) {
     switch (L.unit) {
-      case 16: launch_strip<16>(table, L, pt, s); break;
-      case 8: launch_strip<8>(table, L, pt, s); break;
-      case 4: launch_strip<4>(table, L, pt, s); break;
-      case 2: launch_strip<2>(table, L, pt, s); break;
-      default: launch_strip<1>(table, L, pt, s); break;
+      case 16: launch_strip<16>(t, L, pt, s, pdl); break;
+      case 8: launch_strip<8>(t, L, pt, s, pdl); break;
+      case 4: launch_strip<4>(t, L, pt, s, pdl); break;
+      case 2: launch_strip<2>(t, L, pt, s, pdl); break;
+      default: launch_strip<1>(t, L, pt, s, pdl); break;
     }
   } else if (L.kind == kDevTranspose) {
-    const dim3 grid(L.n_blocks), block(kTransposeThreads);
     switch (L.unit) {
-      case 8: amap_transpose_kernel<8><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
-      case 4: amap_transpose_kernel<4><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
-      case 2: amap_transpose_kernel<2><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
-      default: amap_transpose_kernel<1><<<grid, block, 0, s>>>(table, L.first_piece, L.n_pieces, pt); break;
+      case 8:
+        if (L.wide) launch(amap_transpose_kernel<8, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        else launch(amap_transpose_kernel<8, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        break;
+      case 4:
+        if (L.wide) launch(amap_transpose_kernel<4, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        else launch(amap_transpose_kernel<4, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        break;
+      case 2:
+        if (L.wide) launch(amap_transpose_kernel<2, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        else launch(amap_transpose_kernel<2, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        break;
+      default:
+        if (L.wide) launch(amap_transpose_kernel<1, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        else launch(amap_transpose_kernel<1, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
+        break;
     }
   } else {
     switch (L.unit) {
-      case 16: launch_affine<16>(table, L, pt, s); break;
-      case 8: launch_affine<8>(table, L, pt, s); break;
-      case 4: launch_affine<4>(table, L, pt, s); break;
-      case 2: launch_affine<2>(table, L, pt, s); break;
-      default: launch_affine<1>(table, L, pt, s); break;
+      case 16: launch_affine<16>(t, L, pt, s, pdl); break;
+      case 8: launch_affine<8>(t, L, pt, s, pdl); break;
+      case 4: launch_affine<4>(t, L, pt, s, pdl); break;
+      case 2: launch_affine<2>(t, L, pt, s, pdl); break;
+      default: launch_affine<1>(t, L, pt, s, pdl); break;
     }
   }
   return cudaGetLastError();
@@ -690,7 +742,7 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
     ~Restore() { if (prev != cur) cudaSetDevice(prev); }
   } restore{prev, plan->device};
   for (const Launch &L : plan->launches) {
-    const cudaError_t e = enqueue(plan->dev_table, L, pt, s);
+    const cudaError_t e = enqueue(plan->dev_table, L, pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
   }
   return AMAP_OK;
@@ -778,7 +830,7 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
   // the part of the array this plan uses is overwritten in full; nothing in it needs to start at zero
   CUDA_TRY(cudaMemcpyAsync(table, plan->table.data(), plan->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice, s));
   for (const Launch &L : plan->launches) {
-    const cudaError_t e = enqueue((const DevPiece *)table, L, pt, s);
+    const cudaError_t e = enqueue((const DevPiece *)table, L, pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: kernel launch");
   }
   return AMAP_OK;

@@ -222,6 +222,45 @@ static void canonical_loops(Piece &p) {
   }
 }
 
+// Two unconstrained fill pieces of the same value whose boxes touch along one loop (same strides, same other
+// extents, the second starting where the first ends) are one box; repeated to the fixpoint, this turns the
+// per-operand border slabs of a padded concat into a few long runs.
+static bool try_merge_fill(Piece &a, const Piece &b) {
+  if (a.src != AMAP_CONST || b.src != AMAP_CONST || a.fill != b.fill) return false;
+  if (!a.guards.empty() || !a.domain.empty() || !b.guards.empty() || !b.domain.empty()) return false;
+  if (a.n() != b.n() || a.dst.c != b.dst.c) return false;
+  int diff = -1;
+  for (int k = 0; k < a.n(); ++k)
+    if (a.ext[k] != b.ext[k]) {
+      if (diff >= 0) return false;
+      diff = k;
+    }
+  const int64_t delta = b.dst.c0 - a.dst.c0;
+  for (int k = 0; k < a.n(); ++k) {
+    if (diff >= 0 && k != diff) continue;
+    if (delta == a.ext[k] * a.dst.c[k]) {
+      a.ext[k] += b.ext[k];
+      return true;
+    }
+  }
+  return false;
+}
+
+static void merge_fill_pieces(std::vector<Piece> &pieces) {
+  bool changed = true;
+  while (changed) {
+    changed = false;
+    for (size_t i = 0; i < pieces.size() && !changed; ++i)
+      for (size_t j = 0; j < pieces.size() && !changed; ++j) {
+        if (i == j || !try_merge_fill(pieces[i], pieces[j])) continue;
+        pieces.erase(pieces.begin() + j);
+        Piece &p = pieces[j < i ? i - 1 : i];
+        canonical_loops(p);  // the longer loop may now merge with its neighbour
+        changed = true;
+      }
+  }
+}
+
 Status canonicalise(std::vector<Piece> &pieces) {
   std::vector<Piece> work;
   work.swap(pieces);
@@ -267,6 +306,7 @@ Status canonicalise(std::vector<Piece> &pieces) {
     clip_loop(mid, gk, lo, hi - lo + 1);
     work.push_back(std::move(mid));
   }
+  merge_fill_pieces(pieces);
   // deterministic order: by destination offset
   std::stable_sort(pieces.begin(), pieces.end(), [](const Piece &a, const Piece &b) { return a.dst.c0 < b.dst.c0; });
   return Status();

@@ -53,8 +53,8 @@ def test_static_table_refuses_a_plan_that_does_not_fit():
 
     from paper_2002_12798_b200 import binding as B
 
-    # 14 inputs, each padded on both axes (1 copy + 4 border pieces), joined: 70 pieces > the table's 64 descriptors
-    n_in = 14
+    # 22 inputs, each padded on both axes (a copy piece plus border pieces), joined: more pieces than the table's 64 descriptors
+    n_in = 22
     b = B.Builder(2)
     ids = [b.input([4, 8]) for _ in range(n_in)]
     m = b.compose(b.concat([b.pad(t, [1, 1], [1, 1]) for t in ids], 0))
