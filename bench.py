@@ -161,15 +161,23 @@ def run_ours(args):
     (x,) = W.make_inputs(fwd_c)
     nbytes = x.nbytes
     n_sets = max(2, -(-4 * l2 // (3 * nbytes)))  # x, y, z per set; all sets together >= 4 x L2
+    n_sets += n_sets % 2
     xs = [torch.from_numpy(x.view(np.int16)).to(device) for _ in range(n_sets)]
     ys = [torch.empty_like(xs[0]) for _ in range(n_sets)]
     zs = [torch.empty_like(xs[0]) for _ in range(n_sets)]
 
-    def step(i):
-        s = i % n_sets
-        fwd_p.execute([xs[s]], ys[s], stream)
-        inv_p.execute([ys[s]], zs[s], stream)
+    half = n_sets // 2
 
+    def step(i):
+        # The inverse runs on the set that the forward pass wrote half a rotation ago, so that its input has
+        # left L2 by then (51 MB would otherwise be read back from L2 right after being written).
+        s = i % n_sets
+        r = (s + half) % n_sets
+        fwd_p.execute([xs[s]], ys[s], stream)
+        inv_p.execute([ys[r]], zs[r], stream)
+
+    for s in range(n_sets):  # every y exists before any inverse reads it
+        fwd_p.execute([xs[s]], ys[s], stream)
     for i in range(args.warmup):
         step(i)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -301,7 +309,7 @@ def cpu_baseline(oracle, fwd_c, inv_c, x, bytes_per_step, budget_s=20.0):
     }
 
 
-def all_configs(torch, B, device, stream, l2, peak):
+def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmup=5):
     """Every large configuration, each timed the same way (device time per launch, rotating buffers)."""
     out = {}
     configs = dict(W.full_configs())
@@ -310,7 +318,7 @@ def all_configs(torch, B, device, stream, l2, peak):
         name="plain_copy", dtype="bf16", inputs=[[1 << 28]], ops=[{"kind": "reshape", "src": 0, "shape": [1 << 14, 1 << 14]}]
     )
     for name, chain in configs.items():
-        if name == "c1":
+        if name == "c1" or (only and name != only):
             continue
         xs = W.make_inputs(chain)
         m = B.compose_chain(chain)
@@ -322,8 +330,8 @@ def all_configs(torch, B, device, stream, l2, peak):
         n_sets = max(2, min(8, -(-4 * l2 // foot)))
         ins = [[torch.from_numpy(x.view(SIGNED[es])).to(device) for x in xs] for _ in range(n_sets)]
         outs = [torch.empty(m.out_numel, dtype=ins[0][0].dtype, device=device) for _ in range(n_sets)]
-        iters = max(20, min(2000, int(0.25 / (total / 6.0e12))))
-        sec = time_plan(torch, plan, ins, outs, iters, 5, stream)
+        n_it = iters or max(20, min(2000, int(0.25 / (total / 6.0e12))))
+        sec = time_plan(torch, plan, ins, outs, n_it, warmup, stream)
         out[name] = {
             "gbs": round(total / sec / 1e9, 1),
             "us": round(sec * 1e6, 2),
@@ -392,8 +400,20 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--all-configs", action="store_true", help="also time configurations 3, 4, 5 (adds about a minute)")
+    ap.add_argument("--config", default=None, help="time ONE configuration's kernel loop only (for profiler captures) and print its figures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.config:
+        import torch
+
+        from paper_2002_12798_b200 import binding as B
+
+        device = torch.device("cuda", 0)
+        torch.cuda.set_device(device)
+        peak, _ = measured_peak()
+        l2 = torch.cuda.get_device_properties(device).L2_cache_size
+        print(json.dumps(all_configs(torch, B, device, torch.cuda.current_stream(device), l2, peak, args.config, args.steps, args.warmup)))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
