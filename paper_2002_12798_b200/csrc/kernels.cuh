@@ -21,6 +21,10 @@ template <> struct Unit<16> { using T = uint4; };
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Compiler-only fence: read-only (non-coherent) loads may otherwise be sunk below later stores, which would
+// serialise the requests a thread is meant to keep in flight together.
+__device__ __forceinline__ void issue_barrier() { asm volatile("" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f) {
   const uint32_t t = __umulhi(f.mul, n);
   return (t + ((n - t) >> f.sh1)) >> f.sh2;
@@ -39,9 +43,35 @@ __device__ __forceinline__ typename Unit<V>::T fill_unit(const DevPiece &p) {
   return v;
 }
 
+// Read-only global load.  Written as volatile PTX so that the compiler keeps the loads of a thread together,
+// ahead of the issue_barrier() that follows them (an intrinsic load could be sunk below later stores).
+__device__ __forceinline__ uint4 load_16(const char *p) {
+  uint4 v;
+  asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
 template <int V>
 __device__ __forceinline__ typename Unit<V>::T load_unit(const char *p) {
-  return __ldg(reinterpret_cast<const typename Unit<V>::T *>(p));
+  if constexpr (V == 16) {
+    return load_16(p);
+  } else if constexpr (V == 8) {
+    uint2 v;
+    asm volatile("ld.global.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+  } else if constexpr (V == 4) {
+    uint32_t v;
+    asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+  } else if constexpr (V == 2) {
+    uint16_t v;
+    asm volatile("ld.global.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+  } else {
+    uint32_t v;
+    asm volatile("ld.global.u8 %0, [%1];" : "=r"(v) : "l"(p));
+    return (uint8_t)v;
+  }
 }
 
 template <int V>
@@ -80,11 +110,7 @@ __device__ __forceinline__ void fetch_piece(const DevPiece *__restrict__ table, 
 constexpr int kAffineThreads = 256;
 
 template <int V, int U, int NC, typename OffT>
-__global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPiece *__restrict__ table, int first_piece,
-                                                                      int n_pieces, PtrTable ptrs) {
-  __shared__ DevPiece sp;
-  pdl_launch_dependents();
-  fetch_piece(table, first_piece, n_pieces, &sp);
+__device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &ptrs) {
   using T = typename Unit<V>::T;
   const int n = sp.n_loops;
   const uint64_t item0 = (uint64_t)(blockIdx.x - sp.first_block) * (uint64_t)(kAffineThreads * U) + threadIdx.x;
@@ -144,6 +170,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPi
   pdl_wait();
 #pragma unroll
   for (int u = 0; u < U; ++u) val[u] = load[u] ? load_unit<V>(src + so[u]) : fill;
+  issue_barrier();  // every load is issued before the first store
 #pragma unroll
   for (int u = 0; u < U; ++u)
     if (live[u]) store_unit<V>(dst + doff[u], val[u]);
@@ -159,11 +186,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_affine_kernel(const DevPi
 // loads of a strip are issued before its first store.
 // ---------------------------------------------------------------------------
 template <int V, int NC, typename OffT>
-__global__ void __launch_bounds__(kAffineThreads) amap_strip_kernel(const DevPiece *__restrict__ table, int first_piece,
-                                                                     int n_pieces, PtrTable ptrs) {
-  __shared__ DevPiece sp;
-  pdl_launch_dependents();
-  fetch_piece(table, first_piece, n_pieces, &sp);
+__device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &ptrs) {
   using T = typename Unit<V>::T;
   const uint64_t item = (uint64_t)(blockIdx.x - sp.first_block) * kAffineThreads + threadIdx.x;
   if (item >= sp.n_items) return;
@@ -213,6 +236,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_strip_kernel(const DevPie
   pdl_wait();
 #pragma unroll
   for (int u = 0; u < kStrip; ++u) val[u] = load[u] ? load_unit<V>(src + (OffT)(so + (OffT)u * ss)) : fill;
+  issue_barrier();  // every load is issued before the first store
 #pragma unroll
   for (int u = 0; u < kStrip; ++u)
     if (live[u]) store_unit<V>(dst + (OffT)(dof + (OffT)u * ds), val[u]);
@@ -310,18 +334,14 @@ __device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
 }
 
 template <int ES, typename OffT>
-__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const DevPiece *__restrict__ table,
-                                                                            int first_piece, int n_pieces, PtrTable ptrs) {
+__device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
   constexpr int TA = 8 * EPU;      // rows of the tile: 128 bytes of destination run
   constexpr int RB = kTileB * ES;  // bytes per row
   constexpr int CB = RB / 16;      // chunks per row
   constexpr int U = TA * CB / kTransposeThreads;
   static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB, "tile geometry");
-  __shared__ DevPiece sp;
   __shared__ __align__(128) unsigned char tile[kTileBytes];
-  pdl_launch_dependents();
-  fetch_piece(table, first_piece, n_pieces, &sp);
   if (sp.kind != kDevTranspose) {  // block-uniform
     pdl_wait();
     fill_block(sp, ptrs.dst);
@@ -368,9 +388,10 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
         } else {
           off += (OffT)a * sa0;
         }
-        v[u] = __ldg(reinterpret_cast<const uint4 *>(src + off));
+        v[u] = load_16(src + off);
       }
     }
+    issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
@@ -423,6 +444,69 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_kernel(const
       if (a < ext_a && b < ext_b) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), gather_column<ES>(tile, ca, b_l));
     }
   }
+}
+
+// ---------------------------------------------------------------------------
+// Entry kernels.  Each family has two: the *_param kernels get up to
+// kParamPieces descriptors BY VALUE in the kernel parameters (constant bank: a
+// block starts its index arithmetic without a round trip to global memory),
+// the *_table kernels read them from a descriptor table in global memory
+// (launches with more pieces, and amap_execute_static).
+// ---------------------------------------------------------------------------
+constexpr int kParamPieces = 8;
+struct LaunchDesc {
+  int32_t n_pieces;
+  int32_t pad_;
+  DevPiece piece[kParamPieces];
+};
+
+__device__ __forceinline__ const DevPiece &param_piece(const LaunchDesc &ld) {
+  int p = 0;
+  while (p + 1 < ld.n_pieces && blockIdx.x >= ld.piece[p + 1].first_block) ++p;
+  return ld.piece[p];
+}
+
+template <int V, int U, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_affine_param(const __grid_constant__ LaunchDesc ld, PtrTable ptrs) {
+  pdl_launch_dependents();
+  affine_body<V, U, NC, OffT>(param_piece(ld), ptrs);
+}
+template <int V, int U, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_affine_table(const DevPiece *__restrict__ table, int first_piece,
+                                                                     int n_pieces, PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  affine_body<V, U, NC, OffT>(sp, ptrs);
+}
+
+template <int V, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_strip_param(const __grid_constant__ LaunchDesc ld, PtrTable ptrs) {
+  pdl_launch_dependents();
+  strip_body<V, NC, OffT>(param_piece(ld), ptrs);
+}
+template <int V, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_strip_table(const DevPiece *__restrict__ table, int first_piece,
+                                                                    int n_pieces, PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  strip_body<V, NC, OffT>(sp, ptrs);
+}
+
+template <int ES, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_param(const __grid_constant__ LaunchDesc ld,
+                                                                              PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_body<ES, OffT>(param_piece(ld), ptrs);
+}
+template <int ES, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const DevPiece *__restrict__ table,
+                                                                           int first_piece, int n_pieces, PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_body<ES, OffT>(sp, ptrs);
 }
 
 }  // namespace amap

@@ -52,6 +52,7 @@ struct amap_plan_t {
   std::vector<DevPiece> table;
   std::vector<int> piece_kernel;  // amap_kernel_kind per map piece
   std::vector<Launch> launches;
+  std::vector<LaunchDesc> launch_desc;  // per launch; n_pieces == 0 when it has too many pieces for the parameters
   DevPiece *dev_table = nullptr;
   amap_stats stats;
   // staging for amap_execute_host (allocated on first use)
@@ -577,6 +578,15 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     pl->stats.kernel_kind[slot]++;
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
+  for (const Launch &L : pl->launches) {
+    LaunchDesc ld;
+    memset(&ld, 0, sizeof ld);
+    if (L.n_pieces <= kParamPieces) {
+      ld.n_pieces = L.n_pieces;
+      for (int q = 0; q < L.n_pieces; ++q) ld.piece[q] = pl->table[L.first_piece + q];
+    }
+    pl->launch_desc.push_back(ld);
+  }
 
   if (device < 0) {  // a dry plan: can be inspected, not executed
     *out_plan = pl;
@@ -646,72 +656,75 @@ static void launch(void (*kernel)(P...), uint32_t blocks, int threads, cudaStrea
   cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// Where a launch finds its descriptors: by value in the kernel parameters (`ld`), or in a table in global memory.
+struct DescSource {
+  const LaunchDesc *ld;  // non-null: parameter path
+  const DevPiece *table;
+};
+
+#define AMAP_LAUNCH(KP, KT, threads, ...)                                                              \
+  do {                                                                                                 \
+    if (ds.ld) launch(KP<__VA_ARGS__>, L.n_blocks, threads, s, pdl, *ds.ld, pt);                       \
+    else launch(KT<__VA_ARGS__>, L.n_blocks, threads, s, pdl, ds.table, L.first_piece, L.n_pieces, pt); \
+  } while (0)
+
 template <int V>
-static void launch_affine(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
-  const int fp = L.first_piece, np = L.n_pieces;
+static void launch_affine(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if (L.cons > 2) {
-    if (L.wide) launch(amap_affine_kernel<V, kUnroll, kDevMaxCons, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_affine_kernel<V, kUnroll, kDevMaxCons, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, int64_t);
+    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, uint32_t);
   } else if (L.cons > 0) {
-    if (L.wide) launch(amap_affine_kernel<V, kUnroll, 2, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_affine_kernel<V, kUnroll, 2, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, int64_t);
+    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, uint32_t);
   } else {
-    if (L.wide) launch(amap_affine_kernel<V, kUnroll, 0, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_affine_kernel<V, kUnroll, 0, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, int64_t);
+    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, uint32_t);
   }
 }
 
 template <int V>
-static void launch_strip(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
-  const int fp = L.first_piece, np = L.n_pieces;
+static void launch_strip(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if (L.cons > 2) {
-    if (L.wide) launch(amap_strip_kernel<V, kDevMaxCons, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_strip_kernel<V, kDevMaxCons, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, int64_t);
+    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, uint32_t);
   } else if (L.cons > 0) {
-    if (L.wide) launch(amap_strip_kernel<V, 2, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_strip_kernel<V, 2, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 2, int64_t);
+    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 2, uint32_t);
   } else {
-    if (L.wide) launch(amap_strip_kernel<V, 0, int64_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
-    else launch(amap_strip_kernel<V, 0, uint32_t>, L.n_blocks, kAffineThreads, s, pdl, t, fp, np, pt);
+    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 0, int64_t);
+    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 0, uint32_t);
   }
 }
 
-static cudaError_t enqueue(const DevPiece *t, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
-  const int fp = L.first_piece, np = L.n_pieces;
+template <int ES>
+static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  if (L.wide) AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, int64_t);
+  else AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, uint32_t);
+}
+
+static cudaError_t enqueue(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if (L.kind == kDevStrip) {
     switch (L.unit) {
-      case 16: launch_strip<16>(t, L, pt, s, pdl); break;
-      case 8: launch_strip<8>(t, L, pt, s, pdl); break;
-      case 4: launch_strip<4>(t, L, pt, s, pdl); break;
-      case 2: launch_strip<2>(t, L, pt, s, pdl); break;
-      default: launch_strip<1>(t, L, pt, s, pdl); break;
+      case 16: launch_strip<16>(ds, L, pt, s, pdl); break;
+      case 8: launch_strip<8>(ds, L, pt, s, pdl); break;
+      case 4: launch_strip<4>(ds, L, pt, s, pdl); break;
+      case 2: launch_strip<2>(ds, L, pt, s, pdl); break;
+      default: launch_strip<1>(ds, L, pt, s, pdl); break;
     }
   } else if (L.kind == kDevTranspose) {
     switch (L.unit) {
-      case 8:
-        if (L.wide) launch(amap_transpose_kernel<8, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        else launch(amap_transpose_kernel<8, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        break;
-      case 4:
-        if (L.wide) launch(amap_transpose_kernel<4, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        else launch(amap_transpose_kernel<4, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        break;
-      case 2:
-        if (L.wide) launch(amap_transpose_kernel<2, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        else launch(amap_transpose_kernel<2, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        break;
-      default:
-        if (L.wide) launch(amap_transpose_kernel<1, int64_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        else launch(amap_transpose_kernel<1, uint32_t>, L.n_blocks, kTransposeThreads, s, pdl, t, fp, np, pt);
-        break;
+      case 8: launch_transpose<8>(ds, L, pt, s, pdl); break;
+      case 4: launch_transpose<4>(ds, L, pt, s, pdl); break;
+      case 2: launch_transpose<2>(ds, L, pt, s, pdl); break;
+      default: launch_transpose<1>(ds, L, pt, s, pdl); break;
     }
   } else {
     switch (L.unit) {
-      case 16: launch_affine<16>(t, L, pt, s, pdl); break;
-      case 8: launch_affine<8>(t, L, pt, s, pdl); break;
-      case 4: launch_affine<4>(t, L, pt, s, pdl); break;
-      case 2: launch_affine<2>(t, L, pt, s, pdl); break;
-      default: launch_affine<1>(t, L, pt, s, pdl); break;
+      case 16: launch_affine<16>(ds, L, pt, s, pdl); break;
+      case 8: launch_affine<8>(ds, L, pt, s, pdl); break;
+      case 4: launch_affine<4>(ds, L, pt, s, pdl); break;
+      case 2: launch_affine<2>(ds, L, pt, s, pdl); break;
+      default: launch_affine<1>(ds, L, pt, s, pdl); break;
     }
   }
   return cudaGetLastError();
@@ -741,8 +754,11 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
     int prev, cur;
     ~Restore() { if (prev != cur) cudaSetDevice(prev); }
   } restore{prev, plan->device};
-  for (const Launch &L : plan->launches) {
-    const cudaError_t e = enqueue(plan->dev_table, L, pt, s, plan->pdl);
+  for (size_t li = 0; li < plan->launches.size(); ++li) {
+    const Launch &L = plan->launches[li];
+    const LaunchDesc &ld = plan->launch_desc[li];
+    const DescSource ds{ld.n_pieces > 0 ? &ld : nullptr, plan->dev_table};
+    const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
   }
   return AMAP_OK;
@@ -830,7 +846,8 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
   // the part of the array this plan uses is overwritten in full; nothing in it needs to start at zero
   CUDA_TRY(cudaMemcpyAsync(table, plan->table.data(), plan->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice, s));
   for (const Launch &L : plan->launches) {
-    const cudaError_t e = enqueue((const DevPiece *)table, L, pt, s, plan->pdl);
+    const DescSource ds{nullptr, (const DevPiece *)table};  // always through the fixed table
+    const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: kernel launch");
   }
   return AMAP_OK;
