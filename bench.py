@@ -151,7 +151,7 @@ def run_ours(args):
     t0 = time.perf_counter()
     fwd_m, inv_m = B.compose_chain(fwd_c), B.compose_chain(inv_c)
     t1 = time.perf_counter()
-    fwd_p, inv_p = fwd_m.plan(local), inv_m.plan(local)
+    fwd_p, inv_p = fwd_m.plan(local, flags=args.plan_flags), inv_m.plan(local, flags=args.plan_flags)
     t2 = time.perf_counter()
     stats = fwd_p.stats()
     bytes_per_launch = stats["bytes_read"] + stats["bytes_written"]
@@ -281,7 +281,7 @@ def run_ours(args):
     if rank == 0 and world == 1:
         line["cpu_baseline"] = cpu_baseline(oracle, fwd_c, inv_c, x, bytes_per_step)
         if args.all_configs:
-            line["all_configs"] = all_configs(torch, B, device, stream, l2, peak)
+            line["all_configs"] = all_configs(torch, B, device, stream, l2, peak, flags=args.plan_flags)
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -309,7 +309,7 @@ def cpu_baseline(oracle, fwd_c, inv_c, x, bytes_per_step, budget_s=20.0):
     }
 
 
-def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmup=5):
+def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmup=5, flags=0):
     """Every large configuration, each timed the same way (device time per launch, rotating buffers)."""
     out = {}
     configs = dict(W.full_configs())
@@ -322,7 +322,7 @@ def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmu
             continue
         xs = W.make_inputs(chain)
         m = B.compose_chain(chain)
-        plan = m.plan(device.index)
+        plan = m.plan(device.index, flags=flags)
         st = plan.stats()
         total = st["bytes_read"] + st["bytes_written"]
         es = chain.elem_size
@@ -400,6 +400,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--all-configs", action="store_true", help="also time configurations 3, 4, 5 (adds about a minute)")
+    ap.add_argument("--plan-flags", type=int, default=0, help="amap_plan_opts.flags for every plan (1: no programmatic dependent launch, 2: no L2 prefetch)")
     ap.add_argument("--config", default=None, help="time ONE configuration's kernel loop only (for profiler captures) and print its figures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -412,7 +413,7 @@ def main():
         torch.cuda.set_device(device)
         peak, _ = measured_peak()
         l2 = torch.cuda.get_device_properties(device).L2_cache_size
-        print(json.dumps(all_configs(torch, B, device, torch.cuda.current_stream(device), l2, peak, args.config, args.steps, args.warmup)))
+        print(json.dumps(all_configs(torch, B, device, torch.cuda.current_stream(device), l2, peak, args.config, args.steps, args.warmup, args.plan_flags)))
         return
     if args.impl == "reference":
         run_reference(args)

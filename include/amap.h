@@ -193,6 +193,8 @@ typedef enum amap_kernel_kind {
 /* amap_plan_opts.flags: launch the kernels without programmatic dependent launch (by default a kernel's
  * prologue may overlap the tail of the kernel before it on the stream; it touches no buffer until that one is done) */
 #define AMAP_PLAN_NO_PDL 1
+/* do not prefetch a block's first source lines into L2 while the previous kernel on the stream drains */
+#define AMAP_PLAN_NO_PREFETCH 2
 
 typedef struct amap_plan_opts {
   int32_t force_kernel;     /* amap_kernel_kind; AUTO picks per piece; a family that cannot run a piece falls back to GATHER */

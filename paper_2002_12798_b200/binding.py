@@ -17,6 +17,7 @@ from . import build as _build
 AMAP_CONST = -1
 KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2, 3, 4
 PLAN_NO_PDL = 1
+PLAN_NO_PREFETCH = 2
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
 
 EXPORTS = [

@@ -56,6 +56,8 @@ struct DevPiece {
   int32_t n_guards;
   int32_t n_domain;
   int32_t unit_bytes;
+  int32_t prefetch;  // 1: ask L2 for the block's first source lines before waiting for the previous kernel
+  int32_t pad0_;
   uint32_t first_block;  // first block of this piece inside its launch
   uint32_t n_blocks;
   uint64_t n_items;

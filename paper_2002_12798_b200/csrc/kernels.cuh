@@ -366,7 +366,40 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
   const char *src = ptrs.src[sp.input] + sbase;
   char *dst = ptrs.dst + dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
+  // reads nothing into the SM and is harmless whatever that kernel still writes); the loads after the wait
+  // then start from L2 instead of paying a DRAM round trip with the memory system idle.
+  auto prefetch_rows = [&](const char *base, uint32_t pa0, uint32_t pb0) {
+    const uint32_t a = pa0 + threadIdx.x;
+    if (a < ext_a && pb0 < ext_b) {
+      const uint32_t a_hi = fast_div(a, sp.fd_a_in);
+      const char *row = base + (int64_t)(a - a_hi * sp.fd_a_in.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)pb0 * ES;
+      const uint32_t bytes = min((uint32_t)kTileB, ext_b - pb0) * ES;
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
+    }
+  };
+  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(src, a0, b0);
   pdl_wait();
+  // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
+  // blocks further on in the grid): its loads will find their lines in L2.
+  if (sp.prefetch > 1 && threadIdx.x < TA) {
+    uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
+    if (t2 < sp.n_blocks) {
+      uint32_t q2 = fast_div(t2, sp.fd_tiles_b);
+      const uint32_t nb0 = (t2 - q2 * sp.tiles_b) * kTileB;
+      t2 = q2;
+      q2 = fast_div(t2, sp.fd_tiles_a);
+      const uint32_t na0 = (t2 - q2 * sp.tiles_a) * TA;
+      t2 = q2;
+      int64_t nbase = sp.soff;
+      for (int k = sp.n_loops - 1; k >= 0; --k) {
+        q2 = fast_div(t2, sp.fd[k]);
+        nbase += (int64_t)(t2 - q2 * sp.ext[k]) * sp.sstride[k];
+        t2 = q2;
+      }
+      prefetch_rows(ptrs.src[sp.input] + nbase, na0, nb0);
+    }
+  }
 
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];

@@ -448,7 +448,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   if (opts) o = *opts;
   for (int r : o.reserved)
     if (r != 0) return AMAP_EINVAL;
-  if (o.flags & ~AMAP_PLAN_NO_PDL) return AMAP_EINVAL;
+  if (o.flags & ~(AMAP_PLAN_NO_PDL | AMAP_PLAN_NO_PREFETCH)) return AMAP_EINVAL;
   if (o.force_kernel < AMAP_KERNEL_AUTO || o.force_kernel > AMAP_KERNEL_FILL) return AMAP_EINVAL;
   const Map &m = map->m;
   const int es = m.elem_size;
@@ -578,6 +578,15 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     pl->stats.kernel_kind[slot]++;
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
+  {
+    // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM)
+    int sms = 148;
+    if (device >= 0) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    const char *dist = getenv("AMAP_PREFETCH_DISTANCE");
+    const int ahead = dist ? atoi(dist) : 8 * sms;
+    for (DevPiece &d : pl->table)
+      d.prefetch = (o.flags & AMAP_PLAN_NO_PREFETCH) ? 0 : (d.kind == kDevTranspose && ahead > 1) ? ahead : 1;
+  }
   for (const Launch &L : pl->launches) {
     LaunchDesc ld;
     memset(&ld, 0, sizeof ld);
