@@ -341,6 +341,19 @@ def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmu
             "kernels": st["kernels"],
             "launches": st["n_launches"],
         }
+        # the chain before data-movement elimination: one launch and one temporary per operator, same kernels
+        if len(chain.ops) > 1:
+            uplan = B.compose_chain(chain, B.COMPOSE_NO_FUSE).plan(device.index, flags=flags)
+            usec = time_plan(torch, uplan, ins, outs, max(10, n_it // 4), warmup, stream)
+            ust = uplan.stats()
+            out[name]["unfused"] = {
+                "us": round(usec * 1e6, 2),
+                "gbs_effective": round(total / usec / 1e9, 1),
+                "bytes_moved": ust["bytes_read"] + ust["bytes_written"],
+                "stages": ust["n_stages"],
+                "slowdown": round(usec / sec, 2),
+            }
+            del uplan
         del ins, outs
         torch.cuda.empty_cache()
     return out

@@ -53,7 +53,7 @@ typedef enum amap_status {
 /* One access t[C i + b] (Section 2, equations (load)/(store)).  host pointers. */
 typedef struct amap_access {
   int32_t tensor;   /* id of the tensor accessed, or AMAP_CONST (loads only)       */
-  int32_t rank;     /* m, the tensor's rank                                         */
+  int32_t rank;     /* m, the tensor's rank; 1 for a tensor of higher rank = its flat row-major view */
   const int64_t *C; /* m x n_loops, row-major                                       */
   const int64_t *b; /* m                                                            */
 } amap_access;
@@ -139,7 +139,21 @@ int amap_builder_chain(amap_builder *b, int32_t output, const amap_chain **out);
  * the loops that read it), ENOMEM.
  * ------------------------------------------------------------------------- */
 int amap_compose(const amap_chain *chain, amap_map **out_map);
+/* amap_compose with options.  AMAP_COMPOSE_NO_FUSE keeps EVERY intermediate tensor as a temporary, i.e. runs the
+ * chain operator by operator as the paper's Section 2.1 finds it before the optimisation (the comparison baseline). */
+#define AMAP_COMPOSE_NO_FUSE 1u
+int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map **out_map);
 void amap_map_destroy(amap_map *map);
+
+/* Stages.  A map normally has ONE stage: all intermediates are gone.  Where a load/store pair cannot be
+ * eliminated affinely (Section 3 of the paper reports such a leftover pair too: 123 of 124), the intermediate
+ * stays as a TEMPORARY: an earlier stage writes it and later stages read it.  Stage s owns pieces
+ * [first_piece, first_piece + n_pieces) of the piece list and writes temporary *dst_temp (0-based) or, when
+ * *dst_temp is -1, the output; an amap_piece.input >= n_inputs names temporary (input - n_inputs).
+ * Temporaries live in device memory that amap_plan allocates. */
+int amap_map_num_stages(const amap_map *map, int32_t *n);
+int amap_map_get_stage(const amap_map *map, int32_t s, int32_t *first_piece, int32_t *n_pieces, int32_t *dst_temp,
+                       int64_t *dst_numel);
 
 /* a constraint  0 <= offset + sum_k coef[k] * i_k < extent  on the loop indices */
 typedef struct amap_constraint {
@@ -210,7 +224,8 @@ typedef struct amap_stats {
   int32_t n_pieces;
   int32_t n_launches;     /* kernels one amap_execute enqueues                 */
   int32_t kernel_kind[4]; /* pieces planned per family: [0] gather [1] copy [2] transpose [3] fill */
-  int32_t reserved[2];
+  int32_t n_stages;       /* 1 unless the map keeps temporaries */
+  int32_t reserved[1];
 } amap_stats;
 
 int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts /* host, may be NULL */,
@@ -262,6 +277,8 @@ int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void 
  *    to it.  Arguments and alignment rules are those of amap_execute.
  *  - A plan with more than 64 descriptors is refused with AMAP_ETOOLARGE and
  *    nothing is enqueued (compose fewer operators per call, or use amap_execute).
+ *    A plan whose map keeps temporaries (more than one stage) is refused with
+ *    AMAP_EUNSUPPORTED: temporaries need device memory.
  *  - The first call on each device looks up the array's device address
  *    (cudaGetSymbolAddress); make that first call before starting any stream
  *    capture on that device.

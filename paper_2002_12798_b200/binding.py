@@ -16,6 +16,7 @@ from . import build as _build
 
 AMAP_CONST = -1
 KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2, 3, 4
+COMPOSE_NO_FUSE = 1
 PLAN_NO_PDL = 1
 PLAN_NO_PREFETCH = 2
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
@@ -24,7 +25,7 @@ EXPORTS = [
     "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",
     "amap_builder_transpose", "amap_builder_slice", "amap_builder_concat", "amap_builder_pad",
     "amap_builder_window", "amap_builder_tile", "amap_builder_tensor", "amap_builder_stmt",
-    "amap_builder_chain", "amap_compose", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
+    "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
@@ -70,7 +71,7 @@ class _PlanOpts(Structure):
 class _Stats(Structure):
     _fields_ = [
         ("bytes_read", c_int64), ("bytes_written", c_int64), ("bytes_filled", c_int64), ("n_pieces", c_int32),
-        ("n_launches", c_int32), ("kernel_kind", c_int32 * 4), ("reserved", c_int32 * 2),
+        ("n_launches", c_int32), ("kernel_kind", c_int32 * 4), ("n_stages", c_int32), ("reserved", c_int32 * 1),
     ]
 
 
@@ -193,11 +194,14 @@ class Builder:
         st.fill_bits = int(fill_bits)
         _check(_lib.amap_builder_stmt(self._h, byref(st)), "amap_builder_stmt")
 
-    def compose(self, output) -> "Map":
+    def compose(self, output, flags=0) -> "Map":
         chain = c_void_p()
         _check(_lib.amap_builder_chain(self._h, output, byref(chain)), "amap_builder_chain")
         h = c_void_p()
-        _check(_lib.amap_compose(chain, byref(h)), "amap_compose")
+        if flags:
+            _check(_lib.amap_compose_ex(chain, ctypes.c_uint32(flags), byref(h)), "amap_compose_ex")
+        else:
+            _check(_lib.amap_compose(chain, byref(h)), "amap_compose")
         return Map(h)
 
 
@@ -246,6 +250,17 @@ class Map:
             )
         return out
 
+    def stages(self):
+        """[(first_piece, n_pieces, dst_temp (-1 = output), numel)] in execution order."""
+        n = c_int32()
+        _check(_lib.amap_map_num_stages(self._h, byref(n)), "amap_map_num_stages")
+        out = []
+        for s in range(n.value):
+            fp, np_, dt, ne = c_int32(), c_int32(), c_int32(), c_int64()
+            _check(_lib.amap_map_get_stage(self._h, s, byref(fp), byref(np_), byref(dt), byref(ne)), "amap_map_get_stage")
+            out.append((fp.value, np_.value, dt.value, ne.value))
+        return out
+
     def plan(self, device=0, force_kernel=KERNEL_AUTO, pointer_align=16, flags=0) -> "Plan":
         opts = _PlanOpts()
         opts.force_kernel = force_kernel
@@ -273,7 +288,7 @@ class Plan:
         _check(_lib.amap_plan_stats(self._h, byref(s)), "amap_plan_stats")
         return {
             "bytes_read": s.bytes_read, "bytes_written": s.bytes_written, "bytes_filled": s.bytes_filled,
-            "n_pieces": s.n_pieces, "n_launches": s.n_launches,
+            "n_pieces": s.n_pieces, "n_launches": s.n_launches, "n_stages": s.n_stages,
             "kernels": {"gather": s.kernel_kind[0], "copy": s.kernel_kind[1], "transpose": s.kernel_kind[2], "fill": s.kernel_kind[3]},
         }
 
@@ -354,6 +369,6 @@ def build_chain(chain) -> tuple:
     return b, ids[-1]
 
 
-def compose_chain(chain) -> Map:
+def compose_chain(chain, flags=0) -> Map:
     b, out = build_chain(chain)
-    return b.compose(out)
+    return b.compose(out, flags)

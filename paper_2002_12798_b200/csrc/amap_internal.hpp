@@ -62,11 +62,22 @@ void drop_unit_loops(Piece &p);
 Status canonicalise(std::vector<Piece> &pieces);
 
 // ---- compose.cpp ---------------------------------------------------------
+// A composed map runs as one or more STAGES.  Normally there is one: every intermediate tensor was composed
+// away.  An intermediate that could not be composed affinely (or, on request, every intermediate) is kept as a
+// temporary: an earlier stage writes it, later stages read it like an input (piece.src = n_inputs + temporary).
+struct StageInfo {
+  int first_piece = 0, n_pieces = 0;
+  int dst_temp = -1;  // -1: the stage writes the output
+  int64_t numel = 0;
+};
+
 struct Map {
   int elem_size = 0;
   std::vector<int64_t> in_numel;
   int64_t out_numel = 0;
-  std::vector<Piece> pieces;
+  std::vector<int64_t> temp_numel;
+  std::vector<StageInfo> stages;
+  std::vector<Piece> pieces;  // all stages, in execution order
   // storage for the C views handed out by amap_map_get_piece
   std::vector<std::vector<amap_constraint>> guard_views, domain_views;
 };

@@ -119,6 +119,7 @@ extern "C" int amap_builder_reshape(amap_builder *b, int32_t src, int32_t rank, 
   if (ni != no) return AMAP_EINVAL;
   StmtRec r;
   std::vector<int> in_dim, out_dim;  // which dimension each refined loop belongs to
+  bool aligned = true;
   if (ni > 0) {
     // unit dimensions need no loop: walk the others with two cursors
     std::vector<int> idim, odim;
@@ -133,8 +134,8 @@ extern "C" int amap_builder_reshape(amap_builder *b, int32_t src, int32_t rank, 
       if (a == c) f = a;
       else if (a > c && a % c == 0) f = c;
       else if (c > a && c % a == 0) f = a;
-      else return AMAP_EUNSUPPORTED;  // factors do not line up: no affine loop nest
-      if (r.bounds.size() >= AMAP_MAX_LOOPS) return AMAP_EUNSUPPORTED;
+      else { aligned = false; break; }  // factors do not line up
+      if (r.bounds.size() >= AMAP_MAX_LOOPS) { aligned = false; break; }
       r.bounds.push_back(f);
       in_dim.push_back(idim[i]);
       out_dim.push_back(odim[j]);
@@ -147,6 +148,21 @@ extern "C" int amap_builder_reshape(amap_builder *b, int32_t src, int32_t rank, 
     r.bounds.push_back(0);
     in_dim.push_back(0);
     out_dim.push_back(0);
+  }
+  if (!aligned) {
+    // No common refinement of the two shapes: one loop over the flat views of both tensors (still an affine pair).
+    if (ni > INT64_MAX / 2) return AMAP_EOVERFLOW;
+    r.bounds = {(int64_t)ni};
+    r.lC = {1};
+    r.sC = {1};
+    r.lb = {0};
+    r.sb = {0};
+    r.load_tensor = src;
+    r.load_rank = r.store_rank = 1;
+    r.store_tensor = b->add_tensor(ou);
+    *out = r.store_tensor;
+    b->stmts.push_back(std::move(r));
+    return AMAP_OK;
   }
   const int n = (int)r.bounds.size();
   auto rows = [&](const std::vector<int64_t> &shp, const std::vector<int> &dim_of) {

@@ -53,10 +53,12 @@ struct Rows {
   std::vector<Aff> row;  // one affine expression per tensor dimension
 };
 
-static Status read_access(const amap_access &a, int n, const std::vector<TensorInfo> &T, Rows *rows) {
+static Status read_access(const amap_access &a, int n, const std::vector<TensorInfo> &T, Rows *rows, bool *flat) {
   if (a.tensor < 0 || a.tensor >= (int)T.size()) return err(AMAP_EINVAL, "access names an unknown tensor");
   const TensorInfo &t = T[a.tensor];
-  if (a.rank != (int)t.shape.size()) return err(AMAP_EINVAL, "access rank differs from the tensor's rank");
+  // an access of rank 1 to a tensor of higher rank addresses its flat row-major view
+  *flat = (a.rank == 1 && t.shape.size() > 1);
+  if (!*flat && a.rank != (int)t.shape.size()) return err(AMAP_EINVAL, "access rank differs from the tensor's rank");
   if (!a.b || (n > 0 && !a.C)) return err(AMAP_EINVAL, "null C or b");
   rows->row.resize(a.rank);
   for (int d = 0; d < a.rank; ++d) {
@@ -161,6 +163,7 @@ struct TensorState {
 };
 
 static bool surely_disjoint(const RawStore &a, const RawStore &b) {
+  if (a.lo.size() != b.lo.size()) return false;  // one of them addresses the flat view
   for (size_t d = 0; d < a.lo.size(); ++d) {
     if (a.hi[d] < b.lo[d] || b.hi[d] < a.lo[d]) return true;
     const int64_t g = std::gcd(a.step[d], b.step[d]);
@@ -503,7 +506,7 @@ static int64_t unique_reads(const Piece &p0, int64_t in_numel) {
   return std::min(bound, in_numel);
 }
 
-static Status compose_chain(const amap_chain *ch, Map *out) {
+static Status compose_chain(const amap_chain *ch, uint32_t flags, Map *out) {
   if (!ch) return err(AMAP_EINVAL, "null chain");
   const int es = ch->elem_size;
   if (!(es == 1 || es == 2 || es == 4 || es == 8 || es == 16)) return err(AMAP_EINVAL, "elem_size must be 1, 2, 4, 8 or 16");
@@ -535,6 +538,47 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
   if (T[ch->output].input_slot >= 0) return err(AMAP_EINVAL, "the output tensor is an input");
 
   std::vector<TensorState> S(ch->n_tensors);
+  out->elem_size = es;
+  out->in_numel.resize(ch->n_inputs);
+  for (int q = 0; q < ch->n_inputs; ++q) out->in_numel[q] = T[ch->inputs[q]].numel;
+
+  // closes the definitions of tensor t into a stage that writes temporary `temp` (-1: the output)
+  auto finish_stage = [&](int t, int temp) -> Status {
+    std::vector<Piece> pieces = S[t].defs;
+    int64_t covered = 0;
+    for (auto &p : pieces) {
+      const int64_t c = count_points(p);
+      if (c < 0) return err(AMAP_EUNSUPPORTED, "cannot count the points of a piece");
+      covered += c;
+      if (p.src != AMAP_CONST) p.src = T[p.src].input_slot;
+    }
+    if (covered != T[t].numel)
+      return err(temp < 0 ? AMAP_EUNDEFINED : AMAP_EUNSUPPORTED,
+                 temp < 0 ? "some output elements are never written" : "a partly written intermediate cannot be kept as a temporary");
+    Status s = canonicalise(pieces);
+    if (!s.ok()) return s;
+    for (auto &p : pieces)
+      for (int k = 0; k < p.n(); ++k)
+        if (p.ext[k] > INT32_MAX) return err(AMAP_EOVERFLOW, "a merged loop exceeds 2^31-1 iterations");
+    StageInfo st;
+    st.first_piece = (int)out->pieces.size();
+    st.n_pieces = (int)pieces.size();
+    st.dst_temp = temp;
+    st.numel = T[t].numel;
+    out->stages.push_back(st);
+    out->pieces.insert(out->pieces.end(), pieces.begin(), pieces.end());
+    return Status();
+  };
+  auto materialise = [&](int t) -> Status {
+    const int k = (int)out->temp_numel.size();
+    Status s = finish_stage(t, k);
+    if (!s.ok()) return s;
+    out->temp_numel.push_back(T[t].numel);
+    T[t].input_slot = ch->n_inputs + k;
+    S[t].defs.clear();
+    return Status();
+  };
+
   for (int si = 0; si < ch->n_stmts; ++si) {
     const amap_stmt &st = ch->stmts[si];
     const int n = st.n_loops;
@@ -546,15 +590,28 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
     }
     if (st.store.tensor == AMAP_CONST) return err(AMAP_EINVAL, "a store needs a tensor");
     Rows srow, lrow;
-    Status s = read_access(st.store, n, T, &srow);
+    bool sflat = false, lflat = false;
+    Status s = read_access(st.store, n, T, &srow, &sflat);
     if (!s.ok()) return s;
     const int tsid = st.store.tensor;
-    if (T[tsid].input_slot >= 0) return err(AMAP_EINVAL, "a statement stores to an external input");
+    TensorInfo sview = T[tsid], lview;
+    if (sflat) {
+      sview.shape = {T[tsid].numel};
+      sview.stride = {1};
+    }
+    if (T[tsid].input_slot >= 0)
+      return err(AMAP_EINVAL, T[tsid].input_slot < ch->n_inputs ? "a statement stores to an external input"
+                                                                : "a statement stores to a tensor after it was read");
     const bool is_const = (st.load.tensor == AMAP_CONST);
     if (!is_const) {
-      s = read_access(st.load, n, T, &lrow);
+      s = read_access(st.load, n, T, &lrow, &lflat);
       if (!s.ok()) return s;
       if (st.load.tensor == tsid) return err(AMAP_EINVAL, "a statement reads the tensor it writes");
+      lview = T[st.load.tensor];
+      if (lflat) {
+        lview.shape = {T[st.load.tensor].numel};
+        lview.stride = {1};
+      }
     }
     if (empty) continue;
 
@@ -565,7 +622,7 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
     for (size_t d = 0; d < srow.row.size(); ++d) {
       int64_t lo, hi;
       aff_range(srow.row[d], R.ext, &lo, &hi);
-      if (lo < 0 || hi >= T[tsid].shape[d]) return err(AMAP_EOOB, "a store can leave its tensor");
+      if (lo < 0 || hi >= sview.shape[d]) return err(AMAP_EOOB, "a store can leave its tensor");
       rs.lo.push_back(lo);
       rs.hi.push_back(hi);
       int64_t step = 0;
@@ -579,7 +636,7 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
         rs.rem.push_back(((srow.row[d].c0 % step) + step) % step);
       }
     }
-    if (!linearise(srow, T[tsid], n, &R.dst)) return err(AMAP_EOVERFLOW, "store offset overflows");
+    if (!linearise(srow, sview, n, &R.dst)) return err(AMAP_EOVERFLOW, "store offset overflows");
     s = check_injective(R);
     if (!s.ok()) return s;
     rs.piece = R;
@@ -599,15 +656,19 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
     for (size_t d = 0; d < lrow.row.size(); ++d) {
       int64_t lo, hi;
       aff_range(lrow.row[d], R.ext, &lo, &hi);
-      if (lo >= 0 && hi < T[tl].shape[d]) continue;
+      if (lo >= 0 && hi < lview.shape[d]) continue;
       if (!st.guarded) return err(AMAP_EOOB, "an unguarded load can leave its tensor");
       Con g;
       g.e = lrow.row[d];
-      g.extent = T[tl].shape[d];
+      g.extent = lview.shape[d];
       R.guards.push_back(g);
     }
     R.src = tl;
-    if (!linearise(lrow, T[tl], n, &R.srcoff)) return err(AMAP_EOVERFLOW, "load offset overflows");
+    if (!linearise(lrow, lview, n, &R.srcoff)) return err(AMAP_EOVERFLOW, "load offset overflows");
+    if (T[tl].input_slot < 0 && (flags & AMAP_COMPOSE_NO_FUSE)) {
+      s = materialise(tl);
+      if (!s.ok()) return s;
+    }
     if (T[tl].input_slot >= 0) {
       if (tighten(R)) S[tsid].defs.push_back(R);
       continue;
@@ -615,29 +676,20 @@ static Status compose_chain(const amap_chain *ch, Map *out) {
     if (S[tl].defs.empty() && T[tl].numel > 0)
       return err(AMAP_EUNDEFINED, "a statement reads a tensor that no earlier statement writes");
     s = compose_reader(R, S[tl], T[tl], &S[tsid].defs);
+    if (s.code == AMAP_EUNSUPPORTED) {
+      // This pair cannot be eliminated (the paper's Section 3 also reports a pair that stays): keep t_l as a
+      // temporary written by a stage of its own and read it like an input from here on.
+      const Status m = materialise(tl);
+      if (!m.ok()) return s;
+      if (tighten(R)) S[tsid].defs.push_back(R);
+      continue;
+    }
     if (!s.ok()) return s;
   }
 
-  // the output's definitions are the composed map
-  out->elem_size = es;
-  out->in_numel.resize(ch->n_inputs);
-  for (int q = 0; q < ch->n_inputs; ++q) out->in_numel[q] = T[ch->inputs[q]].numel;
+  // the output's definitions are the last stage
   out->out_numel = T[ch->output].numel;
-  out->pieces = S[ch->output].defs;
-  int64_t covered = 0;
-  for (auto &p : out->pieces) {
-    const int64_t c = count_points(p);
-    if (c < 0) return err(AMAP_EUNSUPPORTED, "cannot count the points of an output piece");
-    covered += c;
-    if (p.src != AMAP_CONST) p.src = T[p.src].input_slot;
-  }
-  if (covered != out->out_numel) return err(AMAP_EUNDEFINED, "some output elements are never written");
-  Status s = canonicalise(out->pieces);
-  if (!s.ok()) return s;
-  for (auto &p : out->pieces)
-    for (int k = 0; k < p.n(); ++k)
-      if (p.ext[k] > INT32_MAX) return err(AMAP_EOVERFLOW, "a merged loop exceeds 2^31-1 iterations");
-  return Status();
+  return finish_stage(ch->output, -1);
 }
 
 int64_t piece_unique_reads(const Piece &p, int64_t in_numel) { return unique_reads(p, in_numel); }
@@ -661,13 +713,15 @@ static void log_map(const Map &m) {
   }
 }
 
-extern "C" int amap_compose(const amap_chain *chain, amap_map **out_map) {
-  if (!out_map) return AMAP_EINVAL;
+extern "C" int amap_compose(const amap_chain *chain, amap_map **out_map) { return amap_compose_ex(chain, 0, out_map); }
+
+extern "C" int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map **out_map) {
+  if (!out_map || (flags & ~(uint32_t)AMAP_COMPOSE_NO_FUSE)) return AMAP_EINVAL;
   amap_map *m = new (std::nothrow) amap_map();
   if (!m) return AMAP_ENOMEM;
   Status s;
   try {
-    s = compose_chain(chain, &m->m);
+    s = compose_chain(chain, flags, &m->m);
   } catch (const std::bad_alloc &) {
     s.code = AMAP_ENOMEM;
   }
@@ -711,6 +765,23 @@ extern "C" int amap_map_get_piece(const amap_map *map, int32_t k, amap_piece *ou
   out->n_domain = (int32_t)p.domain.size();
   out->domain = map->m.domain_views[k].data();
   out->fill_bits = p.fill;
+  return AMAP_OK;
+}
+
+extern "C" int amap_map_num_stages(const amap_map *map, int32_t *n) {
+  if (!map || !n) return AMAP_EINVAL;
+  *n = (int32_t)map->m.stages.size();
+  return AMAP_OK;
+}
+
+extern "C" int amap_map_get_stage(const amap_map *map, int32_t s, int32_t *first_piece, int32_t *n_pieces, int32_t *dst_temp,
+                                  int64_t *dst_numel) {
+  if (!map || s < 0 || s >= (int32_t)map->m.stages.size()) return AMAP_EINVAL;
+  const StageInfo &st = map->m.stages[s];
+  if (first_piece) *first_piece = st.first_piece;
+  if (n_pieces) *n_pieces = st.n_pieces;
+  if (dst_temp) *dst_temp = st.dst_temp;
+  if (dst_numel) *dst_numel = st.numel;
   return AMAP_OK;
 }
 

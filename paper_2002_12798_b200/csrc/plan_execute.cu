@@ -40,6 +40,7 @@ struct Launch {
   int first_piece;
   int n_pieces;
   uint32_t n_blocks;
+  int stage;  // which stage of the map this launch belongs to
 };
 
 struct amap_plan_t {
@@ -49,6 +50,9 @@ struct amap_plan_t {
   bool pdl = true;  // launch with programmatic stream serialisation
   std::vector<int64_t> in_numel;
   int64_t out_numel = 0;
+  std::vector<int64_t> temp_numel;  // temporaries between stages
+  std::vector<int> stage_dst;       // per stage: temporary written, -1 = the output
+  std::vector<void *> temps;        // device memory of the temporaries (owned)
   std::vector<DevPiece> table;
   std::vector<int> piece_kernel;  // amap_kernel_kind per map piece
   std::vector<Launch> launches;
@@ -454,7 +458,9 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   const int es = m.elem_size;
   int align = o.pointer_align ? o.pointer_align : es;
   if (align < es || (align & (align - 1))) return AMAP_EINVAL;
-  if ((int)m.in_numel.size() > kMaxInputs) return AMAP_EUNSUPPORTED;
+  if ((int)(m.in_numel.size() + m.temp_numel.size()) > kMaxInputs) return AMAP_EUNSUPPORTED;
+  std::vector<int64_t> slot_numel = m.in_numel;  // what a piece's source slot holds: inputs, then temporaries
+  slot_numel.insert(slot_numel.end(), m.temp_numel.begin(), m.temp_numel.end());
 
   if (device < -1) return AMAP_EINVAL;
   if (device >= 0) {
@@ -471,6 +477,8 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   pl->pdl = !(o.flags & AMAP_PLAN_NO_PDL);
   pl->in_numel = m.in_numel;
   pl->out_numel = m.out_numel;
+  pl->temp_numel = m.temp_numel;
+  for (const StageInfo &st : m.stages) pl->stage_dst.push_back(st.dst_temp);
   memset(&pl->stats, 0, sizeof pl->stats);
   pl->stats.n_pieces = (int32_t)m.pieces.size();
 
@@ -478,7 +486,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   std::vector<int> unit_of(m.pieces.size());
   std::vector<DevPiece> tr(m.pieces.size());
   std::vector<char> is_tr(m.pieces.size(), 0);
-  std::vector<int64_t> reads(m.in_numel.size(), 0);
+  std::vector<int64_t> reads(slot_numel.size(), 0);
   const bool allow_transpose = (o.force_kernel == AMAP_KERNEL_AUTO || o.force_kernel == AMAP_KERNEL_TRANSPOSE);
   for (size_t q = 0; q < m.pieces.size(); ++q) {
     const Piece &p = m.pieces[q];
@@ -491,7 +499,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       pl->stats.bytes_filled += pts * es;
       kind = AMAP_KERNEL_FILL;
     } else {
-      reads[p.src] += piece_unique_reads(p, m.in_numel[p.src]);
+      reads[p.src] += piece_unique_reads(p, slot_numel[p.src]);
       const bool contiguous = p.n() > 0 && p.srcoff.c[p.n() - 1] == 1 && p.dst.c[p.n() - 1] == 1;
       if (!contiguous && allow_transpose && build_transpose_piece(p, es, align, &tr[q])) {
         is_tr[q] = 1;
@@ -502,7 +510,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     }
     pl->piece_kernel.push_back(kind);
   }
-  for (size_t q = 0; q < reads.size(); ++q) pl->stats.bytes_read += std::min(reads[q], m.in_numel[q]) * es;
+  for (size_t q = 0; q < reads.size(); ++q) pl->stats.bytes_read += std::min(reads[q], slot_numel[q]) * es;
 
   auto fail = [&](int rc, size_t q) {
     if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", q, rc);
@@ -512,12 +520,15 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   // one launch of the transpose kernel for all its pieces (per offset width); fill pieces with 16-byte units and
   // no constraints ride in the first such launch, so that padding borders do not cost a launch of their own
   std::vector<char> placed(m.pieces.size(), 0);
+  for (int stage = 0; stage < (int)m.stages.size(); ++stage) {
+  const size_t q_lo = m.stages[stage].first_piece, q_hi = q_lo + m.stages[stage].n_pieces;
+  const int64_t out_bytes = m.stages[stage].numel * es;
   for (int wide = 0; wide < 2; ++wide) {
-    Launch L{kDevTranspose, es, 0, wide, (int)pl->table.size(), 0, 0};
-    for (size_t q = 0; q < m.pieces.size(); ++q) {
+    Launch L{kDevTranspose, es, 0, wide, (int)pl->table.size(), 0, 0, stage};
+    for (size_t q = q_lo; q < q_hi; ++q) {
       if (!is_tr[q]) continue;
       DevPiece d = tr[q];
-      const int64_t in_bytes = m.in_numel[d.input] * es, out_bytes = m.out_numel * es;
+      const int64_t in_bytes = slot_numel[d.input] * es;
       if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
       if (!check_transpose_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
       if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
@@ -528,13 +539,13 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       placed[q] = 1;
     }
     if (L.n_pieces == 0) continue;
-    for (size_t q = 0; q < m.pieces.size(); ++q) {
+    for (size_t q = q_lo; q < q_hi; ++q) {
       const Piece &p = m.pieces[q];
       if (placed[q] || p.src != AMAP_CONST || unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
       DevPiece d;
       if (build_affine_piece(p, es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
       make_strip(&d);
-      if (!check_affine_piece(d, 0, m.out_numel * es)) return fail(AMAP_EOVERFLOW, q);
+      if (!check_affine_piece(d, 0, out_bytes)) return fail(AMAP_EOVERFLOW, q);
       if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) continue;
       d.first_block = L.n_blocks;
       L.n_blocks += d.n_blocks;
@@ -549,14 +560,13 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     for (int cons : {0, 2, kDevMaxCons})
       for (int wide = 0; wide < 2; ++wide)
        for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
-        Launch L{kind, V, cons, wide, (int)pl->table.size(), 0, 0};
-        for (size_t q = 0; q < m.pieces.size(); ++q) {
+        Launch L{kind, V, cons, wide, (int)pl->table.size(), 0, 0, stage};
+        for (size_t q = q_lo; q < q_hi; ++q) {
           if (placed[q] || unit_of[q] != V) continue;
           const Piece &p = m.pieces[q];
           const int n_cons = (int)(p.guards.size() + p.domain.size());
           if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
-          const int64_t in_bytes = (p.src >= 0) ? m.in_numel[p.src] * es : 0;
-          const int64_t out_bytes = m.out_numel * es;
+          const int64_t in_bytes = (p.src >= 0) ? slot_numel[p.src] * es : 0;
           if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
           DevPiece d;
           const int rc = build_affine_piece(p, es, V, &d);
@@ -573,11 +583,13 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
         }
         if (L.n_pieces > 0) pl->launches.push_back(L);
       }
+  }  // stages
   for (int k : pl->piece_kernel) {
     const int slot = (k == AMAP_KERNEL_GATHER) ? 0 : (k == AMAP_KERNEL_COPY) ? 1 : (k == AMAP_KERNEL_TRANSPOSE) ? 2 : 3;
     pl->stats.kernel_kind[slot]++;
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
+  pl->stats.n_stages = (int32_t)m.stages.size();
   {
     // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM)
     int sms = 148;
@@ -609,11 +621,14 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     if (e == cudaSuccess)
       e = cudaMemcpy(pl->dev_table, pl->table.data(), pl->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice);
   }
+  pl->temps.assign(pl->temp_numel.size(), nullptr);
+  for (size_t k = 0; k < pl->temps.size() && e == cudaSuccess; ++k)
+    if (pl->temp_numel[k] > 0) e = cudaMalloc(&pl->temps[k], (size_t)pl->temp_numel[k] * es);
   cudaSetDevice(prev);
   if (e != cudaSuccess) {
-    if (pl->dev_table) cudaFree(pl->dev_table);
-    delete pl;
-    return cuda_fail(e, "amap_plan: descriptor table upload");
+    const int rc = cuda_fail(e, "amap_plan: device allocation");
+    amap_plan_destroy(pl);
+    return rc;
   }
   *out_plan = pl;
   return AMAP_OK;
@@ -629,6 +644,8 @@ extern "C" void amap_plan_destroy(amap_plan_t *plan) {
   cudaGetDevice(&prev);
   cudaSetDevice(plan->device);
   if (plan->dev_table) cudaFree(plan->dev_table);
+  for (void *p : plan->temps)
+    if (p) cudaFree(p);
   for (void *p : plan->stage_in)
     if (p) cudaFree(p);
   if (plan->stage_out) cudaFree(plan->stage_out);
@@ -747,14 +764,15 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
   PtrTable pt;
   memset(&pt, 0, sizeof pt);
   const uintptr_t mask = (uintptr_t)plan->pointer_align - 1;
-  for (size_t q = 0; q < plan->in_numel.size(); ++q) {
+  const size_t n_in = plan->in_numel.size();
+  for (size_t q = 0; q < n_in; ++q) {
     if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
     if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
     if (src_dev_ptrs[q] == dst_dev_ptr) return AMAP_EINVAL;
     pt.src[q] = (const char *)src_dev_ptrs[q];
   }
+  for (size_t k = 0; k < plan->temps.size(); ++k) pt.src[n_in + k] = (const char *)plan->temps[k];
   if ((uintptr_t)dst_dev_ptr & mask) return AMAP_EALIGN;
-  pt.dst = (char *)dst_dev_ptr;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   int prev = 0;
   CUDA_TRY(cudaGetDevice(&prev));
@@ -766,6 +784,8 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
   for (size_t li = 0; li < plan->launches.size(); ++li) {
     const Launch &L = plan->launches[li];
     const LaunchDesc &ld = plan->launch_desc[li];
+    const int t = plan->stage_dst[L.stage];
+    pt.dst = (t < 0) ? (char *)dst_dev_ptr : (char *)plan->temps[t];  // stages run in stream order
     const DescSource ds{ld.n_pieces > 0 ? &ld : nullptr, plan->dev_table};
     const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
@@ -832,6 +852,7 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
                                    void *cuda_stream) {
   if (!plan || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
   if (plan->table.size() > (size_t)kStaticMaxPieces) return AMAP_ETOOLARGE;
+  if (!plan->temp_numel.empty()) return AMAP_EUNSUPPORTED;  // temporaries would need device memory
   if (plan->out_numel == 0) return AMAP_OK;
   if (!dst_dev_ptr) return AMAP_EINVAL;
   PtrTable pt;

@@ -16,39 +16,48 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def eval_map(m, inputs):
-    """out.flat[C_s i + b_s] = in.flat[C_l i + b_l] for every loop point of every piece."""
-    out = np.zeros(m.out_numel, dtype=inputs[0].dtype)
-    cnt = np.zeros(m.out_numel, dtype=np.int32)
+    """Stage by stage: dst.flat[C_s i + b_s] = src.flat[C_l i + b_l] for every loop point of every piece."""
     flat = [x.reshape(-1) for x in inputs]
-    for p in m.pieces():
-        nl = len(p["bounds"])
-        idx = np.indices(p["bounds"], dtype=np.int64).reshape(nl, -1) if nl else np.zeros((0, 1), dtype=np.int64)
+    pieces = m.pieces()
+    result = None
+    for first, n_pieces, dst_temp, numel in m.stages():
+        out = np.zeros(numel, dtype=inputs[0].dtype)
+        cnt = np.zeros(numel, dtype=np.int32)
+        for p in pieces[first : first + n_pieces]:
+            nl = len(p["bounds"])
+            idx = np.indices(p["bounds"], dtype=np.int64).reshape(nl, -1) if nl else np.zeros((0, 1), dtype=np.int64)
 
-        def aff(c, c0):
-            v = np.full(idx.shape[1], c0, dtype=np.int64)
-            for k, ck in enumerate(c):
-                v += ck * idx[k]
-            return v
+            def aff(c, c0):
+                v = np.full(idx.shape[1], c0, dtype=np.int64)
+                for k, ck in enumerate(c):
+                    v += ck * idx[k]
+                return v
 
-        dom = np.ones(idx.shape[1], bool)
-        for c, o, e in p["domain"]:
-            v = aff(c, o)
-            dom &= (v >= 0) & (v < e)
-        g = np.ones(idx.shape[1], bool)
-        for c, o, e in p["guards"]:
-            v = aff(c, o)
-            g &= (v >= 0) & (v < e)
-        d = aff(p["C_s"], p["b_s"])[dom]
-        if p["input"] >= 0:
-            s = aff(p["C_l"], p["b_l"])[dom]
-            gg = g[dom]
-            vals = np.where(gg, flat[p["input"]][np.where(gg, s, 0)], p["fill_bits"]).astype(out.dtype)
+            dom = np.ones(idx.shape[1], bool)
+            for c, o, e in p["domain"]:
+                v = aff(c, o)
+                dom &= (v >= 0) & (v < e)
+            g = np.ones(idx.shape[1], bool)
+            for c, o, e in p["guards"]:
+                v = aff(c, o)
+                g &= (v >= 0) & (v < e)
+            d = aff(p["C_s"], p["b_s"])[dom]
+            if p["input"] >= 0:
+                s = aff(p["C_l"], p["b_l"])[dom]
+                gg = g[dom]
+                vals = np.where(gg, flat[p["input"]][np.where(gg, s, 0)], p["fill_bits"]).astype(out.dtype)
+            else:
+                vals = np.full(d.shape, p["fill_bits"], dtype=out.dtype)
+            out[d] = vals
+            np.add.at(cnt, d, 1)
+        assert (cnt == 1).all(), "the pieces of a stage must write every element exactly once"
+        if dst_temp >= 0:
+            assert dst_temp == len(flat) - len(inputs), "temporaries are numbered in the order they are written"
+            flat.append(out)
         else:
-            vals = np.full(d.shape, p["fill_bits"], dtype=out.dtype)
-        out[d] = vals
-        np.add.at(cnt, d, 1)
-    assert (cnt == 1).all(), "pieces must write every output element exactly once"
-    return out
+            result = out
+    assert result is not None and m.stages()[-1][2] == -1
+    return result
 
 
 @pytest.mark.parametrize("name", sorted(W.reduced_configs()))
@@ -101,16 +110,12 @@ def test_random_tiny_chains():
     for trial in range(300):
         chain = random_chain(r)
         xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
-        try:
-            m = B.compose_chain(chain)
-        except B.AmapError as e:
-            assert e.code == -9, (trial, chain.ops, str(e))  # only "cannot compose affinely" is acceptable
-            unsupported += 1
-            continue
+        m = B.compose_chain(chain)  # every valid chain composes; what cannot be eliminated stays as a temporary
+        unsupported += len(m.stages()) > 1
         want = oracle.run_chain(chain, xs)
         assert np.array_equal(eval_map(m, xs), want.reshape(-1)), (trial, chain.ops)
         done += 1
-    assert done >= 200, (done, unsupported)
+    assert done == 300 and unsupported < 100, (done, unsupported)
 
 
 def test_pad_written_as_explicit_fill_statements():
@@ -232,12 +237,40 @@ def test_error_codes():
     assert _code(lambda: B.Builder(3)) == -1
     assert _code(lambda: B.Builder(4).reshape(0, [2])) == -1  # no such tensor
 
-    def reshape_that_does_not_factor():
-        b = B.Builder(4)
-        x = b.input([2, 3])
-        b.reshape(x, [3, 2])
 
-    assert _code(reshape_that_does_not_factor) == -9
+def test_reshape_whose_factors_do_not_line_up():
+    """[4,6] -> transpose -> [6,4] -> reshape [8,3] -> transpose -> [3,8]: the reshape has no common refinement
+    with the loops around it.  The library must still return the right answer, with a temporary if need be."""
+    chain = W.Chain(
+        name="awkward", dtype="fp32", inputs=[[4, 6]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},
+            {"kind": "reshape", "src": 1, "shape": [8, 3]},
+            {"kind": "transpose", "src": 2, "perm": [1, 0]},
+        ],
+        values="raw",
+    )
+    xs = W.make_index_tagged_inputs(chain)
+    m = B.compose_chain(chain)
+    assert np.array_equal(eval_map(m, xs), oracle.run_chain(chain, xs).reshape(-1))
+    # a lone reshape of that kind needs no temporary: it is one flat loop
+    b = B.Builder(4)
+    x = b.input([2, 3])
+    m = b.compose(b.reshape(x, [3, 2]))
+    assert len(m.stages()) == 1 and len(m.pieces()) == 1
+
+
+def test_no_fuse_keeps_every_intermediate():
+    """The unfused chain (one stage per operator) gives the same bytes as the composed map."""
+    for name in ("c1", "c3_odd", "c4_odd", "c5_odd"):
+        chain = W.reduced_configs()[name]
+        xs = W.make_inputs(chain)
+        fused, unfused = B.compose_chain(chain), B.compose_chain(chain, B.COMPOSE_NO_FUSE)
+        assert len(fused.stages()) == 1
+        n_ops = len(chain.ops)
+        assert len(unfused.stages()) == n_ops, name
+        want = oracle.run_chain(chain, xs).reshape(-1)
+        assert np.array_equal(eval_map(fused, xs), want) and np.array_equal(eval_map(unfused, xs), want)
 
 
 def test_interleaved_stores_are_told_apart_from_overlap():

@@ -21,11 +21,11 @@ def B():
     return binding
 
 
-def run_gpu(B, chain, xs, force=0, align=16):
+def run_gpu(B, chain, xs, force=0, align=16, compose_flags=0):
     """compose -> plan -> execute on cuda:0; returns the output as a flat numpy array of raw bits."""
     import torch
 
-    m = B.compose_chain(chain)
+    m = B.compose_chain(chain, compose_flags)
     plan = m.plan(device=0, force_kernel=force, pointer_align=align)
     es = chain.elem_size
     dev = [torch.from_numpy(np.ascontiguousarray(x).view(SIGNED[es])).cuda() for x in xs]
@@ -86,6 +86,46 @@ def test_random_tiny_chains(B):
             assert np.array_equal(got, want.reshape(-1)), (trial, force, chain.ops)
         done += 1
     assert done >= 60
+
+
+@pytest.mark.parametrize("name", ["c1", "c2_fwd_rag", "c3_odd", "c4", "c4_odd", "c5"])
+def test_unfused_chain_gives_the_same_bytes(B, name):
+    """One stage and one temporary per operator (the chain before data-movement elimination)."""
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, plan = run_gpu(B, chain, xs, compose_flags=B.COMPOSE_NO_FUSE)
+    assert plan.stats()["n_stages"] == len(chain.ops)
+    assert np.array_equal(got, want.reshape(-1))
+
+
+def test_pairs_that_cannot_be_eliminated_become_temporaries(B):
+    chain = W.Chain(
+        name="awkward", dtype="bf16", inputs=[[40, 24]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},
+            {"kind": "reshape", "src": 1, "shape": [64, 15]},
+            {"kind": "transpose", "src": 2, "perm": [1, 0]},
+            {"kind": "pad", "src": 3, "lo": [1, 0], "hi": [0, 2]},
+        ],
+        values="normal",
+    )
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, plan = run_gpu(B, chain, xs)
+    assert plan.stats()["n_stages"] >= 2
+    assert np.array_equal(got, want.reshape(-1))
+
+
+def test_tile_broadcast(B):
+    chain = W.Chain(
+        name="tile", dtype="fp16", inputs=[[3, 40]],
+        ops=[{"kind": "tile", "src": 0, "reps": [5, 2]}, {"kind": "transpose", "src": 1, "perm": [1, 0]}],
+        values="uniform_pm1",
+    )
+    xs = W.make_inputs(chain)
+    got, _ = run_gpu(B, chain, xs)
+    assert np.array_equal(got.reshape(80, 15), np.tile(xs[0], (5, 2)).T)
 
 
 @pytest.mark.parametrize("dtype,es", [("u8", 1), ("u64", 8)])
