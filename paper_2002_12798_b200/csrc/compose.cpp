@@ -45,6 +45,8 @@ static inline int64_t floordiv(int64_t a, int64_t b) {
 static inline int64_t ceildiv(int64_t a, int64_t b) { return -floordiv(-a, b); }
 
 static const int64_t kBig = INT64_MAX / 4;
+static const int kMaxPieceConstraints = 6;  // = the device descriptor's constraint slots
+static const int kMaxPiecesPerReader = 64;  // a reader that shatters into more pieces is cheaper through a temporary
 
 // ---------------------------------------------------------------------------
 // linearisation and validation of one access
@@ -429,6 +431,12 @@ static Status compose_reader(const Piece &R, const TensorState &ts, const Tensor
         cands.push_back({std::move(pr), std::move(in)});
       }
     }
+  // the kernels evaluate at most kMaxPieceConstraints constraints per piece: beyond that the pair is not worth
+  // eliminating (the caller keeps the tensor as a temporary instead)
+  for (auto &c : cands)
+    if (c.in.guards.size() + c.in.domain.size() + R.guards.size() > (size_t)kMaxPieceConstraints)
+      return err(AMAP_EUNSUPPORTED, "the composed piece needs too many constraints");
+  if (cands.size() > (size_t)kMaxPiecesPerReader) return err(AMAP_EUNSUPPORTED, "the pair shatters into too many pieces");
   if (have != need) {
     if (ts.defined_points < ti.numel && have < need)
       return err(AMAP_EUNDEFINED, "a statement reads elements of an intermediate tensor that nothing writes");

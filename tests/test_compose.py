@@ -253,6 +253,19 @@ def test_reshape_whose_factors_do_not_line_up():
     xs = W.make_index_tagged_inputs(chain)
     m = B.compose_chain(chain)
     assert np.array_equal(eval_map(m, xs), oracle.run_chain(chain, xs).reshape(-1))
+    # two such reshapes in a row shatter the loops: the library keeps a temporary rather than dozens of pieces
+    chain.inputs = [[40, 24]]
+    chain.ops = [
+        {"kind": "transpose", "src": 0, "perm": [1, 0]},
+        {"kind": "reshape", "src": 1, "shape": [64, 15]},
+        {"kind": "transpose", "src": 2, "perm": [1, 0]},
+        {"kind": "reshape", "src": 3, "shape": [24, 40]},
+        {"kind": "transpose", "src": 4, "perm": [1, 0]},
+    ]
+    xs = W.make_index_tagged_inputs(chain)
+    m = B.compose_chain(chain)
+    assert len(m.stages()) >= 2
+    assert np.array_equal(eval_map(m, xs), oracle.run_chain(chain, xs).reshape(-1))
     # a lone reshape of that kind needs no temporary: it is one flat loop
     b = B.Builder(4)
     x = b.input([2, 3])

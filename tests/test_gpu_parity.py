@@ -106,14 +106,16 @@ def test_pairs_that_cannot_be_eliminated_become_temporaries(B):
             {"kind": "transpose", "src": 0, "perm": [1, 0]},
             {"kind": "reshape", "src": 1, "shape": [64, 15]},
             {"kind": "transpose", "src": 2, "perm": [1, 0]},
-            {"kind": "pad", "src": 3, "lo": [1, 0], "hi": [0, 2]},
+            {"kind": "reshape", "src": 3, "shape": [24, 40]},
+            {"kind": "transpose", "src": 4, "perm": [1, 0]},
+            {"kind": "pad", "src": 5, "lo": [1, 0], "hi": [0, 2]},
         ],
         values="normal",
     )
     xs = W.make_inputs(chain)
     want = oracle.run_chain(chain, xs)
     got, plan = run_gpu(B, chain, xs)
-    assert plan.stats()["n_stages"] >= 2
+    assert plan.stats()["n_stages"] >= 2  # two reshapes that do not line up with the transposes around them
     assert np.array_equal(got, want.reshape(-1))
 
 
