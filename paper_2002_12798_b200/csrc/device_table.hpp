@@ -74,6 +74,8 @@ struct DevPiece {
   int64_t ku_ss, ku_ds;
   int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
+  int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less
+  int32_t pad1_;
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b
   FastDiv fd_tiles_a, fd_tiles_b;

@@ -480,6 +480,94 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
 }
 
 // ---------------------------------------------------------------------------
+// The same tiled transpose for pieces that are only aligned to UB < 16 bytes
+// (extents that are multiples of UB/ES but not of 16/ES, e.g. 14x14 or 7x7
+// feature maps): the tile, its shared-memory layout and the swizzle are
+// unchanged, only the global accesses shrink to UB bytes.  Loads are issued in
+// groups of eight.  Far slower than the 16-byte kernel per byte, but both
+// global sides stay coalesced, which the element-wise gather cannot offer.
+// ---------------------------------------------------------------------------
+template <int ES>
+__device__ __forceinline__ int tile_offset(int row, int col_byte) {
+  constexpr int RB = kTileB * ES;
+  return row * RB + ((((col_byte >> 4) ^ ((row / (16 / ES)) & 7)) << 4) | (col_byte & 15));
+}
+
+template <int ES, int UB, typename OffT>
+__device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const PtrTable &ptrs) {
+  static_assert(UB >= ES && UB < 16, "narrow units");
+  constexpr int EPN = UB / ES;          // elements per unit
+  constexpr int TA = 8 * (16 / ES);     // tile rows, as in the 16-byte kernel
+  constexpr int RB = kTileB * ES;
+  constexpr int CBU = RB / UB;          // units per row
+  constexpr int NCA = TA / EPN;         // units per destination run
+  constexpr int N = kTileBytes / UB;    // units per tile
+  constexpr int G = 8;                  // loads in flight per thread
+  using T = typename Unit<UB>::T;
+  using E = typename Unit<ES>::T;
+  __shared__ __align__(128) unsigned char tile[kTileBytes];
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_b);
+  const uint32_t b0 = (t - q * sp.tiles_b) * kTileB;
+  t = q;
+  q = fast_div(t, sp.fd_tiles_a);
+  const uint32_t a0 = (t - q * sp.tiles_a) * TA;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const char *src = ptrs.src[sp.input] + sbase;
+  char *dst = ptrs.dst + dbase;
+  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
+  const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1], db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
+  pdl_wait();
+
+  for (int base = 0; base < N; base += G * kTransposeThreads) {
+    T v[G];
+    bool ok[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const int idx = base + threadIdx.x + g * kTransposeThreads;
+      const int a_l = idx / CBU, cu = idx % CBU;
+      const uint32_t a = a0 + a_l, b = b0 + cu * EPN;
+      ok[g] = a < ext_a && b < ext_b;
+      if (ok[g]) {
+        const uint32_t a_hi = fast_div(a, fa);
+        v[g] = load_unit<UB>(src + (OffT)((OffT)(b * ES) + (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1));
+      }
+    }
+    issue_barrier();
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const int idx = base + threadIdx.x + g * kTransposeThreads;
+      if (ok[g]) *reinterpret_cast<T *>(tile + tile_offset<ES>(idx / CBU, (idx % CBU) * UB)) = v[g];
+    }
+  }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < N; idx += kTransposeThreads) {
+    const int ca = idx % NCA, b_l = idx / NCA;
+    const uint32_t a = a0 + ca * EPN, b = b0 + b_l;
+    if (a < ext_a && b < ext_b) {
+      union {
+        T v;
+        E e[EPN];
+      } pk;
+#pragma unroll
+      for (int j = 0; j < EPN; ++j) pk.e[j] = *reinterpret_cast<const E *>(tile + tile_offset<ES>(ca * EPN + j, b_l * ES));
+      const uint32_t b_hi = fast_div(b, fb);
+      store_unit<UB>(dst + (OffT)((OffT)(a * ES) + (OffT)(b - b_hi * fb.d) * db0 + (OffT)b_hi * db1), pk.v);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Entry kernels.  Each family has two: the *_param kernels get up to
 // kParamPieces descriptors BY VALUE in the kernel parameters (constant bank: a
 // block starts its index arithmetic without a round trip to global memory),
@@ -540,6 +628,22 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const 
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
   transpose_body<ES, OffT>(sp, ptrs);
+}
+
+template <int ES, int UB, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_narrow_param(const __grid_constant__ LaunchDesc ld,
+                                                                                  PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_narrow_body<ES, UB, OffT>(param_piece(ld), ptrs);
+}
+template <int ES, int UB, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_narrow_table(const DevPiece *__restrict__ table,
+                                                                                  int first_piece, int n_pieces,
+                                                                                  PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_narrow_body<ES, UB, OffT>(sp, ptrs);
 }
 
 }  // namespace amap

@@ -307,10 +307,9 @@ static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_
 // strides in a padded NHWC destination).
 // ---------------------------------------------------------------------------
 static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiece *d) {
-  if (es > 8 || ptr_align < 16 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
+  if (es > 8 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
   const int n = p.n();
   if (n < 2) return false;
-  const int epu = 16 / es;
   const int ia = n - 1;
   if (p.dst.c[ia] != 1 || p.srcoff.c[ia] == 1) return false;
   int ib = -1;
@@ -324,7 +323,8 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
   int ib_hi = -1;
   for (int k = 0; k < n; ++k)
     if (k != ia && k != ia_hi && k != ib && p.srcoff.c[k] == p.ext[ib]) ib_hi = k;
-  auto try_build = [&](int a_hi, int b_hi) -> bool {
+  auto try_build = [&](int a_hi, int b_hi, int ub) -> bool {
+    const int epu = ub / es;
     const int64_t ext_a = p.ext[ia] * (a_hi >= 0 ? p.ext[a_hi] : 1);
     const int64_t ext_b = p.ext[ib] * (b_hi >= 0 ? p.ext[b_hi] : 1);
     if (ext_a % epu || ext_b % epu || ext_a > INT32_MAX || ext_b > INT32_MAX) return false;
@@ -332,6 +332,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
     d->kind = kDevTranspose;
     d->input = p.src;
     d->unit_bytes = es;
+    d->tr_unit = ub;
     d->soff = p.srcoff.c0 * es;
     d->doff = p.dst.c0 * es;
     d->ext_a = (uint32_t)ext_a;
@@ -342,8 +343,8 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
     d->sa[1] = a_hi >= 0 ? p.srcoff.c[a_hi] * es : 0;
     d->db[0] = p.dst.c[ib] * es;
     d->db[1] = b_hi >= 0 ? p.dst.c[b_hi] * es : 0;
-    bool aligned = (d->soff % 16 == 0) && (d->doff % 16 == 0) && (d->sa[0] % 16 == 0) && (d->sa[1] % 16 == 0) &&
-                   (d->db[0] % 16 == 0) && (d->db[1] % 16 == 0);
+    bool aligned = (d->soff % ub == 0) && (d->doff % ub == 0) && (d->sa[0] % ub == 0) && (d->sa[1] % ub == 0) &&
+                   (d->db[0] % ub == 0) && (d->db[1] % ub == 0);
     int j = 0;
     unsigned __int128 batch = 1;
     for (int k = 0; k < n; ++k) {
@@ -353,13 +354,13 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
       d->fd[j] = make_fastdiv((uint32_t)p.ext[k]);
       d->sstride[j] = p.srcoff.c[k] * es;
       d->dstride[j] = p.dst.c[k] * es;
-      if (d->sstride[j] % 16 || d->dstride[j] % 16) aligned = false;
+      if (d->sstride[j] % ub || d->dstride[j] % ub) aligned = false;
       batch *= (uint64_t)p.ext[k];
       ++j;
     }
     if (!aligned) return false;
     d->n_loops = j;
-    const int ta = 8 * epu;
+    const int ta = 8 * (16 / es);
     d->tiles_a = (uint32_t)((ext_a + ta - 1) / ta);
     d->tiles_b = (uint32_t)((ext_b + kTileB - 1) / kTileB);
     d->fd_tiles_a = make_fastdiv(d->tiles_a);
@@ -370,16 +371,19 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
     d->n_items = (uint64_t)blocks;
     return true;
   };
-  if (try_build(ia_hi, ib_hi)) return true;
-  if (ib_hi >= 0 && try_build(ia_hi, -1)) return true;
-  if (ia_hi >= 0 && try_build(-1, ib_hi)) return true;
-  if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1)) return true;
+  for (int ub = 16; ub >= es; ub >>= 1) {
+    if (ub > ptr_align) continue;
+    if (try_build(ia_hi, ib_hi, ub)) return true;
+    if (ib_hi >= 0 && try_build(ia_hi, -1, ub)) return true;
+    if (ia_hi >= 0 && try_build(-1, ib_hi, ub)) return true;
+    if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1, ub)) return true;
+  }
   return false;
 }
 
 // the kernel's address arithmetic for one block, replayed on the host
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
-  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu, cb_n = kTileB * es / 16;
+  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
   uint32_t t = blk;
   uint32_t q = host_fast_div(t, d.fd_tiles_b);
   if (q != t / d.tiles_b) return false;
@@ -399,31 +403,33 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
     dbase += (int64_t)i * d.dstride[k];
   }
   if (t != 0) return false;
-  for (int idx = 0; idx < ta * cb_n; ++idx) {
+  const int ub = d.tr_unit, epn = ub / es, rb = kTileB * es, cbu = rb / ub, nca = ta / epn;
+  auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ ((row / epu) & 7)) << 4) | (col & 15)); };
+  for (int idx = 0; idx < kTileBytes / ub; ++idx) {
     {  // phase 1
-      const int a_l = idx / cb_n, cb = idx % cb_n;
-      const uint32_t a = a0 + a_l, b = b0 + cb * epu;
+      const int a_l = idx / cbu, cu = idx % cbu;
+      const uint32_t a = a0 + a_l, b = b0 + cu * epn;
       if (a < d.ext_a && b < d.ext_b) {
         const uint32_t a_hi = host_fast_div(a, d.fd_a_in);
         if (a_hi != a / d.fd_a_in.d) return false;
         const uint32_t a_lo = a - a_hi * d.fd_a_in.d;
         const int64_t s = sbase + (int64_t)a_lo * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
-        if (s % 16 || s < 0 || s + 16 > in_bytes) return false;
-        const int sm = a_l * (kTileB * es) + ((cb ^ ((a_l / epu) & 7)) << 4);
-        if (sm < 0 || sm + 16 > kTileBytes) return false;
+        if (s % ub || s < 0 || s + ub > in_bytes) return false;
+        const int sm = tile_off(a_l, cu * ub);
+        if (sm < 0 || sm + ub > kTileBytes || sm % ub) return false;
       }
     }
     {  // phase 2
-      const int ca = idx & 7, b_l = idx >> 3;
-      const uint32_t a = a0 + ca * epu, b = b0 + b_l;
+      const int ca = idx % nca, b_l = idx / nca;
+      const uint32_t a = a0 + ca * epn, b = b0 + b_l;
       if (a < d.ext_a && b < d.ext_b) {
         const uint32_t b_hi = host_fast_div(b, d.fd_b_in);
         if (b_hi != b / d.fd_b_in.d) return false;
         const uint32_t b_lo = b - b_hi * d.fd_b_in.d;
         const int64_t o = dbase + (int64_t)b_lo * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a * es;
-        if (o % 16 || o < 0 || o + 16 > out_bytes) return false;
-        const int sm = (ca * epu + epu - 1) * (kTileB * es) + (((b_l / epu) ^ ca) << 4) + (b_l % epu) * es;
-        if (sm + es > kTileBytes) return false;
+        if (o % ub || o < 0 || o + ub > out_bytes) return false;
+        const int sm = tile_off(ca * epn + epn - 1, b_l * es);
+        if (sm < 0 || sm + es > kTileBytes) return false;
       }
     }
   }
@@ -523,10 +529,11 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   for (int stage = 0; stage < (int)m.stages.size(); ++stage) {
   const size_t q_lo = m.stages[stage].first_piece, q_hi = q_lo + m.stages[stage].n_pieces;
   const int64_t out_bytes = m.stages[stage].numel * es;
+  for (int ub = 16; ub >= es; ub >>= 1)
   for (int wide = 0; wide < 2; ++wide) {
-    Launch L{kDevTranspose, es, 0, wide, (int)pl->table.size(), 0, 0, stage};
+    Launch L{kDevTranspose, es, ub, wide, (int)pl->table.size(), 0, 0, stage};  // `cons` carries the access width
     for (size_t q = q_lo; q < q_hi; ++q) {
-      if (!is_tr[q]) continue;
+      if (!is_tr[q] || tr[q].tr_unit != ub) continue;
       DevPiece d = tr[q];
       const int64_t in_bytes = slot_numel[d.input] * es;
       if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
@@ -539,7 +546,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       placed[q] = 1;
     }
     if (L.n_pieces == 0) continue;
-    for (size_t q = q_lo; q < q_hi; ++q) {
+    for (size_t q = q_lo; q < q_hi && ub == 16; ++q) {
       const Piece &p = m.pieces[q];
       if (placed[q] || p.src != AMAP_CONST || unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
       DevPiece d;
@@ -722,8 +729,23 @@ static void launch_strip(const DescSource &ds, const Launch &L, const PtrTable &
   }
 }
 
+template <int ES, int UB>
+static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  if constexpr (UB >= ES && UB < 16) {
+    if (L.wide) AMAP_LAUNCH(amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, int64_t);
+    else AMAP_LAUNCH(amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, uint32_t);
+  }
+}
+
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  switch (L.cons) {  // access width of the launch
+    case 8: launch_transpose_narrow<ES, 8>(ds, L, pt, s, pdl); return;
+    case 4: launch_transpose_narrow<ES, 4>(ds, L, pt, s, pdl); return;
+    case 2: launch_transpose_narrow<ES, 2>(ds, L, pt, s, pdl); return;
+    case 1: launch_transpose_narrow<ES, 1>(ds, L, pt, s, pdl); return;
+    default: break;
+  }
   if (L.wide) AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, int64_t);
   else AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, uint32_t);
 }
