@@ -178,11 +178,19 @@ static bool make_strip(DevPiece *d) {
   const int n = d->n_loops;
   if (n < 2) return false;
   int ku = -1;
-  for (int k = n - 2; k >= 0; --k)
-    if (d->ext[k] % kStrip == 0) {
-      ku = k;
-      break;
-    }
+  // a loop along which the source advances by less than a 32-byte sector: walking it makes a thread's loads
+  // share sectors (element-wise gathers such as transposes with odd extents)
+  if (d->input >= 0)
+    for (int k = n - 2; k >= 0; --k)
+      if (d->sstride[k] != 0 && std::llabs(d->sstride[k]) < 32 && d->ext[k] >= kStrip &&
+          (ku < 0 || std::llabs(d->sstride[k]) < std::llabs(d->sstride[ku])))
+        ku = k;
+  if (ku < 0)
+    for (int k = n - 2; k >= 0; --k)
+      if (d->ext[k] % kStrip == 0) {
+        ku = k;
+        break;
+      }
   if (ku < 0) {
     ku = n - 2;
     for (int k = n - 3; k >= 0; --k)
@@ -371,7 +379,8 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
     d->n_items = (uint64_t)blocks;
     return true;
   };
-  for (int ub = 16; ub >= es; ub >>= 1) {
+  // units of a single element gain nothing over the strip kernel's gather (measured): at least two per access
+  for (int ub = 16; ub >= 2 * es; ub >>= 1) {
     if (ub > ptr_align) continue;
     if (try_build(ia_hi, ib_hi, ub)) return true;
     if (ib_hi >= 0 && try_build(ia_hi, -1, ub)) return true;
