@@ -126,6 +126,19 @@ def time_plan(torch, plan, in_sets, out_sets, iters, warmup, stream):
     return start.elapsed_time(stop) * 1e-3 / iters
 
 
+def whole_job_rate(units_per_rank, elapsed_local, world, dist=None, device=None):
+    """Weak scaling without any exchange: every rank moved `units_per_rank`; the job took as long as its slowest
+    rank.  Returns (aggregate units per second over all ranks, max elapsed)."""
+    elapsed = float(elapsed_local)
+    if world > 1:
+        import torch
+
+        t = torch.tensor([elapsed], dtype=torch.float64, device=device if device is not None else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed = float(t.item())
+    return world * units_per_rank / elapsed, elapsed
+
+
 def run_ours(args):
     import torch
 
@@ -192,17 +205,14 @@ def run_ours(args):
         torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    elapsed = start.elapsed_time(stop) * 1e-3
-    if world > 1:
-        t = torch.tensor([elapsed], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed = float(t.item())
+    rate, elapsed = whole_job_rate(bytes_per_step * args.steps, start.elapsed_time(stop) * 1e-3, world,
+                                   dist if world > 1 else None, device)
     # parity of the timed buffers: the round trip must give back the input, bit for bit
     for s in range(n_sets):
         if not torch.equal(zs[s], xs[s]):
             raise SystemExit("round trip differs from the input on buffer set %d" % s)
 
-    value = world * bytes_per_step * args.steps / elapsed / 1e9
+    value = rate / 1e9
     launch_s = elapsed / (args.steps * launches_per_step)
     achieved = bytes_per_launch / launch_s / 1e9
 
@@ -222,14 +232,11 @@ def run_ours(args):
         fwd_p.execute_host([hx], hy, stream.cuda_stream)
         inv_p.execute_host([hy], hz, stream.cuda_stream)
     torch.cuda.synchronize()
-    e2e_elapsed = time.perf_counter() - t3
-    if world > 1:
-        t = torch.tensor([e2e_elapsed], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_elapsed = float(t.item())
+    e2e_rate, e2e_elapsed = whole_job_rate(bytes_per_step * e2e_steps, time.perf_counter() - t3, world,
+                                           dist if world > 1 else None, device)
     if not torch.equal(hz, hx):
         raise SystemExit("host round trip differs from the input")
-    e2e_value = world * bytes_per_step * e2e_steps / e2e_elapsed / 1e9
+    e2e_value = e2e_rate / 1e9
 
     line = {
         "metric": METRIC,

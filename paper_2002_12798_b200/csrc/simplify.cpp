@@ -307,6 +307,24 @@ Status canonicalise(std::vector<Piece> &pieces) {
     work.push_back(std::move(mid));
   }
   merge_fill_pieces(pieces);
+  // The kernels index a piece's items with 32 bits: cut pieces of 2^31 points or more in two along their
+  // outermost loop until every piece is smaller.
+  for (size_t q = 0; q < pieces.size();) {
+    __int128 pts = 1;
+    for (int64_t e : pieces[q].ext) pts *= e;
+    if (pts < ((__int128)1 << 31) || pieces[q].n() == 0) {
+      ++q;
+      continue;
+    }
+    Piece lo = pieces[q], hi = pieces[q];
+    const int64_t half = lo.ext[0] / 2;
+    clip_loop(lo, 0, 0, half);
+    clip_loop(hi, 0, half, hi.ext[0] - half);
+    canonical_loops(lo);
+    canonical_loops(hi);
+    pieces[q] = lo;
+    pieces.insert(pieces.begin() + q + 1, hi);
+  }
   // deterministic order: by destination offset
   std::stable_sort(pieces.begin(), pieces.end(), [](const Piece &a, const Piece &b) { return a.dst.c0 < b.dst.c0; });
   return Status();

@@ -299,6 +299,18 @@ def test_interleaved_stores_are_told_apart_from_overlap():
     assert np.array_equal(eval_map(m, [a, c]), want)
 
 
+def test_huge_pieces_are_cut_below_2_31_points():
+    """An 18 GB byte tensor (shapes only, nothing is allocated): the planner's 32-bit item index must still cover it."""
+    b = B.Builder(1)
+    x = b.input([3, 1 << 16, 3 << 15])
+    m = b.compose(b.transpose(b.slice(x, [0, 0, 1], [3, 1 << 16, 3 << 15], [1, 1, 2]), [1, 0, 2]))
+    ps = m.pieces()
+    assert len(ps) > 1 and all(int(np.prod(p["bounds"], dtype=np.int64)) < 2**31 for p in ps)
+    assert sum(int(np.prod(p["bounds"], dtype=np.int64)) for p in ps) == m.out_numel
+    st = m.plan(device=-1).stats()  # the dry plan walks sampled addresses of every descriptor
+    assert st["bytes_written"] == m.out_numel
+
+
 def test_empty_and_scalar_shapes():
     b = B.Builder(2)
     x = b.input([1, 1])
