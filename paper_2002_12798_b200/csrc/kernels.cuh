@@ -333,8 +333,11 @@ __device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
   }
 }
 
+struct LaunchDesc;
+__device__ __forceinline__ const DevPiece *piece_of_block(const LaunchDesc *ld, uint32_t block);
+
 template <int ES, typename OffT>
-__device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs) {
+__device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs, const LaunchDesc *ld) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
   constexpr int TA = 8 * EPU;      // rows of the tile: 128 bytes of destination run
   constexpr int RB = kTileB * ES;  // bytes per row
@@ -369,38 +372,17 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
   // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
   // reads nothing into the SM and is harmless whatever that kernel still writes); the loads after the wait
   // then start from L2 instead of paying a DRAM round trip with the memory system idle.
-  auto prefetch_rows = [&](const char *base, uint32_t pa0, uint32_t pb0) {
+  auto prefetch_rows = [&](const DevPiece &pp, const char *base, uint32_t pa0, uint32_t pb0) {
     const uint32_t a = pa0 + threadIdx.x;
-    if (a < ext_a && pb0 < ext_b) {
-      const uint32_t a_hi = fast_div(a, sp.fd_a_in);
-      const char *row = base + (int64_t)(a - a_hi * sp.fd_a_in.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)pb0 * ES;
-      const uint32_t bytes = min((uint32_t)kTileB, ext_b - pb0) * ES;
+    if (a < pp.ext_a && pb0 < pp.ext_b) {
+      const uint32_t a_hi = fast_div(a, pp.fd_a_in);
+      const char *row = base + (int64_t)(a - a_hi * pp.fd_a_in.d) * pp.sa[0] + (int64_t)a_hi * pp.sa[1] + (int64_t)pb0 * ES;
+      const uint32_t bytes = min((uint32_t)kTileB, pp.ext_b - pb0) * ES;
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
     }
   };
-  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(src, a0, b0);
+  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(sp, src, a0, b0);
   pdl_wait();
-  // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
-  // blocks further on in the grid): its loads will find their lines in L2.
-  if (sp.prefetch > 1 && threadIdx.x < TA) {
-    uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
-    if (t2 < sp.n_blocks) {
-      uint32_t q2 = fast_div(t2, sp.fd_tiles_b);
-      const uint32_t nb0 = (t2 - q2 * sp.tiles_b) * kTileB;
-      t2 = q2;
-      q2 = fast_div(t2, sp.fd_tiles_a);
-      const uint32_t na0 = (t2 - q2 * sp.tiles_a) * TA;
-      t2 = q2;
-      int64_t nbase = sp.soff;
-      for (int k = sp.n_loops - 1; k >= 0; --k) {
-        q2 = fast_div(t2, sp.fd[k]);
-        nbase += (int64_t)(t2 - q2 * sp.ext[k]) * sp.sstride[k];
-        t2 = q2;
-      }
-      prefetch_rows(ptrs.src[sp.input] + nbase, na0, nb0);
-    }
-  }
-
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];
   {
@@ -425,6 +407,31 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
       }
     }
     issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
+    // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
+    // blocks further on in the grid): its loads will find their lines in L2.
+    if (sp.prefetch > 1 && threadIdx.x < TA) {
+      const uint32_t g = blockIdx.x + (uint32_t)sp.prefetch;
+      // only within this piece: on a launch of several small pieces (measured on configuration 4) hints for
+      // another piece's tiles cost more than they save
+      const DevPiece *np = (g - sp.first_block < sp.n_blocks) ? &sp : nullptr;
+      (void)ld;
+      if (np != nullptr && np->kind == kDevTranspose) {
+        uint32_t t2 = g - np->first_block;
+        uint32_t q2 = fast_div(t2, np->fd_tiles_b);
+        const uint32_t nb0 = (t2 - q2 * np->tiles_b) * kTileB;
+        t2 = q2;
+        q2 = fast_div(t2, np->fd_tiles_a);
+        const uint32_t na0 = (t2 - q2 * np->tiles_a) * TA;
+        t2 = q2;
+        int64_t nbase = np->soff;
+        for (int k = np->n_loops - 1; k >= 0; --k) {
+          q2 = fast_div(t2, np->fd[k]);
+          nbase += (int64_t)(t2 - q2 * np->ext[k]) * np->sstride[k];
+          t2 = q2;
+        }
+        prefetch_rows(*np, ptrs.src[np->input] + nbase, na0, nb0);
+      }
+    }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
@@ -581,6 +588,15 @@ struct LaunchDesc {
   DevPiece piece[kParamPieces];
 };
 
+// the piece that owns block `block` of the launch, or null (past the end, or descriptors not in the parameters)
+__device__ __forceinline__ const DevPiece *piece_of_block(const LaunchDesc *ld, uint32_t block) {
+  if (ld == nullptr) return nullptr;
+  int p = 0;
+  while (p + 1 < ld->n_pieces && block >= ld->piece[p + 1].first_block) ++p;
+  const DevPiece *d = &ld->piece[p];
+  return (block - d->first_block < d->n_blocks) ? d : nullptr;
+}
+
 __device__ __forceinline__ const DevPiece &param_piece(const LaunchDesc &ld) {
   int p = 0;
   while (p + 1 < ld.n_pieces && blockIdx.x >= ld.piece[p + 1].first_block) ++p;
@@ -619,7 +635,7 @@ template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_param(const __grid_constant__ LaunchDesc ld,
                                                                               PtrTable ptrs) {
   pdl_launch_dependents();
-  transpose_body<ES, OffT>(param_piece(ld), ptrs);
+  transpose_body<ES, OffT>(param_piece(ld), ptrs, &ld);
 }
 template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const DevPiece *__restrict__ table,
@@ -627,7 +643,7 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const 
   __shared__ DevPiece sp;
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
-  transpose_body<ES, OffT>(sp, ptrs);
+  transpose_body<ES, OffT>(sp, ptrs, nullptr);
 }
 
 template <int ES, int UB, typename OffT>

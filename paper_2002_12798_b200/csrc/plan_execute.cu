@@ -541,20 +541,20 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   for (int ub = 16; ub >= es; ub >>= 1)
   for (int wide = 0; wide < 2; ++wide) {
     Launch L{kDevTranspose, es, ub, wide, (int)pl->table.size(), 0, 0, stage};  // `cons` carries the access width
+    std::vector<DevPiece> tps, fills;
+    std::vector<size_t> taken;
     for (size_t q = q_lo; q < q_hi; ++q) {
       if (!is_tr[q] || tr[q].tr_unit != ub) continue;
       DevPiece d = tr[q];
       const int64_t in_bytes = slot_numel[d.input] * es;
       if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
       if (!check_transpose_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
-      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
-      d.first_block = L.n_blocks;
-      L.n_blocks += d.n_blocks;
-      L.n_pieces++;
-      pl->table.push_back(d);
-      placed[q] = 1;
+      tps.push_back(d);
+      taken.push_back(q);
     }
-    if (L.n_pieces == 0) continue;
+    if (tps.empty()) continue;
+    // fill pieces with 16-byte units and no constraints ride in the same launch; they go first (stores only,
+    // nothing to wait for), so that the launch's tail is made of blocks that all move data both ways
     for (size_t q = q_lo; q < q_hi && ub == 16; ++q) {
       const Piece &p = m.pieces[q];
       if (placed[q] || p.src != AMAP_CONST || unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
@@ -562,13 +562,18 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       if (build_affine_piece(p, es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
       make_strip(&d);
       if (!check_affine_piece(d, 0, out_bytes)) return fail(AMAP_EOVERFLOW, q);
-      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) continue;
+      fills.push_back(d);
+      taken.push_back(q);
+    }
+    fills.insert(fills.end(), tps.begin(), tps.end());
+    for (DevPiece &d : fills) {
+      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q_lo);
       d.first_block = L.n_blocks;
       L.n_blocks += d.n_blocks;
       L.n_pieces++;
       pl->table.push_back(d);
-      placed[q] = 1;
     }
+    for (size_t q : taken) placed[q] = 1;
     pl->launches.push_back(L);
   }
   // affine kernel: one launch per (unit width, constraints, offset width) present
