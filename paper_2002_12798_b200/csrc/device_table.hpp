@@ -74,8 +74,9 @@ struct DevPiece {
   int64_t ku_ss, ku_ds;
   int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
-  int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less
+  int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less; 0: shifted rows
   int32_t pad1_;
+  int64_t src_bytes;          // size of the source tensor (shifted-row kernel: guards the last aligned chunk)
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b
   FastDiv fd_tiles_a, fd_tiles_b;

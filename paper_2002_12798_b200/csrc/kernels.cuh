@@ -575,6 +575,132 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
 }
 
 // ---------------------------------------------------------------------------
+// The tiled transpose for pieces whose rows are NOT 16-byte aligned (odd
+// extents: 7x7, 13x13, 55x55 feature maps ...).  Global memory is still only
+// touched with aligned 16-byte accesses (plus a few element accesses on edges):
+//   phase 1  for each tile row a, the aligned 16-byte chunks that cover its
+//            source bytes are loaded and stored as chunks of the row; the row's
+//            elements therefore sit shifted by (row address mod 16) bytes;
+//   phase 2  a thread owns one aligned 16-byte slot of a destination row; it
+//            finds each of the slot's elements in its source row, un-shifting
+//            the column, and stores the slot whole when all its elements belong
+//            to the tile, element by element otherwise.
+// Tile: 7 chunks of a by 14 chunks of b, so that a shifted row still fits the
+// 16-chunk shared-memory row and a shifted destination run fits 8 slots.
+// ---------------------------------------------------------------------------
+template <int ES>
+__device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const PtrTable &ptrs) {
+  constexpr int EPU = 16 / ES;
+  constexpr int TAS = 7 * EPU, TBS = 14 * EPU;  // tile extents in elements
+  constexpr int U = (TAS * 16 + kTransposeThreads - 1) / kTransposeThreads;
+  using E = typename Unit<ES>::T;
+  __shared__ __align__(128) unsigned char tile[TAS * 256];
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_b);
+  const uint32_t b0 = (t - q * sp.tiles_b) * TBS;
+  t = q;
+  q = fast_div(t, sp.fd_tiles_a);
+  const uint32_t a0 = (t - q * sp.tiles_a) * TAS;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;  // byte offsets inside the source / destination tensors
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const char *src = ptrs.src[sp.input];
+  char *dst = ptrs.dst;
+  const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
+  const int64_t sa0 = sp.sa[0], sa1 = sp.sa[1], db0 = sp.db[0], db1 = sp.db[1];
+  const int na = (int)min((uint32_t)TAS, sp.ext_a - a0), nb = (int)min((uint32_t)TBS, sp.ext_b - b0);
+  auto row_offset = [&](uint32_t a) -> int64_t {  // source byte offset of element (a, b0)
+    const uint32_t a_hi = fast_div(a, fa);
+    return sbase + (int64_t)(a - a_hi * fa.d) * sa0 + (int64_t)a_hi * sa1 + (int64_t)b0 * ES;
+  };
+  pdl_wait();
+
+  uint4 v[U];
+  bool have[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int idx = threadIdx.x + u * kTransposeThreads;
+    const int a_l = idx >> 4, k = idx & 15;
+    have[u] = false;
+    if (a_l < na) {
+      const int64_t g = row_offset(a0 + a_l);
+      const int64_t first = g & ~(int64_t)15;
+      const int nch = (int)((((g + (int64_t)nb * ES + 15) & ~(int64_t)15) - first) >> 4);
+      const int64_t addr = first + 16 * k;
+      if (k < nch) {
+        have[u] = true;
+        if (addr + 16 <= sp.src_bytes) {
+          v[u] = load_16(src + addr);
+        } else {  // the last chunk of the tensor: only the elements that exist
+          union {
+            uint4 w;
+            E e[EPU];
+          } pk;
+          pk.w = make_uint4(0, 0, 0, 0);
+#pragma unroll
+          for (int e = 0; e < EPU; ++e)
+            if (addr + (e + 1) * ES <= sp.src_bytes) pk.e[e] = load_unit<ES>(src + addr + e * ES);
+          v[u] = pk.w;
+        }
+      }
+    }
+  }
+  issue_barrier();
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const int idx = threadIdx.x + u * kTransposeThreads;
+    const int a_l = idx >> 4, k = idx & 15;
+    if (have[u]) *reinterpret_cast<uint4 *>(tile + a_l * 256 + ((k ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+  }
+  __syncthreads();
+
+  const bool split = fa.d < sp.ext_a;
+  const int row0_shift = (int)(row_offset(a0) & 15);  // valid when a does not merge two loops
+  const int row_step = (int)(sa0 & 15);
+#pragma unroll 1
+  for (int idx = threadIdx.x; idx < TBS * 8; idx += kTransposeThreads) {
+    const int slot = idx & 7, b_l = idx >> 3;
+    if (b_l >= nb) continue;
+    const uint32_t b = b0 + b_l;
+    const uint32_t b_hi = fast_div(b, fb);
+    const int64_t D = dbase + (int64_t)(b - b_hi * fb.d) * db0 + (int64_t)b_hi * db1 + (int64_t)a0 * ES;
+    const int64_t A = (D & ~(int64_t)15) + 16 * slot;
+    const int rel0 = (int)((A - D) / ES);  // tile row of the slot's first element (may be negative)
+    if (rel0 >= na || rel0 + EPU <= 0) continue;
+    union {
+      uint4 w;
+      E e[EPU];
+    } pk;
+    bool all = true;
+#pragma unroll
+    for (int e = 0; e < EPU; ++e) {
+      const int row = rel0 + e;
+      const bool ok = row >= 0 && row < na;
+      all = all && ok;
+      if (ok) {
+        const int shift = split ? (int)(row_offset(a0 + row) & 15) : ((row0_shift + row * row_step) & 15);
+        const int col = b_l * ES + shift;  // byte column inside the shifted row
+        pk.e[e] = *reinterpret_cast<const E *>(tile + row * 256 + ((((col >> 4) ^ ((row / EPU) & 7)) << 4) | (col & 15)));
+      }
+    }
+    if (all) {
+      __stcs(reinterpret_cast<uint4 *>(dst + A), pk.w);
+    } else {
+#pragma unroll
+      for (int e = 0; e < EPU; ++e)
+        if (rel0 + e >= 0 && rel0 + e < na) store_unit<ES>(dst + A + e * ES, pk.e[e]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Entry kernels.  Each family has two: the *_param kernels get up to
 // kParamPieces descriptors BY VALUE in the kernel parameters (constant bank: a
 // block starts its index arithmetic without a round trip to global memory),
@@ -660,6 +786,22 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_narrow_table
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
   transpose_narrow_body<ES, UB, OffT>(sp, ptrs);
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_shifted_param(const __grid_constant__ LaunchDesc ld,
+                                                                                   PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_shifted_body<ES>(param_piece(ld), ptrs);
+}
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_shifted_table(const DevPiece *__restrict__ table,
+                                                                                   int first_piece, int n_pieces,
+                                                                                   PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_shifted_body<ES>(sp, ptrs);
 }
 
 }  // namespace amap

@@ -314,7 +314,7 @@ static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_
 // on that one side only (e.g. (h, w) is one run in an NCHW source but two
 // strides in a padded NHWC destination).
 // ---------------------------------------------------------------------------
-static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiece *d) {
+static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t in_bytes, DevPiece *d) {
   if (es > 8 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
   const int n = p.n();
   if (n < 2) return false;
@@ -387,11 +387,74 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, DevPiec
     if (ia_hi >= 0 && try_build(-1, ib_hi, ub)) return true;
     if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1, ub)) return true;
   }
+  // rows that are not aligned at all: the shifted-row kernel (aligned 16-byte accesses, elements un-shifted in
+  // shared memory); its tile is 7 x 14 chunks
+  if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es)) {
+    const int epu16 = 16 / es;
+    d->tr_unit = 0;
+    d->src_bytes = in_bytes;
+    d->tiles_a = (d->ext_a + 7 * epu16 - 1) / (7 * epu16);
+    d->tiles_b = (d->ext_b + 14 * epu16 - 1) / (14 * epu16);
+    d->fd_tiles_a = make_fastdiv(d->tiles_a);
+    d->fd_tiles_b = make_fastdiv(d->tiles_b);
+    unsigned __int128 blocks = (unsigned __int128)d->tiles_a * d->tiles_b;
+    for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
+    if (blocks > 0x7FFFFFFFull) return false;
+    d->n_blocks = (uint32_t)blocks;
+    d->n_items = (uint64_t)blocks;
+    return true;
+  }
   return false;
+}
+
+// the shifted-row kernel's address arithmetic for one block, replayed on the host
+static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
+  const int es = d.unit_bytes, epu = 16 / es, tas = 7 * epu, tbs = 14 * epu;
+  if (d.src_bytes != in_bytes) return false;
+  uint32_t t = blk;
+  uint32_t q = t / d.tiles_b;
+  const uint32_t b0 = (t - q * d.tiles_b) * tbs;
+  t = q;
+  q = t / d.tiles_a;
+  const uint32_t a0 = (t - q * d.tiles_a) * tas;
+  t = q;
+  int64_t sbase = d.soff, dbase = d.doff;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    q = t / d.ext[k];
+    sbase += (int64_t)(t - q * d.ext[k]) * d.sstride[k];
+    dbase += (int64_t)(t - q * d.ext[k]) * d.dstride[k];
+    t = q;
+  }
+  if (t != 0 || a0 >= d.ext_a || b0 >= d.ext_b) return false;
+  const int na = (int)std::min<uint32_t>(tas, d.ext_a - a0), nb = (int)std::min<uint32_t>(tbs, d.ext_b - b0);
+  auto row_offset = [&](uint32_t a) {
+    const uint32_t a_hi = a / d.fd_a_in.d;
+    return sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b0 * es;
+  };
+  for (int a_l = 0; a_l < na; ++a_l) {
+    const int64_t g = row_offset(a0 + a_l);
+    if (g < 0 || g + (int64_t)nb * es > in_bytes) return false;
+    const int64_t first = g & ~(int64_t)15;
+    const int nch = (int)((((g + (int64_t)nb * es + 15) & ~(int64_t)15) - first) >> 4);
+    if (nch > 16 || first < 0) return false;
+    for (int b_l = 0; b_l < nb; ++b_l) {  // every element must be found inside the 16-chunk row
+      const int col = b_l * es + (int)(g & 15);
+      if ((col >> 4) >= nch || (col >> 4) > 15) return false;
+    }
+  }
+  for (int b_l = 0; b_l < nb; ++b_l) {
+    const uint32_t b = b0 + b_l, b_hi = b / d.fd_b_in.d;
+    const int64_t D = dbase + (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a0 * es;
+    if (D < 0 || D + (int64_t)na * es > out_bytes) return false;
+    // the destination run must fit the 8 aligned slots a thread group covers
+    if (((D & 15) + (int64_t)na * es + 15) / 16 > 8) return false;
+  }
+  return true;
 }
 
 // the kernel's address arithmetic for one block, replayed on the host
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
+  if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
   uint32_t t = blk;
   uint32_t q = host_fast_div(t, d.fd_tiles_b);
@@ -516,7 +579,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     } else {
       reads[p.src] += piece_unique_reads(p, slot_numel[p.src]);
       const bool contiguous = p.n() > 0 && p.srcoff.c[p.n() - 1] == 1 && p.dst.c[p.n() - 1] == 1;
-      if (!contiguous && allow_transpose && build_transpose_piece(p, es, align, &tr[q])) {
+      if (!contiguous && allow_transpose && build_transpose_piece(p, es, align, slot_numel[p.src] * es, &tr[q])) {
         is_tr[q] = 1;
         kind = AMAP_KERNEL_TRANSPOSE;
       } else {
@@ -538,8 +601,9 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   for (int stage = 0; stage < (int)m.stages.size(); ++stage) {
   const size_t q_lo = m.stages[stage].first_piece, q_hi = q_lo + m.stages[stage].n_pieces;
   const int64_t out_bytes = m.stages[stage].numel * es;
-  for (int ub = 16; ub >= es; ub >>= 1)
+  for (int ub : {16, 8, 4, 2, 0})
   for (int wide = 0; wide < 2; ++wide) {
+    if (ub != 0 && ub < 2 * es && ub != 16) continue;
     Launch L{kDevTranspose, es, ub, wide, (int)pl->table.size(), 0, 0, stage};  // `cons` carries the access width
     std::vector<DevPiece> tps, fills;
     std::vector<size_t> taken;
@@ -547,7 +611,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
       if (!is_tr[q] || tr[q].tr_unit != ub) continue;
       DevPiece d = tr[q];
       const int64_t in_bytes = slot_numel[d.input] * es;
-      if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
+      if ((int)((in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && ub != 0) != wide) continue;
       if (!check_transpose_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
       tps.push_back(d);
       taken.push_back(q);
@@ -754,6 +818,9 @@ static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
+    case 0:
+      if constexpr (ES <= 4) AMAP_LAUNCH(amap_transpose_shifted_param, amap_transpose_shifted_table, kTransposeThreads, ES);
+      return;
     case 8: launch_transpose_narrow<ES, 8>(ds, L, pt, s, pdl); return;
     case 4: launch_transpose_narrow<ES, 4>(ds, L, pt, s, pdl); return;
     case 2: launch_transpose_narrow<ES, 2>(ds, L, pt, s, pdl); return;
