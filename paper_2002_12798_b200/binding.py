@@ -309,6 +309,24 @@ class Plan:
         arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
         _check(_lib.amap_execute_static(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute_static")
 
+    def bind(self, srcs, dst, stream=None):
+        """Marshal the arguments of amap_execute once; the returned callable only makes the C call.
+        Keeps `srcs` and `dst` alive.  For loops that launch the same plan on the same buffers many times."""
+        import torch
+
+        s = (stream or torch.cuda.current_stream(dst.device)).cuda_stream
+        arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(t.data_ptr()) for t in srcs])
+        h, d, st, fn = self._h, c_void_p(dst.data_ptr()), c_void_p(s), _lib.amap_execute
+        keep = (list(srcs), dst, self)
+
+        def call():
+            rc = fn(h, arr, d, st)
+            if rc != 0:
+                raise AmapError(rc, "amap_execute")
+
+        call.keep = keep
+        return call
+
     def execute(self, srcs, dst, stream=None):
         """srcs: CUDA tensors (contiguous), dst: CUDA tensor; stream: torch.cuda.Stream or None (current)."""
         import torch

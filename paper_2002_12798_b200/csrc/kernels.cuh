@@ -558,6 +558,7 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
     }
   }
   __syncthreads();
+#pragma unroll 4
   for (int idx = threadIdx.x; idx < N; idx += kTransposeThreads) {
     const int ca = idx % NCA, b_l = idx / NCA;
     const uint32_t a = a0 + ca * EPN, b = b0 + b_l;
