@@ -805,4 +805,33 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_shifted_tabl
   transpose_shifted_body<ES>(sp, ptrs);
 }
 
+// Single-piece launches (the common case) pass just that descriptor: a ninth of the parameter bytes.
+template <int V, int U, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_affine_one(const __grid_constant__ DevPiece p, PtrTable ptrs) {
+  pdl_launch_dependents();
+  affine_body<V, U, NC, OffT>(p, ptrs);
+}
+template <int V, int NC, typename OffT>
+__global__ void __launch_bounds__(kAffineThreads) amap_strip_one(const __grid_constant__ DevPiece p, PtrTable ptrs) {
+  pdl_launch_dependents();
+  strip_body<V, NC, OffT>(p, ptrs);
+}
+template <int ES, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_one(const __grid_constant__ DevPiece p, PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_body<ES, OffT>(p, ptrs, nullptr);
+}
+template <int ES, int UB, typename OffT>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_narrow_one(const __grid_constant__ DevPiece p,
+                                                                                PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_narrow_body<ES, UB, OffT>(p, ptrs);
+}
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_shifted_one(const __grid_constant__ DevPiece p,
+                                                                                 PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_shifted_body<ES>(p, ptrs);
+}
+
 }  // namespace amap

@@ -776,45 +776,46 @@ struct DescSource {
   const DevPiece *table;
 };
 
-#define AMAP_LAUNCH(KP, KT, threads, ...)                                                              \
+#define AMAP_LAUNCH(KO, KP, KT, threads, ...)                                                          \
   do {                                                                                                 \
-    if (ds.ld) launch(KP<__VA_ARGS__>, L.n_blocks, threads, s, pdl, *ds.ld, pt);                       \
+    if (ds.ld && ds.ld->n_pieces == 1) launch(KO<__VA_ARGS__>, L.n_blocks, threads, s, pdl, ds.ld->piece[0], pt); \
+    else if (ds.ld) launch(KP<__VA_ARGS__>, L.n_blocks, threads, s, pdl, *ds.ld, pt);                  \
     else launch(KT<__VA_ARGS__>, L.n_blocks, threads, s, pdl, ds.table, L.first_piece, L.n_pieces, pt); \
   } while (0)
 
 template <int V>
 static void launch_affine(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if (L.cons > 2) {
-    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, int64_t);
-    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, int64_t);
+    else AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, kDevMaxCons, uint32_t);
   } else if (L.cons > 0) {
-    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, int64_t);
-    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, int64_t);
+    else AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 2, uint32_t);
   } else {
-    if (L.wide) AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, int64_t);
-    else AMAP_LAUNCH(amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, int64_t);
+    else AMAP_LAUNCH(amap_affine_one, amap_affine_param, amap_affine_table, kAffineThreads, V, kUnroll, 0, uint32_t);
   }
 }
 
 template <int V>
 static void launch_strip(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if (L.cons > 2) {
-    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, int64_t);
-    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, int64_t);
+    else AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, kDevMaxCons, uint32_t);
   } else if (L.cons > 0) {
-    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 2, int64_t);
-    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 2, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, 2, int64_t);
+    else AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, 2, uint32_t);
   } else {
-    if (L.wide) AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 0, int64_t);
-    else AMAP_LAUNCH(amap_strip_param, amap_strip_table, kAffineThreads, V, 0, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, 0, int64_t);
+    else AMAP_LAUNCH(amap_strip_one, amap_strip_param, amap_strip_table, kAffineThreads, V, 0, uint32_t);
   }
 }
 
 template <int ES, int UB>
 static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   if constexpr (UB >= ES && UB < 16) {
-    if (L.wide) AMAP_LAUNCH(amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, int64_t);
-    else AMAP_LAUNCH(amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, uint32_t);
+    if (L.wide) AMAP_LAUNCH(amap_transpose_narrow_one, amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, int64_t);
+    else AMAP_LAUNCH(amap_transpose_narrow_one, amap_transpose_narrow_param, amap_transpose_narrow_table, kTransposeThreads, ES, UB, uint32_t);
   }
 }
 
@@ -822,7 +823,7 @@ template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
     case 0:
-      if constexpr (ES <= 4) AMAP_LAUNCH(amap_transpose_shifted_param, amap_transpose_shifted_table, kTransposeThreads, ES);
+      if constexpr (ES <= 4) AMAP_LAUNCH(amap_transpose_shifted_one, amap_transpose_shifted_param, amap_transpose_shifted_table, kTransposeThreads, ES);
       return;
     case 8: launch_transpose_narrow<ES, 8>(ds, L, pt, s, pdl); return;
     case 4: launch_transpose_narrow<ES, 4>(ds, L, pt, s, pdl); return;
@@ -830,8 +831,8 @@ static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTab
     case 1: launch_transpose_narrow<ES, 1>(ds, L, pt, s, pdl); return;
     default: break;
   }
-  if (L.wide) AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, int64_t);
-  else AMAP_LAUNCH(amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, uint32_t);
+  if (L.wide) AMAP_LAUNCH(amap_transpose_one, amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, int64_t);
+  else AMAP_LAUNCH(amap_transpose_one, amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, uint32_t);
 }
 
 static cudaError_t enqueue(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
