@@ -35,7 +35,8 @@ extern "C" const char *amap_last_cuda_error(void) { return g_cuda_error.c_str();
 struct Launch {
   int kind;  // DevKind
   int unit;  // bytes per item (affine kernel) / element size (transpose kernel)
-  int cons;  // affine kernel: constraint slots evaluated per unit (0, 2 or kDevMaxCons)
+  int cons;  // affine / strip kernel: constraint slots evaluated per unit (0, 2 or kDevMaxCons)
+             // transpose kernel: bytes per global access (16, 8, 4, 2) or 0 for the shifted-row kernel
   int wide;  // affine kernel: 1 when a byte offset can reach 4 GiB (64-bit offsets)
   int first_piece;
   int n_pieces;
@@ -526,6 +527,113 @@ static bool check_transpose_piece(const DevPiece &d, int64_t in_bytes, int64_t o
   return true;
 }
 
+// ---------------------------------------------------------------------------
+// Building the launches of one stage
+// ---------------------------------------------------------------------------
+struct PlanCtx {
+  const Map &m;
+  const amap_plan_opts &o;
+  int es;
+  const std::vector<int64_t> &slot_numel;  // elements behind each source slot: inputs, then temporaries
+  const std::vector<int> &unit_of;         // unit width chosen per piece (affine / strip kernels)
+  const std::vector<DevPiece> &tr;         // transpose descriptor per piece (valid where is_tr)
+  const std::vector<char> &is_tr;
+  std::vector<char> placed;                // piece already belongs to a launch
+  amap_plan_t *pl;
+};
+
+static int plan_fail(int rc, size_t piece) {
+  if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", piece, rc);
+  return rc;
+}
+
+static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
+  if ((uint64_t)L->n_blocks + d.n_blocks > 0x7FFFFFFFull) return false;
+  d.first_block = L->n_blocks;
+  L->n_blocks += d.n_blocks;
+  L->n_pieces++;
+  pl->table.push_back(d);
+  return true;
+}
+
+// One launch of the transpose kernel per (access width, offset width) present.  Fill pieces with 16-byte units
+// and no constraints ride in the 16-byte launch (first: they only store and wait for nothing), so that padding
+// borders do not cost a launch of their own.
+static int plan_stage_transposes(PlanCtx &c, int stage) {
+  const StageInfo &st = c.m.stages[stage];
+  const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
+  const int64_t out_bytes = st.numel * c.es;
+  for (int access : {16, 8, 4, 2, 0})
+    for (int wide = 0; wide < 2; ++wide) {
+      Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
+      std::vector<DevPiece> transposes, fills;
+      std::vector<size_t> taken;
+      for (size_t q = q_lo; q < q_hi; ++q) {
+        if (!c.is_tr[q] || c.tr[q].tr_unit != access) continue;
+        const DevPiece &d = c.tr[q];
+        const int64_t in_bytes = c.slot_numel[d.input] * c.es;
+        const bool needs_wide = (in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && access != 0;
+        if ((int)needs_wide != wide) continue;
+        if (!check_transpose_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
+        transposes.push_back(d);
+        taken.push_back(q);
+      }
+      if (transposes.empty()) continue;
+      for (size_t q = q_lo; q < q_hi && access == 16; ++q) {
+        const Piece &p = c.m.pieces[q];
+        if (c.placed[q] || p.src != AMAP_CONST || c.unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
+        DevPiece d;
+        if (build_affine_piece(p, c.es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
+        make_strip(&d);
+        if (!check_affine_piece(d, 0, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
+        fills.push_back(d);
+        taken.push_back(q);
+      }
+      for (const DevPiece &d : fills)
+        if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
+      for (const DevPiece &d : transposes)
+        if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
+      for (size_t q : taken) c.placed[q] = 1;
+      c.pl->launches.push_back(L);
+    }
+  return AMAP_OK;
+}
+
+// Everything else: one launch per (unit width, constraint slots, offset width, strip or per-unit kernel) present.
+static int plan_stage_strips(PlanCtx &c, int stage) {
+  const StageInfo &st = c.m.stages[stage];
+  const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
+  const int64_t out_bytes = st.numel * c.es;
+  for (int V = 16; V >= 1; V >>= 1)
+    for (int cons : {0, 2, kDevMaxCons})
+      for (int wide = 0; wide < 2; ++wide)
+        for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
+          Launch L{kind, V, cons, wide, (int)c.pl->table.size(), 0, 0, stage};
+          for (size_t q = q_lo; q < q_hi; ++q) {
+            if (c.placed[q] || c.unit_of[q] != V) continue;
+            const Piece &p = c.m.pieces[q];
+            const int n_cons = (int)(p.guards.size() + p.domain.size());
+            if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
+            const int64_t in_bytes = (p.src >= 0) ? c.slot_numel[p.src] * c.es : 0;
+            if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
+            DevPiece d;
+            const int rc = build_affine_piece(p, c.es, V, &d);
+            if (rc != AMAP_OK) return plan_fail(rc, q);
+            if (d.n_items == 0) {
+              c.placed[q] = 1;
+              continue;
+            }
+            if (c.o.force_kernel != AMAP_KERNEL_GATHER) make_strip(&d);
+            if (d.kind != kind) continue;
+            if (!check_affine_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
+            if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q);
+            c.placed[q] = 1;
+          }
+          if (L.n_pieces > 0) c.pl->launches.push_back(L);
+        }
+  return AMAP_OK;
+}
+
 extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts, amap_plan_t **out_plan) {
   if (!map || !out_plan) return AMAP_EINVAL;
   amap_plan_opts o;
@@ -593,85 +701,15 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   }
   for (size_t q = 0; q < reads.size(); ++q) pl->stats.bytes_read += std::min(reads[q], slot_numel[q]) * es;
 
-  auto fail = [&](int rc, size_t q) {
-    if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", q, rc);
-    delete pl;
-    return rc;
-  };
-  // one launch of the transpose kernel for all its pieces (per offset width); fill pieces with 16-byte units and
-  // no constraints ride in the first such launch, so that padding borders do not cost a launch of their own
-  std::vector<char> placed(m.pieces.size(), 0);
+  PlanCtx ctx{m, o, es, slot_numel, unit_of, tr, is_tr, std::vector<char>(m.pieces.size(), 0), pl};
   for (int stage = 0; stage < (int)m.stages.size(); ++stage) {
-  const size_t q_lo = m.stages[stage].first_piece, q_hi = q_lo + m.stages[stage].n_pieces;
-  const int64_t out_bytes = m.stages[stage].numel * es;
-  for (int ub : {16, 8, 4, 2, 0})
-  for (int wide = 0; wide < 2; ++wide) {
-    if (ub != 0 && ub < 2 * es && ub != 16) continue;
-    Launch L{kDevTranspose, es, ub, wide, (int)pl->table.size(), 0, 0, stage};  // `cons` carries the access width
-    std::vector<DevPiece> tps, fills;
-    std::vector<size_t> taken;
-    for (size_t q = q_lo; q < q_hi; ++q) {
-      if (!is_tr[q] || tr[q].tr_unit != ub) continue;
-      DevPiece d = tr[q];
-      const int64_t in_bytes = slot_numel[d.input] * es;
-      if ((int)((in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && ub != 0) != wide) continue;
-      if (!check_transpose_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
-      tps.push_back(d);
-      taken.push_back(q);
+    int rc = plan_stage_transposes(ctx, stage);
+    if (rc == AMAP_OK) rc = plan_stage_strips(ctx, stage);
+    if (rc != AMAP_OK) {
+      delete pl;
+      return rc;
     }
-    if (tps.empty()) continue;
-    // fill pieces with 16-byte units and no constraints ride in the same launch; they go first (stores only,
-    // nothing to wait for), so that the launch's tail is made of blocks that all move data both ways
-    for (size_t q = q_lo; q < q_hi && ub == 16; ++q) {
-      const Piece &p = m.pieces[q];
-      if (placed[q] || p.src != AMAP_CONST || unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
-      DevPiece d;
-      if (build_affine_piece(p, es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
-      make_strip(&d);
-      if (!check_affine_piece(d, 0, out_bytes)) return fail(AMAP_EOVERFLOW, q);
-      fills.push_back(d);
-      taken.push_back(q);
-    }
-    fills.insert(fills.end(), tps.begin(), tps.end());
-    for (DevPiece &d : fills) {
-      if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q_lo);
-      d.first_block = L.n_blocks;
-      L.n_blocks += d.n_blocks;
-      L.n_pieces++;
-      pl->table.push_back(d);
-    }
-    for (size_t q : taken) placed[q] = 1;
-    pl->launches.push_back(L);
   }
-  // affine kernel: one launch per (unit width, constraints, offset width) present
-  for (int V = 16; V >= 1; V >>= 1)
-    for (int cons : {0, 2, kDevMaxCons})
-      for (int wide = 0; wide < 2; ++wide)
-       for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
-        Launch L{kind, V, cons, wide, (int)pl->table.size(), 0, 0, stage};
-        for (size_t q = q_lo; q < q_hi; ++q) {
-          if (placed[q] || unit_of[q] != V) continue;
-          const Piece &p = m.pieces[q];
-          const int n_cons = (int)(p.guards.size() + p.domain.size());
-          if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
-          const int64_t in_bytes = (p.src >= 0) ? slot_numel[p.src] * es : 0;
-          if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
-          DevPiece d;
-          const int rc = build_affine_piece(p, es, V, &d);
-          if (rc != AMAP_OK) return fail(rc, q);
-          if (d.n_items == 0) continue;
-          if (o.force_kernel != AMAP_KERNEL_GATHER) make_strip(&d);
-          if (d.kind != kind) continue;
-          if (!check_affine_piece(d, in_bytes, out_bytes)) return fail(AMAP_EOVERFLOW, q);
-          if ((uint64_t)L.n_blocks + d.n_blocks > 0x7FFFFFFFull) return fail(AMAP_EUNSUPPORTED, q);
-          d.first_block = L.n_blocks;
-          L.n_blocks += d.n_blocks;
-          L.n_pieces++;
-          pl->table.push_back(d);
-        }
-        if (L.n_pieces > 0) pl->launches.push_back(L);
-      }
-  }  // stages
   for (int k : pl->piece_kernel) {
     const int slot = (k == AMAP_KERNEL_GATHER) ? 0 : (k == AMAP_KERNEL_COPY) ? 1 : (k == AMAP_KERNEL_TRANSPOSE) ? 2 : 3;
     pl->stats.kernel_kind[slot]++;
