@@ -209,6 +209,8 @@ typedef enum amap_kernel_kind {
 #define AMAP_PLAN_NO_PDL 1
 /* do not prefetch a block's first source lines into L2 while the previous kernel on the stream drains */
 #define AMAP_PLAN_NO_PREFETCH 2
+/* (The environment variable AMAP_PREFETCH_DISTANCE, read by amap_plan, overrides how many blocks ahead the
+ * transpose kernel prefetches; the default is the number of blocks resident on the device at once.) */
 
 typedef struct amap_plan_opts {
   int32_t force_kernel;     /* amap_kernel_kind; AUTO picks per piece; a family that cannot run a piece falls back to GATHER */
@@ -242,7 +244,8 @@ int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
  *   dst_dev_ptr   DEVICE pointer to the output (out_numel * elem_size bytes)
  *   cuda_stream   a cudaStream_t (NULL = the legacy default stream)
  * Enqueues the plan's kernel(s) and returns without synchronising or
- * allocating.  Source and destination must not overlap.  Pointers must be
+ * allocating.  Source and destination must not overlap (AMAP_EINVAL if the
+ * byte ranges do).  Pointers must be
  * aligned to the plan's pointer_align, else AMAP_EALIGN and nothing is
  * enqueued.  Launch failures give AMAP_ECUDA.
  * ------------------------------------------------------------------------- */

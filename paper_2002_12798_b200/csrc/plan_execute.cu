@@ -913,7 +913,11 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
   for (size_t q = 0; q < n_in; ++q) {
     if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
     if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
-    if (src_dev_ptrs[q] == dst_dev_ptr) return AMAP_EINVAL;
+    {  // source and destination ranges must not overlap
+      const uintptr_t s0 = (uintptr_t)src_dev_ptrs[q], s1 = s0 + (uintptr_t)plan->in_numel[q] * plan->elem_size;
+      const uintptr_t d0 = (uintptr_t)dst_dev_ptr, d1 = d0 + (uintptr_t)plan->out_numel * plan->elem_size;
+      if (s0 < d1 && d0 < s1) return AMAP_EINVAL;
+    }
     pt.src[q] = (const char *)src_dev_ptrs[q];
   }
   for (size_t k = 0; k < plan->temps.size(); ++k) pt.src[n_in + k] = (const char *)plan->temps[k];

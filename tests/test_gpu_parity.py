@@ -176,6 +176,42 @@ def test_misaligned_pointer_is_refused(B):
     assert np.array_equal(got, want.reshape(-1))
 
 
+def test_overlapping_buffers_are_refused(B):
+    import torch
+
+    chain = W.reduced_configs()["c2_fwd_rag"]
+    m = B.compose_chain(chain)
+    plan = m.plan(0)
+    buf = torch.zeros(m.out_numel * 2 + 64, dtype=torch.int16, device="cuda")
+    with pytest.raises(B.AmapError) as e:  # output starts inside the input
+        plan.execute_ptrs([buf.data_ptr()], buf.data_ptr() + 32, 0)
+    assert e.value.code == -1
+
+
+def test_execute_can_be_captured_in_a_cuda_graph(B):
+    """amap_execute neither synchronises nor allocates, so a stream capture can record it; replays must copy."""
+    import torch
+
+    chain = W.reduced_configs()["c2_fwd_mid"]
+    (x,) = W.make_inputs(chain)
+    want = oracle.run_chain(chain, [x]).reshape(-1)
+    m = B.compose_chain(chain)
+    plan = m.plan(0)
+    src = torch.from_numpy(x.view(np.int16)).cuda()
+    dst = torch.zeros(m.out_numel, dtype=torch.int16, device="cuda")
+    plan.execute([src], dst)  # first use outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        plan.execute([src], dst)
+        plan.execute([src], dst)
+    for _ in range(3):
+        dst.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(dst.cpu().numpy().view(np.uint16), want)
+
+
 def test_plan_stats_count_algorithmic_bytes(B):
     full = W.full_configs()
     want = {
