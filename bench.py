@@ -201,20 +201,60 @@ def run_ours(args):
         fwd_p.execute([xs[s]], ys[s], stream)
     for i in range(args.warmup):
         step(i)
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if world > 1:
-        dist.barrier()
     torch.cuda.synchronize()
-    with ClockSampler(local) as clocks:
-        start.record(stream)
+
+    # The timed loop is launch-bound (16 us kernels): capture G steps once in a CUDA graph and replay it K / G times.
+    # The same amap_execute calls are recorded, so the same kernels run; only the host's launch work disappears.
+    graph, G, gstream = None, 0, None
+    if not args.no_graph:
+        G = max((g for g in range(n_sets, 201, n_sets) if args.steps % g == 0), default=0)
+    if G:
+        try:
+            gstream = torch.cuda.Stream(device)
+            gf = [fwd_p.bind([xs[s]], ys[s], gstream) for s in range(n_sets)]
+            gi = [inv_p.bind([ys[s]], zs[s], gstream) for s in range(n_sets)]
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gstream):
+                for i in range(G):
+                    gf[i % n_sets]()
+                    gi[(i % n_sets + half) % n_sets]()
+        except Exception as exc:  # capture not available: time plain stream launches
+            print("CUDA graph capture failed (%s); timing stream launches" % exc, file=sys.stderr)
+            graph = None
+
+    def timed(run, on_stream):
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        with ClockSampler(local) as clk:
+            start.record(on_stream)
+            run()
+            stop.record(on_stream)
+            torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        r, el = whole_job_rate(bytes_per_step * args.steps, start.elapsed_time(stop) * 1e-3, world,
+                               dist if world > 1 else None, device)
+        return r, el, clk
+
+    def stream_loop():
         for i in range(args.steps):
             step(i)
-        stop.record(stream)
-        torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    rate, elapsed = whole_job_rate(bytes_per_step * args.steps, start.elapsed_time(stop) * 1e-3, world,
-                                   dist if world > 1 else None, device)
+
+    stream_rate, stream_elapsed, clocks = timed(stream_loop, stream)
+    rate, elapsed, launch_mode = stream_rate, stream_elapsed, "stream launches"
+    if graph is not None:
+        with torch.cuda.stream(gstream):
+            for _ in range(max(1, args.warmup // G)):
+                graph.replay()
+
+            def graph_loop():
+                for _ in range(args.steps // G):
+                    graph.replay()
+
+            rate, elapsed, clocks = timed(graph_loop, gstream)
+        launch_mode = "CUDA graph of %d steps replayed %d times" % (G, args.steps // G)
     # parity of the timed buffers: the round trip must give back the input, bit for bit
     for s in range(n_sets):
         if not torch.equal(zs[s], xs[s]):
@@ -266,6 +306,7 @@ def run_ours(args):
             "l2": "inputs larger than L2: rotation over %d buffer sets, %d MB in all (L2 %d MB)"
             % (n_sets, 3 * n_sets * nbytes // 2**20, l2 // 2**20),
             "parallelism": "replicas (batch shards, no exchange)" if world > 1 else "single GPU",
+            "launch_mode": launch_mode,
         },
         "pct_of_nominal_8TBs": round(100 * value / world / NOMINAL_PEAK_GBS, 1),
         "roofline": {
@@ -289,6 +330,12 @@ def run_ours(args):
             "steps": e2e_steps,
         },
         "gpu_launches": args.steps * launches_per_step,
+        "stream_launches": {
+            "value": round(stream_rate / 1e9, 1),
+            "unit": "GB/s",
+            "us_per_launch": round(stream_elapsed / (args.steps * launches_per_step) * 1e6, 2),
+            "note": "the same K steps as individual amap_execute calls on the stream, no graph",
+        },
         "clocks": clocks.summary(),
         "host_compose_ms": round((t1 - t0) * 1e3, 3),
         "host_plan_ms": round((t2 - t1) * 1e3, 3),
@@ -428,6 +475,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=100)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="time individual stream launches only")
     ap.add_argument("--all-configs", action="store_true", help="also time configurations 3, 4, 5 (adds about a minute)")
     ap.add_argument("--plan-flags", type=int, default=0, help="amap_plan_opts.flags for every plan (1: no programmatic dependent launch, 2: no L2 prefetch)")
     ap.add_argument("--config", default=None, help="time ONE configuration's kernel loop only (for profiler captures) and print its figures")
