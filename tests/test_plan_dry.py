@@ -1,0 +1,74 @@
+"""Planner decisions on the CPU (dry plans: amap_plan with device = -1 makes no CUDA call).  The dry plan also
+replays every descriptor's address arithmetic on the host, so a wrong table fails here, not on a GPU."""
+import pytest
+
+from paper_2002_12798_b200 import binding as B
+from paper_2002_12798_b200 import workloads as W
+
+
+def kernels(chain, **kw):
+    st = B.compose_chain(chain).plan(device=-1, **kw).stats()
+    return st["kernels"], st["n_launches"], st["n_stages"]
+
+
+def test_full_configurations_each_run_as_one_launch():
+    full = W.full_configs()
+    assert kernels(full["c2_fwd"]) == ({"gather": 0, "copy": 0, "transpose": 1, "fill": 0}, 1, 1)
+    assert kernels(full["c2_inv"]) == ({"gather": 0, "copy": 0, "transpose": 1, "fill": 0}, 1, 1)
+    assert kernels(full["c3"]) == ({"gather": 0, "copy": 2, "transpose": 0, "fill": 0}, 1, 1)
+    assert kernels(full["c4"]) == ({"gather": 0, "copy": 0, "transpose": 4, "fill": 4}, 1, 1)
+    assert kernels(full["c5"]) == ({"gather": 0, "copy": 1, "transpose": 0, "fill": 0}, 1, 1)
+    assert kernels(full["c1"])[0]["gather"] == 1  # a strided innermost load: element-wise gather
+
+
+def test_forced_families():
+    c2 = W.full_configs()["c2_fwd"]
+    assert kernels(c2, force_kernel=B.KERNEL_GATHER)[0]["gather"] == 1
+    assert kernels(c2, force_kernel=B.KERNEL_COPY)[0]["transpose"] == 0
+    assert kernels(c2, pointer_align=2)[0]["transpose"] == 0  # no 16-byte promise: no vector kernels
+
+
+@pytest.mark.parametrize(
+    "shape,expect",
+    [
+        ((4, 256, 56, 56), "transpose"),  # 16-byte rows on both sides
+        ((4, 256, 14, 14), "transpose"),  # 8-byte aligned rows: narrow units
+        ((4, 254, 54, 54), "transpose"),  # 4-byte aligned
+        ((4, 256, 27, 27), "gather"),     # odd source rows, aligned destination rows: strip kernel
+    ],
+)
+def test_transpose_family_by_alignment(shape, expect):
+    n, c, h, w = shape
+    k, launches, _ = kernels(W.c2_nchw_to_nhwc(N=n, C=c, H=h, W=w))
+    assert k[expect] == 1 and launches == 1
+
+
+def test_shifted_transpose_for_misaligned_destination_rows():
+    k, _, _ = kernels(W.c2_nhwc_to_nchw(N=4, C=256, H=27, W=27))
+    assert k["transpose"] == 1
+    k, _, _ = kernels(W.c2_nhwc_to_nchw(N=4, C=255, H=27, W=27))  # source rows misaligned too
+    assert k["gather"] == 1
+
+
+def test_unfused_chain_has_one_stage_per_operator_and_moves_more_bytes():
+    c3 = W.full_configs()["c3"]
+    fused = B.compose_chain(c3).plan(device=-1).stats()
+    unfused = B.compose_chain(c3, B.COMPOSE_NO_FUSE).plan(device=-1).stats()
+    assert fused["n_stages"] == 1 and unfused["n_stages"] == 7
+    assert fused["bytes_read"] + fused["bytes_written"] == 805306368
+    assert unfused["bytes_read"] + unfused["bytes_written"] == 3758096384
+
+
+def test_dry_plan_cannot_execute():
+    plan = B.compose_chain(W.c1_small_chain()).plan(device=-1)
+    with pytest.raises(B.AmapError) as e:
+        plan.execute_ptrs([0x1000], 0x2000, 0)
+    assert e.value.code == -1
+
+
+def test_bad_plan_options():
+    m = B.compose_chain(W.c1_small_chain())
+    for kw in ({"pointer_align": 3}, {"pointer_align": 2}, {"flags": 64}, {"force_kernel": 9}, {"device": -2}):
+        with pytest.raises(B.AmapError) as e:
+            m.plan(**{"device": -1, **kw})
+        assert e.value.code == -1, kw
