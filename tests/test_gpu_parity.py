@@ -130,6 +130,23 @@ def test_tile_broadcast(B):
     assert np.array_equal(got.reshape(80, 15), np.tile(xs[0], (5, 2)).T)
 
 
+def test_random_statement_chains(B):
+    """Raw load/store statements with arbitrary small affine maps (interleaved and merged stores, guards,
+    temporaries where a pair cannot be eliminated)."""
+    from test_compose_fuzz import random_stmt_chain
+
+    r = np.random.default_rng(2002)
+    staged = 0
+    for trial in range(150):
+        chain = random_stmt_chain(r)
+        xs = [x + np.uint32(100) for x in W.make_index_tagged_inputs(chain)]
+        want = oracle.run_chain(chain, xs)
+        got, plan = run_gpu(B, chain, xs, force=trial % 3)
+        staged += plan.stats()["n_stages"] > 1
+        assert np.array_equal(got, want.reshape(-1)), (trial, chain.ops)
+    assert staged > 0
+
+
 @pytest.mark.parametrize("dtype,es", [("u8", 1), ("u64", 8)])
 def test_other_element_sizes(B, dtype, es):
     chain = W.c3_head_split(B=2, S=20, heads=3, D=16, keep=11, dtype=dtype)
