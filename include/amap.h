@@ -209,8 +209,6 @@ typedef enum amap_kernel_kind {
 #define AMAP_PLAN_NO_PDL 1
 /* do not prefetch a block's first source lines into L2 while the previous kernel on the stream drains */
 #define AMAP_PLAN_NO_PREFETCH 2
-/* keep the transposed pieces of a concat as separate pieces instead of joining them into one whose tiles span the joins */
-#define AMAP_PLAN_NO_JOIN 4
 /* (The environment variable AMAP_PREFETCH_DISTANCE, read by amap_plan, overrides how many blocks ahead the
  * transpose kernel prefetches; the default is the number of blocks resident on the device at once.) */
 

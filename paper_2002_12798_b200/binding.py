@@ -19,7 +19,6 @@ KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2
 COMPOSE_NO_FUSE = 1
 PLAN_NO_PDL = 1
 PLAN_NO_PREFETCH = 2
-PLAN_NO_JOIN = 4
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
 
 EXPORTS = [

@@ -7,8 +7,6 @@ namespace amap {
 constexpr int kDevMaxLoops = 12;
 constexpr int kDevMaxCons = 6;
 constexpr int kMaxInputs = 24;
-constexpr int kMaxSegments = 4;     // sources joined along a in one transpose piece
-constexpr int kSegBatchLoops = 4;   // batch loops such a piece may have
 constexpr int kStrip = 8;  // units per thread in the affine and strip kernels
 
 // unsigned 32-bit division by an invariant divisor, multiply-and-shift form
@@ -85,16 +83,6 @@ struct DevPiece {
   FastDiv fd_a_in, fd_b_in;  // inner extents of the merged indices
   int64_t sa[2];             // source byte strides of (a_lo, a_hi)
   int64_t db[2];             // destination byte strides of (b_lo, b_hi)
-  // Joined sources: a concat along the destination-contiguous index followed by a transpose gives pieces that
-  // differ only in their source.  n_seg > 1 makes them ONE piece whose rows [seg_a[q], seg_a[q+1]) come from
-  // source slot seg_input[q] at byte offset seg_soff[q] + sum_k i_k * seg_ss[q][k] over the batch loops (unused
-  // seg_a entries hold 0xFFFFFFFF).  Tiles then span the joins, so no tile is left half empty by a short operand.
-  int32_t n_seg;
-  int32_t seg_input[kMaxSegments];
-  uint32_t seg_a[kMaxSegments];
-  int32_t pad2_;
-  int64_t seg_soff[kMaxSegments];
-  int64_t seg_ss[kMaxSegments][kSegBatchLoops];
 };
 
 struct PtrTable {

@@ -336,7 +336,7 @@ __device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
 struct LaunchDesc;
 __device__ __forceinline__ const DevPiece *piece_of_block(const LaunchDesc *ld, uint32_t block);
 
-template <int ES, typename OffT, bool MULTI = false>
+template <int ES, typename OffT>
 __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs, const LaunchDesc *ld) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
   constexpr int TA = 8 * EPU;      // rows of the tile: 128 bytes of destination run
@@ -369,32 +369,6 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
   const char *src = ptrs.src[sp.input] + sbase;
   char *dst = ptrs.dst + dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
-  __shared__ const char *segbase[kMaxSegments];  // MULTI: where row seg_a[q] of this batch starts in its source
-  if constexpr (MULTI) {
-    if (threadIdx.x < (unsigned)sp.n_seg) {
-      const int sg = threadIdx.x;
-      uint32_t tb = (blockIdx.x - sp.first_block);
-      tb = fast_div(fast_div(tb, sp.fd_tiles_b), sp.fd_tiles_a);
-      int64_t off = sp.seg_soff[sg];
-      for (int k = sp.n_loops - 1; k >= 0; --k) {
-        const uint32_t qq = fast_div(tb, sp.fd[k]);
-        off += (int64_t)(tb - qq * sp.ext[k]) * sp.seg_ss[sg][k];
-        tb = qq;
-      }
-      segbase[sg] = ptrs.src[sp.seg_input[sg]] + off;
-    }
-    __syncthreads();
-  }
-  // the source row of tile index a (MULTI: pick the operand that holds it)
-  auto row_ptr = [&](uint32_t a) -> const char * {
-    if constexpr (MULTI) {
-      const int sg = (int)(a >= sp.seg_a[1]) + (int)(a >= sp.seg_a[2]) + (int)(a >= sp.seg_a[3]);
-      return segbase[sg] + (int64_t)(a - sp.seg_a[sg]) * sp.sa[0];
-    } else {
-      const uint32_t a_hi = fast_div(a, sp.fd_a_in);
-      return src + (int64_t)(a - a_hi * sp.fd_a_in.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1];
-    }
-  };
   // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
   // reads nothing into the SM and is harmless whatever that kernel still writes); the loads after the wait
   // then start from L2 instead of paying a DRAM round trip with the memory system idle.
@@ -407,15 +381,7 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
     }
   };
-  if constexpr (MULTI) {
-    if (sp.prefetch && threadIdx.x < TA && a0 + threadIdx.x < ext_a && b0 < ext_b) {
-      const uint32_t bytes = min((uint32_t)kTileB, ext_b - b0) * ES;
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row_ptr(a0 + threadIdx.x) + (int64_t)b0 * ES), "r"(bytes)
-                   : "memory");
-    }
-  } else {
-    if (sp.prefetch && threadIdx.x < TA) prefetch_rows(sp, src, a0, b0);
-  }
+  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(sp, src, a0, b0);
   pdl_wait();
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];
@@ -430,24 +396,20 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
       const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
       v[u] = make_uint4(0, 0, 0, 0);
       if (a < ext_a && b < ext_b) {
-        if constexpr (MULTI) {
-          v[u] = load_16(row_ptr(a) + (int64_t)b * ES);
+        OffT off = (OffT)(b * ES);
+        if (split) {
+          const uint32_t a_hi = fast_div(a, fa);
+          off += (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1;
         } else {
-          OffT off = (OffT)(b * ES);
-          if (split) {
-            const uint32_t a_hi = fast_div(a, fa);
-            off += (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1;
-          } else {
-            off += (OffT)a * sa0;
-          }
-          v[u] = load_16(src + off);
+          off += (OffT)a * sa0;
         }
+        v[u] = load_16(src + off);
       }
     }
     issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
     // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
     // blocks further on in the grid): its loads will find their lines in L2.
-    if (!MULTI && sp.prefetch > 1 && threadIdx.x < TA) {
+    if (sp.prefetch > 1 && threadIdx.x < TA) {
       const uint32_t g = blockIdx.x + (uint32_t)sp.prefetch;
       // only within this piece: on a launch of several small pieces (measured on configuration 4) hints for
       // another piece's tiles cost more than they save
@@ -809,28 +771,6 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const 
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
   transpose_body<ES, OffT>(sp, ptrs, nullptr);
-}
-
-template <int ES, typename OffT>
-__global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_joined_param(const __grid_constant__ LaunchDesc ld,
-                                                                                     PtrTable ptrs) {
-  pdl_launch_dependents();
-  transpose_body<ES, OffT, true>(param_piece(ld), ptrs, &ld);
-}
-template <int ES, typename OffT>
-__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_joined_table(const DevPiece *__restrict__ table,
-                                                                                  int first_piece, int n_pieces,
-                                                                                  PtrTable ptrs) {
-  __shared__ DevPiece sp;
-  pdl_launch_dependents();
-  fetch_piece(table, first_piece, n_pieces, &sp);
-  transpose_body<ES, OffT, true>(sp, ptrs, nullptr);
-}
-template <int ES, typename OffT>
-__global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_joined_one(const __grid_constant__ DevPiece p,
-                                                                                   PtrTable ptrs) {
-  pdl_launch_dependents();
-  transpose_body<ES, OffT, true>(p, ptrs, nullptr);
 }
 
 template <int ES, int UB, typename OffT>

@@ -42,7 +42,6 @@ struct Launch {
   int n_pieces;
   uint32_t n_blocks;
   int stage;  // which stage of the map this launch belongs to
-  int multi;  // transpose kernel: some piece joins several sources (joined-source kernel)
 };
 
 struct amap_plan_t {
@@ -458,8 +457,7 @@ static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_byte
 }
 
 // the kernel's address arithmetic for one block, replayed on the host
-static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes,
-                                  const std::vector<int64_t> *slot_bytes = nullptr) {
+static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
   uint32_t t = blk;
@@ -472,8 +470,6 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
   const uint32_t a0 = (t - q * d.tiles_a) * ta;
   t = q;
   int64_t sbase = d.soff, dbase = d.doff;
-  int64_t segoff[kMaxSegments];
-  for (int sg = 0; sg < kMaxSegments; ++sg) segoff[sg] = d.seg_soff[sg];
   for (int k = d.n_loops - 1; k >= 0; --k) {
     q = host_fast_div(t, d.fd[k]);
     if (q != t / d.ext[k]) return false;
@@ -481,10 +477,8 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
     t = q;
     sbase += (int64_t)i * d.sstride[k];
     dbase += (int64_t)i * d.dstride[k];
-    for (int sg = 0; sg < d.n_seg && k < kSegBatchLoops; ++sg) segoff[sg] += (int64_t)i * d.seg_ss[sg][k];
   }
   if (t != 0) return false;
-  if (d.n_seg > 0 && (!slot_bytes || d.n_loops > kSegBatchLoops || d.seg_a[0] != 0)) return false;
   const int ub = d.tr_unit, epn = ub / es, rb = kTileB * es, cbu = rb / ub, nca = ta / epn;
   auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ ((row / epu) & 7)) << 4) | (col & 15)); };
   for (int idx = 0; idx < kTileBytes / ub; ++idx) {
@@ -495,15 +489,8 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
         const uint32_t a_hi = host_fast_div(a, d.fd_a_in);
         if (a_hi != a / d.fd_a_in.d) return false;
         const uint32_t a_lo = a - a_hi * d.fd_a_in.d;
-        int64_t s = sbase + (int64_t)a_lo * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
-        int64_t limit = in_bytes;
-        if (d.n_seg > 0) {  // joined sources: the row's operand
-          const int sg = (int)(a >= d.seg_a[1]) + (int)(a >= d.seg_a[2]) + (int)(a >= d.seg_a[3]);
-          if (sg >= d.n_seg) return false;
-          s = segoff[sg] + (int64_t)(a - d.seg_a[sg]) * d.sa[0] + (int64_t)b * es;
-          limit = (*slot_bytes)[d.seg_input[sg]];
-        }
-        if (s % ub || s < 0 || s + ub > limit) return false;
+        const int64_t s = sbase + (int64_t)a_lo * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
+        if (s % ub || s < 0 || s + ub > in_bytes) return false;
         const int sm = tile_off(a_l, cu * ub);
         if (sm < 0 || sm + ub > kTileBytes || sm % ub) return false;
       }
@@ -525,18 +512,17 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
   return true;
 }
 
-static bool check_transpose_piece(const DevPiece &d, int64_t in_bytes, int64_t out_bytes,
-                                  const std::vector<int64_t> *slot_bytes = nullptr) {
+static bool check_transpose_piece(const DevPiece &d, int64_t in_bytes, int64_t out_bytes) {
   if (d.n_blocks <= 256) {
     for (uint32_t b = 0; b < d.n_blocks; ++b)
-      if (!check_transpose_block(d, b, in_bytes, out_bytes, slot_bytes)) return false;
+      if (!check_transpose_block(d, b, in_bytes, out_bytes)) return false;
     return true;
   }
   uint64_t x = 0x9E3779B97F4A7C15ull;
   for (int t = 0; t < 256; ++t) {
     x ^= x << 13; x ^= x >> 7; x ^= x << 17;  // xorshift64
     const uint32_t b = (t == 0) ? 0 : (t == 1) ? d.n_blocks - 1 : (uint32_t)(x % d.n_blocks);
-    if (!check_transpose_block(d, b, in_bytes, out_bytes, slot_bytes)) return false;
+    if (!check_transpose_block(d, b, in_bytes, out_bytes)) return false;
   }
   return true;
 }
@@ -570,64 +556,6 @@ static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
   return true;
 }
 
-// A concat along the destination-contiguous index followed by a transpose leaves pieces that differ only in
-// their source (and in where their rows start in the destination).  Joining them into one piece lets tiles span the
-// joins: no tile is half empty because an operand has 32 or 96 channels.  Returns true when anything was joined;
-// then every piece of `v` is in joined form (n_seg >= 1) and the launch must use the joined-source kernel.
-static bool as_segment_form(DevPiece *d) {
-  if (d->n_seg > 0) return true;
-  if (d->tr_unit != 16 || d->n_loops > kSegBatchLoops || d->sa[1] != 0 || d->fd_a_in.d != d->ext_a) return false;
-  d->n_seg = 1;
-  for (int sg = 0; sg < kMaxSegments; ++sg) d->seg_a[sg] = 0xFFFFFFFFu;
-  d->seg_a[0] = 0;
-  d->seg_input[0] = d->input;
-  d->seg_soff[0] = d->soff;
-  for (int k = 0; k < d->n_loops; ++k) d->seg_ss[0][k] = d->sstride[k];
-  return true;
-}
-
-static bool join_transposes(std::vector<DevPiece> *v, int es) {
-  if (v->size() < 2) return false;
-  std::vector<DevPiece> w = *v;
-  for (DevPiece &d : w)
-    if (!as_segment_form(&d)) return false;
-  std::sort(w.begin(), w.end(), [](const DevPiece &a, const DevPiece &b) { return a.doff < b.doff; });
-  std::vector<DevPiece> out;
-  bool joined = false;
-  for (const DevPiece &b : w) {
-    bool done = false;
-    if (!out.empty()) {
-      DevPiece &a = out.back();
-      bool same = a.n_seg + b.n_seg <= kMaxSegments && a.n_loops == b.n_loops && a.ext_b == b.ext_b &&
-                  a.fd_b_in.d == b.fd_b_in.d && a.db[0] == b.db[0] && a.db[1] == b.db[1] && a.sa[0] == b.sa[0] &&
-                  b.doff == a.doff + (int64_t)a.ext_a * es;
-      for (int k = 0; k < a.n_loops && same; ++k) same = a.ext[k] == b.ext[k] && a.dstride[k] == b.dstride[k];
-      if (same) {
-        for (int sg = 0; sg < b.n_seg; ++sg) {
-          const int t = a.n_seg + sg;
-          a.seg_a[t] = a.ext_a + b.seg_a[sg];
-          a.seg_input[t] = b.seg_input[sg];
-          a.seg_soff[t] = b.seg_soff[sg];
-          for (int k = 0; k < kSegBatchLoops; ++k) a.seg_ss[t][k] = b.seg_ss[sg][k];
-        }
-        a.n_seg += b.n_seg;
-        a.ext_a += b.ext_a;
-        a.fd_a_in = make_fastdiv(a.ext_a);
-        const uint32_t ta = 8 * (16 / es);
-        const uint64_t batch = a.n_blocks / ((uint64_t)a.tiles_a * a.tiles_b);
-        a.tiles_a = (a.ext_a + ta - 1) / ta;
-        a.fd_tiles_a = make_fastdiv(a.tiles_a);
-        a.n_blocks = (uint32_t)(batch * a.tiles_a * a.tiles_b);
-        a.n_items = a.n_blocks;
-        joined = done = true;
-      }
-    }
-    if (!done) out.push_back(b);
-  }
-  if (joined) v->swap(out);
-  return joined;
-}
-
 // One launch of the transpose kernel per (access width, offset width) present.  Fill pieces with 16-byte units
 // and no constraints ride in the 16-byte launch (first: they only store and wait for nothing), so that padding
 // borders do not cost a launch of their own.
@@ -637,7 +565,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
   const int64_t out_bytes = st.numel * c.es;
   for (int access : {16, 8, 4, 2, 0})
     for (int wide = 0; wide < 2; ++wide) {
-      Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage, 0};
+      Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
       std::vector<DevPiece> transposes, fills;
       std::vector<size_t> taken;
       for (size_t q = q_lo; q < q_hi; ++q) {
@@ -651,13 +579,6 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
         taken.push_back(q);
       }
       if (transposes.empty()) continue;
-      if (access == 16 && !(c.o.flags & AMAP_PLAN_NO_JOIN) && join_transposes(&transposes, c.es)) {
-        std::vector<int64_t> slot_bytes;
-        for (int64_t n : c.slot_numel) slot_bytes.push_back(n * c.es);
-        for (const DevPiece &d : transposes)
-          if (!check_transpose_piece(d, 0, out_bytes, &slot_bytes)) return plan_fail(AMAP_EOVERFLOW, q_lo);
-        L.multi = 1;
-      }
       for (size_t q = q_lo; q < q_hi && access == 16; ++q) {
         const Piece &p = c.m.pieces[q];
         if (c.placed[q] || p.src != AMAP_CONST || c.unit_of[q] != 16 || !p.guards.empty() || !p.domain.empty()) continue;
@@ -687,7 +608,7 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
     for (int cons : {0, 2, kDevMaxCons})
       for (int wide = 0; wide < 2; ++wide)
         for (int kind : {(int)kDevStrip, (int)kDevAffine}) {
-          Launch L{kind, V, cons, wide, (int)c.pl->table.size(), 0, 0, stage, 0};
+          Launch L{kind, V, cons, wide, (int)c.pl->table.size(), 0, 0, stage};
           for (size_t q = q_lo; q < q_hi; ++q) {
             if (c.placed[q] || c.unit_of[q] != V) continue;
             const Piece &p = c.m.pieces[q];
@@ -720,7 +641,7 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
   if (opts) o = *opts;
   for (int r : o.reserved)
     if (r != 0) return AMAP_EINVAL;
-  if (o.flags & ~(AMAP_PLAN_NO_PDL | AMAP_PLAN_NO_PREFETCH | AMAP_PLAN_NO_JOIN)) return AMAP_EINVAL;
+  if (o.flags & ~(AMAP_PLAN_NO_PDL | AMAP_PLAN_NO_PREFETCH)) return AMAP_EINVAL;
   if (o.force_kernel < AMAP_KERNEL_AUTO || o.force_kernel > AMAP_KERNEL_FILL) return AMAP_EINVAL;
   const Map &m = map->m;
   const int es = m.elem_size;
@@ -794,10 +715,6 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     pl->stats.kernel_kind[slot]++;
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
-  if (getenv("AMAP_LOG"))
-    for (const Launch &L : pl->launches)
-      fprintf(stderr, "[amap] launch: stage %d kind %d unit %d pieces %d blocks %u%s\n", L.stage, L.kind, L.unit, L.n_pieces,
-              L.n_blocks, L.multi ? " (joined sources)" : "");
   pl->stats.n_stages = (int32_t)m.stages.size();
   {
     // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM)
@@ -951,11 +868,6 @@ static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTab
     case 2: launch_transpose_narrow<ES, 2>(ds, L, pt, s, pdl); return;
     case 1: launch_transpose_narrow<ES, 1>(ds, L, pt, s, pdl); return;
     default: break;
-  }
-  if (L.multi) {
-    if (L.wide) AMAP_LAUNCH(amap_transpose_joined_one, amap_transpose_joined_param, amap_transpose_joined_table, kTransposeThreads, ES, int64_t);
-    else AMAP_LAUNCH(amap_transpose_joined_one, amap_transpose_joined_param, amap_transpose_joined_table, kTransposeThreads, ES, uint32_t);
-    return;
   }
   if (L.wide) AMAP_LAUNCH(amap_transpose_one, amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, int64_t);
   else AMAP_LAUNCH(amap_transpose_one, amap_transpose_param, amap_transpose_table, kTransposeThreads, ES, uint32_t);
