@@ -74,7 +74,7 @@ struct DevPiece {
   int64_t ku_ss, ku_ds;
   int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
-  int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less; 0: shifted rows
+  int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less; 0: shifted rows, -1: realigned source rows
   int32_t pad1_;
   int64_t src_bytes;          // size of the source tensor (shifted-row kernel: guards the last aligned chunk)
   uint32_t ext_a, ext_b;      // merged extents, in elements

@@ -702,6 +702,155 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
 }
 
 // ---------------------------------------------------------------------------
+// The tiled transpose for pieces whose SOURCE rows are not 16-byte aligned but
+// whose destination rows are (NCHW -> NHWC with an odd H*W: 7x7, 35x35, 55x55
+// maps).  Phase 1 still loads aligned 16-byte chunks: the 16 lanes that share a
+// row load the chunks that cover its bytes, then every lane builds the
+// UN-shifted chunk (row bytes [16k + s, 16k + 16 + s), s = row address mod 16)
+// from its own four words and its neighbour's (one shuffle per word, a
+// two-stage word select and a funnel shift) and stores it where the aligned
+// kernel would have.  Phase 2 is the aligned kernel's.  Tile: 128 bytes of a by
+// 14 chunks of b, so that a shifted row needs at most 15 aligned chunks.
+// ---------------------------------------------------------------------------
+template <int ES>
+__device__ __forceinline__ void transpose_realign_body(const DevPiece &sp, const PtrTable &ptrs) {
+  constexpr int EPU = 16 / ES;
+  constexpr int TA = 8 * EPU;      // rows
+  constexpr int TBR = 14 * EPU;    // elements of b per tile
+  constexpr int PITCH = 256;       // bytes per shared-memory row (16 chunks)
+  constexpr int PASSES = TA / 16;  // 16 rows per pass: 16 lanes per row
+  __shared__ __align__(128) unsigned char tile[TA * PITCH];
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_b);
+  const uint32_t b0 = (t - q * sp.tiles_b) * TBR;
+  t = q;
+  q = fast_div(t, sp.fd_tiles_a);
+  const uint32_t a0 = (t - q * sp.tiles_a) * TA;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const char *src = ptrs.src[sp.input];
+  char *dst = ptrs.dst + dbase;
+  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
+  const int nb = (int)min((uint32_t)TBR, ext_b - b0);
+  const int k = threadIdx.x & 15;  // chunk of the row this lane loads and, un-shifted, stores
+  pdl_wait();
+
+  uint4 v[PASSES];
+  int shift[PASSES];
+#pragma unroll
+  for (int u = 0; u < PASSES; ++u) {
+    const int a_l = (threadIdx.x >> 4) + 16 * u;
+    const uint32_t a = a0 + a_l;
+    v[u] = make_uint4(0, 0, 0, 0);
+    shift[u] = 0;
+    if (a < ext_a) {
+      const uint32_t a_hi = fast_div(a, fa);
+      const int64_t g = sbase + (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)b0 * ES;
+      shift[u] = (int)(g & 15);
+      const int64_t addr = (g & ~(int64_t)15) + 16 * k;
+      if (addr < g + (int64_t)nb * ES) {  // the chunk overlaps the row's bytes
+        if (addr + 16 <= sp.src_bytes) {
+          v[u] = load_16(src + addr);
+        } else {  // the tensor ends inside this chunk
+          union {
+            uint4 w;
+            typename Unit<ES>::T e[EPU];
+          } pk;
+          pk.w = make_uint4(0, 0, 0, 0);
+#pragma unroll
+          for (int e = 0; e < EPU; ++e)
+            if (addr + (e + 1) * ES <= sp.src_bytes) pk.e[e] = load_unit<ES>(src + addr + e * ES);
+          v[u] = pk.w;
+        }
+      }
+    }
+  }
+  issue_barrier();
+#pragma unroll
+  for (int u = 0; u < PASSES; ++u) {
+    const int a_l = (threadIdx.x >> 4) + 16 * u;
+    // the neighbour's chunk (lane k + 1 of the same 16-lane row group); every lane takes part
+    uint32_t w[8] = {v[u].x, v[u].y, v[u].z, v[u].w, 0, 0, 0, 0};
+    w[4] = __shfl_down_sync(0xFFFFFFFFu, v[u].x, 1, 16);
+    w[5] = __shfl_down_sync(0xFFFFFFFFu, v[u].y, 1, 16);
+    w[6] = __shfl_down_sync(0xFFFFFFFFu, v[u].z, 1, 16);
+    w[7] = __shfl_down_sync(0xFFFFFFFFu, v[u].w, 1, 16);
+    const int o = shift[u] >> 2, bits = (shift[u] & 3) * 8;
+    uint32_t x[6], y[5];
+#pragma unroll
+    for (int i = 0; i < 6; ++i) x[i] = (o & 2) ? w[i + 2] : w[i];
+#pragma unroll
+    for (int i = 0; i < 5; ++i) y[i] = (o & 1) ? x[i + 1] : x[i];
+    uint4 out;
+    out.x = __funnelshift_r(y[0], y[1], bits);
+    out.y = __funnelshift_r(y[1], y[2], bits);
+    out.z = __funnelshift_r(y[2], y[3], bits);
+    out.w = __funnelshift_r(y[3], y[4], bits);
+    if (a0 + a_l < ext_a && k * EPU < nb)
+      *reinterpret_cast<uint4 *>(tile + a_l * PITCH + ((k ^ ((a_l / EPU) & 7)) << 4)) = out;
+  }
+  __syncthreads();
+
+  const bool split_b = fb.d < ext_b;
+  auto dst_of = [&](uint32_t a, uint32_t b) -> char * {
+    int64_t off = (int64_t)a * ES;
+    if (split_b) {
+      const uint32_t b_hi = fast_div(b, fb);
+      off += (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1];
+    } else {
+      off += (int64_t)b * sp.db[0];
+    }
+    return dst + off;
+  };
+  if constexpr (ES == 2) {
+#pragma unroll 2
+    for (int idx = threadIdx.x; idx < (TBR / 2) * 8; idx += kTransposeThreads) {
+      const int ca = idx & 7, b_l = (idx >> 3) * 2;
+      const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
+      if (a < ext_a && b_l < nb) {
+        const unsigned char *p = tile + (ca * EPU) * PITCH + (((b_l / EPU) ^ ca) << 4) + (b_l % EPU) * ES;
+        uint32_t r[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * PITCH);
+        uint4 lo, hi;
+        lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
+        lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
+        lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
+        lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
+        __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), lo);
+        if (b_l + 1 < nb) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b + 1)), hi);  // an odd extent ends on a lone b
+      }
+    }
+  } else {
+#pragma unroll 2
+    for (int idx = threadIdx.x; idx < TBR * 8; idx += kTransposeThreads) {
+      const int ca = idx & 7, b_l = idx >> 3;
+      const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
+      if (a < ext_a && b_l < nb) {
+        union {
+          uint4 w;
+          typename Unit<ES>::T e[EPU];
+        } pk;
+        const int col = b_l * ES;
+#pragma unroll
+        for (int j = 0; j < EPU; ++j)
+          pk.e[j] = *reinterpret_cast<const typename Unit<ES>::T *>(tile + (ca * EPU + j) * PITCH + (((col >> 4) ^ ca) << 4) + (col & 15));
+        __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), pk.w);
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------
 // Entry kernels.  Each family has two: the *_param kernels get up to
 // kParamPieces descriptors BY VALUE in the kernel parameters (constant bank: a
 // block starts its index arithmetic without a round trip to global memory),
@@ -832,6 +981,28 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_shifted_one(
                                                                                  PtrTable ptrs) {
   pdl_launch_dependents();
   transpose_shifted_body<ES>(p, ptrs);
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_realign_param(const __grid_constant__ LaunchDesc ld,
+                                                                                   PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_realign_body<ES>(param_piece(ld), ptrs);
+}
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_realign_table(const DevPiece *__restrict__ table,
+                                                                                   int first_piece, int n_pieces,
+                                                                                   PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_realign_body<ES>(sp, ptrs);
+}
+template <int ES>
+__global__ void __launch_bounds__(kTransposeThreads) amap_transpose_realign_one(const __grid_constant__ DevPiece p,
+                                                                                 PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_realign_body<ES>(p, ptrs);
 }
 
 }  // namespace amap

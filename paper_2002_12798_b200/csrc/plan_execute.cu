@@ -388,6 +388,28 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     if (ia_hi >= 0 && try_build(-1, ib_hi, ub)) return true;
     if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1, ub)) return true;
   }
+  // source rows misaligned, destination rows aligned: the realigning kernel (tr_unit = -1; tile 8 x 14 chunks)
+  if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_a % (16 / es) == 0 && d->doff % 16 == 0 &&
+      d->db[0] % 16 == 0 && d->db[1] % 16 == 0) {
+    bool dst_aligned = true;
+    for (int j = 0; j < d->n_loops; ++j) dst_aligned = dst_aligned && d->dstride[j] % 16 == 0;
+    if (dst_aligned) {
+      const int epu16 = 16 / es;
+      d->tr_unit = -1;
+      d->src_bytes = in_bytes;
+      d->tiles_a = (d->ext_a + 8 * epu16 - 1) / (8 * epu16);
+      d->tiles_b = (d->ext_b + 14 * epu16 - 1) / (14 * epu16);
+      d->fd_tiles_a = make_fastdiv(d->tiles_a);
+      d->fd_tiles_b = make_fastdiv(d->tiles_b);
+      unsigned __int128 blocks = (unsigned __int128)d->tiles_a * d->tiles_b;
+      for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
+      if (blocks <= 0x7FFFFFFFull) {
+        d->n_blocks = (uint32_t)blocks;
+        d->n_items = (uint64_t)blocks;
+        return true;
+      }
+    }
+  }
   // rows that are not aligned at all: the shifted-row kernel (aligned 16-byte accesses, elements un-shifted in
   // shared memory); its tile is 7 x 14 chunks
   // Measured: it doubles the strip kernel's rate when only the DESTINATION rows are misaligned (e.g. NHWC -> NCHW
@@ -456,9 +478,45 @@ static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_byte
   return true;
 }
 
+// the realigning kernel's address arithmetic for one block, replayed on the host
+static bool check_realign_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
+  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu, tbr = 14 * epu;
+  if (d.src_bytes != in_bytes || d.ext_a % epu) return false;
+  uint32_t t = blk;
+  uint32_t q = t / d.tiles_b;
+  const uint32_t b0 = (t - q * d.tiles_b) * tbr;
+  t = q;
+  q = t / d.tiles_a;
+  const uint32_t a0 = (t - q * d.tiles_a) * ta;
+  t = q;
+  int64_t sbase = d.soff, dbase = d.doff;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    q = t / d.ext[k];
+    sbase += (int64_t)(t - q * d.ext[k]) * d.sstride[k];
+    dbase += (int64_t)(t - q * d.ext[k]) * d.dstride[k];
+    t = q;
+  }
+  if (t != 0 || a0 >= d.ext_a || b0 >= d.ext_b) return false;
+  const int nb = (int)std::min<uint32_t>(tbr, d.ext_b - b0);
+  for (uint32_t a = a0; a < std::min<uint32_t>(a0 + ta, d.ext_a); ++a) {
+    const uint32_t a_hi = a / d.fd_a_in.d;
+    const int64_t g = sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b0 * es;
+    if (g < 0 || g % es || g + (int64_t)nb * es > in_bytes) return false;
+    // the row's bytes must be covered by at most 15 aligned chunks, so that lane 14 holds the last one needed
+    if ((((g + (int64_t)nb * es + 15) & ~(int64_t)15) - (g & ~(int64_t)15)) / 16 > 15) return false;
+    for (int b_l = 0; b_l < nb; ++b_l) {
+      const uint32_t b = b0 + b_l, b_hi = b / d.fd_b_in.d;
+      const int64_t o = dbase + (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a * es;
+      if (o < 0 || o + es > out_bytes || ((a - a0) % epu == 0 && o % 16)) return false;
+    }
+  }
+  return true;
+}
+
 // the kernel's address arithmetic for one block, replayed on the host
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
+  if (d.tr_unit < 0) return check_realign_block(d, blk, in_bytes, out_bytes);
   const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
   uint32_t t = blk;
   uint32_t q = host_fast_div(t, d.fd_tiles_b);
@@ -563,7 +621,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
   const int64_t out_bytes = st.numel * c.es;
-  for (int access : {16, 8, 4, 2, 0})
+  for (int access : {16, 8, 4, 2, 0, -1})
     for (int wide = 0; wide < 2; ++wide) {
       Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
       std::vector<DevPiece> transposes, fills;
@@ -572,7 +630,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
         if (!c.is_tr[q] || c.tr[q].tr_unit != access) continue;
         const DevPiece &d = c.tr[q];
         const int64_t in_bytes = c.slot_numel[d.input] * c.es;
-        const bool needs_wide = (in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && access != 0;
+        const bool needs_wide = (in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && access > 0;
         if ((int)needs_wide != wide) continue;
         if (!check_transpose_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
         transposes.push_back(d);
@@ -860,6 +918,10 @@ static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
+    case -1:
+      if constexpr (ES <= 4)
+        AMAP_LAUNCH(amap_transpose_realign_one, amap_transpose_realign_param, amap_transpose_realign_table, kTransposeThreads, ES);
+      return;
     case 0:
       if constexpr (ES <= 4) AMAP_LAUNCH(amap_transpose_shifted_one, amap_transpose_shifted_param, amap_transpose_shifted_table, kTransposeThreads, ES);
       return;

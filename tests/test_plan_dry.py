@@ -34,7 +34,8 @@ def test_forced_families():
         ((4, 256, 56, 56), "transpose"),  # 16-byte rows on both sides
         ((4, 256, 14, 14), "transpose"),  # 8-byte aligned rows: narrow units
         ((4, 254, 54, 54), "transpose"),  # 4-byte aligned
-        ((4, 256, 27, 27), "gather"),     # odd source rows, aligned destination rows: strip kernel
+        ((4, 256, 27, 27), "transpose"),  # odd source rows, aligned destination rows: realigning kernel
+        ((4, 255, 27, 27), "gather"),     # both sides misaligned: strip kernel
     ],
 )
 def test_transpose_family_by_alignment(shape, expect):
