@@ -576,35 +576,35 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
 }
 
 // ---------------------------------------------------------------------------
-// The tiled transpose for pieces whose rows are NOT 16-byte aligned (odd
-// extents: 7x7, 13x13, 55x55 feature maps ...).  Global memory is still only
-// touched with aligned 16-byte accesses (plus a few element accesses on edges):
-//   phase 1  for each tile row a, the aligned 16-byte chunks that cover its
-//            source bytes are loaded and stored as chunks of the row; the row's
-//            elements therefore sit shifted by (row address mod 16) bytes;
-//   phase 2  a thread owns one aligned 16-byte slot of a destination row; it
-//            finds each of the slot's elements in its source row, un-shifting
-//            the column, and stores the slot whole when all its elements belong
-//            to the tile, element by element otherwise.
-// Tile: 7 chunks of a by 14 chunks of b, so that a shifted row still fits the
-// 16-chunk shared-memory row and a shifted destination run fits 8 slots.
+// The tiled transpose for pieces whose DESTINATION rows are not 16-byte aligned
+// but whose source rows are (NHWC -> NCHW with an odd H*W).  Phase 1 is the
+// aligned kernel's.  In phase 2 the eight lanes that share a destination row b
+// each gather their 16 bytes of the tile's run (a0 + 8ca ...), then build the
+// ALIGNED 16-byte slot of the destination that starts inside their predecessor's
+// bytes: the last s bytes of lane ca-1's vector and the first 16-s of their own
+// (s = destination address mod 16; one shuffle per word, a word select and a
+// funnel shift).  Slots that are not wholly inside the tile's run -- the first
+// and, through lane 7, a ninth one, and whatever crosses the end of the row --
+// are stored element by element; the neighbouring tile writes their other part.
 // ---------------------------------------------------------------------------
 template <int ES>
 __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const PtrTable &ptrs) {
   constexpr int EPU = 16 / ES;
-  constexpr int TAS = 7 * EPU, TBS = 14 * EPU;  // tile extents in elements
-  constexpr int U = (TAS * 16 + kTransposeThreads - 1) / kTransposeThreads;
+  constexpr int TA = 8 * EPU;
+  constexpr int RB = kTileB * ES;
+  constexpr int CB = RB / 16;
+  constexpr int U = TA * CB / kTransposeThreads;
   using E = typename Unit<ES>::T;
-  __shared__ __align__(128) unsigned char tile[TAS * 256];
+  __shared__ __align__(128) unsigned char tile[kTileBytes];
 
   uint32_t t = blockIdx.x - sp.first_block;
   uint32_t q = fast_div(t, sp.fd_tiles_b);
-  const uint32_t b0 = (t - q * sp.tiles_b) * TBS;
+  const uint32_t b0 = (t - q * sp.tiles_b) * kTileB;
   t = q;
   q = fast_div(t, sp.fd_tiles_a);
-  const uint32_t a0 = (t - q * sp.tiles_a) * TAS;
+  const uint32_t a0 = (t - q * sp.tiles_a) * TA;
   t = q;
-  int64_t sbase = sp.soff, dbase = sp.doff;  // byte offsets inside the source / destination tensors
+  int64_t sbase = sp.soff, dbase = sp.doff;
   for (int k = sp.n_loops - 1; k >= 0; --k) {
     q = fast_div(t, sp.fd[k]);
     const uint32_t i = t - q * sp.ext[k];
@@ -612,91 +612,109 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
     sbase += (int64_t)i * sp.sstride[k];
     dbase += (int64_t)i * sp.dstride[k];
   }
-  const char *src = ptrs.src[sp.input];
-  char *dst = ptrs.dst;
+  const char *src = ptrs.src[sp.input] + sbase;
+  char *dst = ptrs.dst;  // dbase stays a byte offset: the slots are aligned relative to the tensor's start
+  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
-  const int64_t sa0 = sp.sa[0], sa1 = sp.sa[1], db0 = sp.db[0], db1 = sp.db[1];
-  const int na = (int)min((uint32_t)TAS, sp.ext_a - a0), nb = (int)min((uint32_t)TBS, sp.ext_b - b0);
-  auto row_offset = [&](uint32_t a) -> int64_t {  // source byte offset of element (a, b0)
-    const uint32_t a_hi = fast_div(a, fa);
-    return sbase + (int64_t)(a - a_hi * fa.d) * sa0 + (int64_t)a_hi * sa1 + (int64_t)b0 * ES;
-  };
+  const int na = (int)min((uint32_t)TA, ext_a - a0);  // rows of the tile that exist
   pdl_wait();
 
+  // phase 1: as in the aligned kernel (rows past the end of a stay unwritten and are never stored)
   uint4 v[U];
-  bool have[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     const int idx = threadIdx.x + u * kTransposeThreads;
-    const int a_l = idx >> 4, k = idx & 15;
-    have[u] = false;
-    if (a_l < na) {
-      const int64_t g = row_offset(a0 + a_l);
-      const int64_t first = g & ~(int64_t)15;
-      const int nch = (int)((((g + (int64_t)nb * ES + 15) & ~(int64_t)15) - first) >> 4);
-      const int64_t addr = first + 16 * k;
-      if (k < nch) {
-        have[u] = true;
-        if (addr + 16 <= sp.src_bytes) {
-          v[u] = load_16(src + addr);
-        } else {  // the last chunk of the tensor: only the elements that exist
-          union {
-            uint4 w;
-            E e[EPU];
-          } pk;
-          pk.w = make_uint4(0, 0, 0, 0);
-#pragma unroll
-          for (int e = 0; e < EPU; ++e)
-            if (addr + (e + 1) * ES <= sp.src_bytes) pk.e[e] = load_unit<ES>(src + addr + e * ES);
-          v[u] = pk.w;
-        }
-      }
+    const int a_l = idx / CB, cb = idx % CB;
+    const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
+    v[u] = make_uint4(0, 0, 0, 0);
+    if (a < ext_a && b < ext_b) {
+      const uint32_t a_hi = fast_div(a, fa);
+      v[u] = load_16(src + (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)b * ES);
     }
   }
   issue_barrier();
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     const int idx = threadIdx.x + u * kTransposeThreads;
-    const int a_l = idx >> 4, k = idx & 15;
-    if (have[u]) *reinterpret_cast<uint4 *>(tile + a_l * 256 + ((k ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+    const int a_l = idx / CB, cb = idx % CB;
+    *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ ((a_l / EPU) & 7)) << 4)) = v[u];
   }
   __syncthreads();
 
-  const bool split = fa.d < sp.ext_a;
-  const int row0_shift = (int)(row_offset(a0) & 15);  // valid when a does not merge two loops
-  const int row_step = (int)(sa0 & 15);
-#pragma unroll 1
-  for (int idx = threadIdx.x; idx < TBS * 8; idx += kTransposeThreads) {
-    const int slot = idx & 7, b_l = idx >> 3;
-    if (b_l >= nb) continue;
-    const uint32_t b = b0 + b_l;
+  // one destination row: lane ca of the row's eight lanes holds run bytes [16 ca, 16 ca + 16) in `own`
+  auto emit_row = [&](uint4 own, int ca, uint32_t b, bool row_ok) {
     const uint32_t b_hi = fast_div(b, fb);
-    const int64_t D = dbase + (int64_t)(b - b_hi * fb.d) * db0 + (int64_t)b_hi * db1 + (int64_t)a0 * ES;
-    const int64_t A = (D & ~(int64_t)15) + 16 * slot;
-    const int rel0 = (int)((A - D) / ES);  // tile row of the slot's first element (may be negative)
-    if (rel0 >= na || rel0 + EPU <= 0) continue;
-    union {
-      uint4 w;
-      E e[EPU];
-    } pk;
-    bool all = true;
+    const int64_t D = dbase + (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1] + (int64_t)a0 * ES;
+    const int sh = (int)(D & 15);
+    uint32_t w[9];
+    w[0] = __shfl_up_sync(0xFFFFFFFFu, own.x, 1, 8);
+    w[1] = __shfl_up_sync(0xFFFFFFFFu, own.y, 1, 8);
+    w[2] = __shfl_up_sync(0xFFFFFFFFu, own.z, 1, 8);
+    w[3] = __shfl_up_sync(0xFFFFFFFFu, own.w, 1, 8);
+    w[4] = own.x, w[5] = own.y, w[6] = own.z, w[7] = own.w, w[8] = 0;
+    // slot `s` = run bytes [16 s - sh, 16 s - sh + 16); lane 7 also owns slot 8 (its own tail)
 #pragma unroll
-    for (int e = 0; e < EPU; ++e) {
-      const int row = rel0 + e;
-      const bool ok = row >= 0 && row < na;
-      all = all && ok;
-      if (ok) {
-        const int shift = split ? (int)(row_offset(a0 + row) & 15) : ((row0_shift + row * row_step) & 15);
-        const int col = b_l * ES + shift;  // byte column inside the shifted row
-        pk.e[e] = *reinterpret_cast<const E *>(tile + row * 256 + ((((col >> 4) ^ ((row / EPU) & 7)) << 4) | (col & 15)));
+    for (int pass = 0; pass < 2; ++pass) {
+      const int s = ca + pass;
+      if (pass == 1) {
+        if (ca != 7 || sh == 0) break;
+        w[0] = own.x, w[1] = own.y, w[2] = own.z, w[3] = own.w, w[4] = w[5] = w[6] = w[7] = 0;
+      }
+      const int first = 16 - sh;  // where the slot starts inside the 32-byte window
+      const int o = first >> 2, bits = (first & 3) * 8;
+      // z[i] = w[i + o], o in 0..4, by a three-stage word select (w[8] = 0 pads the window)
+      uint32_t x[8], y[6], z[5];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = (o & 4) ? (i + 4 <= 8 ? w[i + 4 <= 8 ? i + 4 : 8] : 0u) : w[i];
+#pragma unroll
+      for (int i = 0; i < 6; ++i) y[i] = (o & 2) ? x[i + 2] : x[i];
+#pragma unroll
+      for (int i = 0; i < 5; ++i) z[i] = (o & 1) ? y[i + 1] : y[i];
+      union {
+        uint4 vec;
+        E e[EPU];
+      } out;
+      out.vec.x = __funnelshift_r(z[0], z[1], bits);
+      out.vec.y = __funnelshift_r(z[1], z[2], bits);
+      out.vec.z = __funnelshift_r(z[2], z[3], bits);
+      out.vec.w = __funnelshift_r(z[3], z[4], bits);
+      if (!row_ok) continue;
+      const int rel0 = (16 * s - sh) / ES;  // tile row of the slot's first element (negative for slot 0 when sh > 0)
+      const int64_t A = D - sh + 16 * s;
+      if (rel0 >= 0 && rel0 + EPU <= na) {
+        __stcs(reinterpret_cast<uint4 *>(dst + A), out.vec);
+      } else {
+#pragma unroll
+        for (int e = 0; e < EPU; ++e)
+          if (rel0 + e >= 0 && rel0 + e < na) store_unit<ES>(dst + A + e * ES, out.e[e]);
       }
     }
-    if (all) {
-      __stcs(reinterpret_cast<uint4 *>(dst + A), pk.w);
-    } else {
+  };
+
+  if constexpr (ES == 2) {
 #pragma unroll
-      for (int e = 0; e < EPU; ++e)
-        if (rel0 + e >= 0 && rel0 + e < na) store_unit<ES>(dst + A + e * ES, pk.e[e]);
+    for (int u = 0; u < U / 2; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int ca = idx & 7, b_l = (idx >> 3) * 2;
+      const uint32_t b = b0 + b_l;
+      const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ ca) << 4) + (b_l % EPU) * ES;
+      uint32_t r[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * RB);
+      uint4 lo, hi;
+      lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
+      lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
+      lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
+      lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
+      emit_row(lo, ca, b, b < ext_b);
+      emit_row(hi, ca, b + 1, b + 1 < ext_b);
+    }
+  } else {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int idx = threadIdx.x + u * kTransposeThreads;
+      const int ca = idx & 7, b_l = idx >> 3;
+      emit_row(gather_column<ES>(tile, ca, b_l), ca, b0 + b_l, b0 + b_l < ext_b);
     }
   }
 }

@@ -410,39 +410,31 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       }
     }
   }
-  // rows that are not aligned at all: the shifted-row kernel (aligned 16-byte accesses, elements un-shifted in
-  // shared memory); its tile is 7 x 14 chunks
-  // Measured: it doubles the strip kernel's rate when only the DESTINATION rows are misaligned (e.g. NHWC -> NCHW
-  // with an odd H*W) and gains nothing when the source rows are, so it is chosen for the first case only.
-  if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) &&
-      (d->sa[0] % 16 == 0 && d->sa[1] % 16 == 0) && (d->db[0] % 16 != 0 || d->db[1] % 16 != 0)) {
-    const int epu16 = 16 / es;
-    d->tr_unit = 0;
-    d->src_bytes = in_bytes;
-    d->tiles_a = (d->ext_a + 7 * epu16 - 1) / (7 * epu16);
-    d->tiles_b = (d->ext_b + 14 * epu16 - 1) / (14 * epu16);
-    d->fd_tiles_a = make_fastdiv(d->tiles_a);
-    d->fd_tiles_b = make_fastdiv(d->tiles_b);
-    unsigned __int128 blocks = (unsigned __int128)d->tiles_a * d->tiles_b;
-    for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
-    if (blocks > 0x7FFFFFFFull) return false;
-    d->n_blocks = (uint32_t)blocks;
-    d->n_items = (uint64_t)blocks;
-    return true;
+  // destination rows misaligned, source rows aligned: the shifted-destination kernel (tr_unit = 0; the aligned
+  // kernel's tile, destination slots realigned in registers)
+  if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_b % (16 / es) == 0 && d->soff % 16 == 0 &&
+      d->sa[0] % 16 == 0 && d->sa[1] % 16 == 0) {
+    bool src_aligned = true;
+    for (int j = 0; j < d->n_loops; ++j) src_aligned = src_aligned && d->sstride[j] % 16 == 0;
+    if (src_aligned) {
+      d->tr_unit = 0;
+      d->src_bytes = in_bytes;
+      return true;  // tiles and blocks as try_build computed them: 8 chunks of a by kTileB of b
+    }
   }
   return false;
 }
 
-// the shifted-row kernel's address arithmetic for one block, replayed on the host
+// the shifted-destination kernel's address arithmetic for one block, replayed on the host
 static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
-  const int es = d.unit_bytes, epu = 16 / es, tas = 7 * epu, tbs = 14 * epu;
-  if (d.src_bytes != in_bytes) return false;
+  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
+  if (d.ext_b % epu) return false;
   uint32_t t = blk;
   uint32_t q = t / d.tiles_b;
-  const uint32_t b0 = (t - q * d.tiles_b) * tbs;
+  const uint32_t b0 = (t - q * d.tiles_b) * kTileB;
   t = q;
   q = t / d.tiles_a;
-  const uint32_t a0 = (t - q * d.tiles_a) * tas;
+  const uint32_t a0 = (t - q * d.tiles_a) * ta;
   t = q;
   int64_t sbase = d.soff, dbase = d.doff;
   for (int k = d.n_loops - 1; k >= 0; --k) {
@@ -452,28 +444,23 @@ static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_byte
     t = q;
   }
   if (t != 0 || a0 >= d.ext_a || b0 >= d.ext_b) return false;
-  const int na = (int)std::min<uint32_t>(tas, d.ext_a - a0), nb = (int)std::min<uint32_t>(tbs, d.ext_b - b0);
-  auto row_offset = [&](uint32_t a) {
-    const uint32_t a_hi = a / d.fd_a_in.d;
-    return sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b0 * es;
-  };
-  for (int a_l = 0; a_l < na; ++a_l) {
-    const int64_t g = row_offset(a0 + a_l);
-    if (g < 0 || g + (int64_t)nb * es > in_bytes) return false;
-    const int64_t first = g & ~(int64_t)15;
-    const int nch = (int)((((g + (int64_t)nb * es + 15) & ~(int64_t)15) - first) >> 4);
-    if (nch > 16 || first < 0) return false;
-    for (int b_l = 0; b_l < nb; ++b_l) {  // every element must be found inside the 16-chunk row
-      const int col = b_l * es + (int)(g & 15);
-      if ((col >> 4) >= nch || (col >> 4) > 15) return false;
+  const int na = (int)std::min<uint32_t>(ta, d.ext_a - a0);
+  for (int a_l = 0; a_l < na; ++a_l)  // aligned 16-byte loads along b
+    for (uint32_t b = b0; b < std::min<uint32_t>(b0 + kTileB, d.ext_b); b += epu) {
+      const uint32_t a = a0 + a_l, a_hi = a / d.fd_a_in.d;
+      const int64_t s = sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
+      if (s % 16 || s < 0 || s + 16 > in_bytes) return false;
     }
-  }
-  for (int b_l = 0; b_l < nb; ++b_l) {
-    const uint32_t b = b0 + b_l, b_hi = b / d.fd_b_in.d;
+  for (uint32_t b = b0; b < std::min<uint32_t>(b0 + kTileB, d.ext_b); ++b) {
+    const uint32_t b_hi = b / d.fd_b_in.d;
     const int64_t D = dbase + (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a0 * es;
-    if (D < 0 || D + (int64_t)na * es > out_bytes) return false;
-    // the destination run must fit the 8 aligned slots a thread group covers
-    if (((D & 15) + (int64_t)na * es + 15) / 16 > 8) return false;
+    if (D < 0 || D % es || D + (int64_t)na * es > out_bytes) return false;
+    const int sh = (int)(D & 15);
+    for (int s = 0; s <= 8; ++s) {  // every slot: whole ones are aligned and inside, partial ones store valid elements only
+      const int rel0 = (16 * s - sh) / es;
+      const int64_t A = D - sh + 16 * s;
+      if (rel0 >= 0 && rel0 + epu <= na && (A % 16 || A < 0 || A + 16 > out_bytes)) return false;
+    }
   }
   return true;
 }
