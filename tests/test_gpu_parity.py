@@ -147,6 +147,74 @@ def test_random_statement_chains(B):
     assert staged > 0
 
 
+def test_offsets_beyond_4_gib(B):
+    """A 5 GiB byte tensor: the pieces' source offsets do not fit 32 bits, so the 64-bit kernel variants run
+    (strip kernel for the slice, transpose kernel for the slice + transpose).  Only a slab near the end is
+    filled and read; the oracle sees a host array of the same shape whose untouched pages are never allocated."""
+    import torch
+
+    shape = [5, 32768, 32768]
+    lo_row, rows = 100, 64
+    slab = np.random.default_rng(5).integers(1, 255, size=(rows, shape[2]), dtype=np.uint8)
+    host = np.zeros(shape, dtype=np.uint8)  # lazily mapped
+    host[4, lo_row : lo_row + rows] = slab
+    dev = torch.zeros(shape, dtype=torch.uint8, device="cuda")
+    dev[4, lo_row : lo_row + rows] = torch.from_numpy(slab).cuda()
+    sl = {"kind": "slice", "src": 0, "start": [4, lo_row, 0], "stop": [5, lo_row + rows, shape[2]], "step": [1, 1, 1]}
+    for ops, kernel in (([sl], "copy"), ([sl, {"kind": "transpose", "src": 1, "perm": [0, 2, 1]}], "transpose")):
+        chain = W.Chain(name="big", dtype="u8", inputs=[shape], ops=ops, values="raw")
+        want = oracle.run_chain(chain, [host])
+        m = B.compose_chain(chain)
+        plan = m.plan(0)
+        assert plan.stats()["kernels"][kernel] == 1
+        out = torch.zeros(m.out_numel, dtype=torch.uint8, device="cuda")
+        plan.execute([dev], out)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy(), want.reshape(-1)), kernel
+    del dev
+
+
+def test_three_guards_in_one_piece(B):
+    """A 3-D window gather written as one raw guarded statement: three guards, so the kernels' larger
+    constraint variant runs."""
+    D, H, Wd = 6, 7, 9
+    chain = W.Chain(
+        name="stencil", dtype="fp32", inputs=[[D, H, Wd]],
+        ops=[{
+            "kind": "stmts", "shape": [D * H * Wd, 27],
+            "stmts": [{
+                "bounds": [D, H, Wd, 3, 3, 3],
+                "load": (0, [[1, 0, 0, 1, 0, 0], [0, 1, 0, 0, 1, 0], [0, 0, 1, 0, 0, 1]], [-1, -1, -1]),
+                "store": ([[H * Wd, Wd, 1, 0, 0, 0], [0, 0, 0, 9, 3, 1]], [0, 0]),
+                "guarded": True, "fill": 0,
+            }],
+        }],
+        values="raw",
+    )
+    xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
+    want = oracle.run_chain(chain, xs)
+    assert len(B.compose_chain(chain).pieces()[0]["guards"]) == 3
+    for force in (0, 1):
+        got, _ = run_gpu(B, chain, xs, force=force)
+        assert np.array_equal(got, want.reshape(-1))
+
+
+def test_sixteen_byte_elements_against_torch(B):
+    """elem_size 16 (complex128): every element is a whole 16-byte unit.  Checked against torch's own permute
+    (a library routine as third opinion; the oracle's Python front end stops at 8-byte elements)."""
+    import torch
+
+    x = torch.randn(3, 10, 7, dtype=torch.complex128, device="cuda")
+    b = B.Builder(16)
+    t = b.input([3, 10, 7])
+    m = b.compose(b.pad(b.transpose(t, [2, 0, 1]), [1, 0, 0], [0, 0, 2]))
+    out = torch.full((8, 3, 12), 7 + 7j, dtype=torch.complex128, device="cuda")
+    m.plan(0).execute([x], out)
+    torch.cuda.synchronize()
+    want = torch.nn.functional.pad(x.permute(2, 0, 1), (0, 2, 0, 0, 1, 0))
+    assert torch.equal(out.view(torch.int64), want.contiguous().view(torch.int64))
+
+
 @pytest.mark.parametrize("dtype,es", [("u8", 1), ("u64", 8)])
 def test_other_element_sizes(B, dtype, es):
     chain = W.c3_head_split(B=2, S=20, heads=3, D=16, keep=11, dtype=dtype)
