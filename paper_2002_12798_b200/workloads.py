@@ -271,6 +271,8 @@ def reduced_configs() -> dict:
         "c2_fwd_odd_gather": c2_nchw_to_nhwc(N=2, C=255, H=27, W=27),
         "c2_fwd_odd_u8": c2_nchw_to_nhwc(N=2, C=64, H=11, W=13, dtype="u8"),
         "c2_fwd_odd_f32b": c2_nchw_to_nhwc(N=2, C=36, H=7, W=9, dtype="fp32"),
+        "c2_fwd_narrow": c2_nchw_to_nhwc(N=2, C=72, H=14, W=14),
+        "c2_inv_narrow": c2_nhwc_to_nchw(N=2, C=68, H=14, W=14),
         "c3": c3_head_split(B=2, S=80, heads=3, D=128, keep=50),
         "c3_odd": c3_head_split(B=2, S=33, heads=5, D=24, keep=17),
         "c3_merge": c3_head_merge(B=2, S=70, heads=3, D=128),

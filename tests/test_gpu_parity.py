@@ -174,6 +174,22 @@ def test_offsets_beyond_4_gib(B):
     del dev
 
 
+def test_launch_with_more_pieces_than_fit_the_kernel_parameters(B):
+    """Twelve operands joined and transposed: twelve pieces in one launch, so the kernels read their descriptors
+    from the plan's table in device memory instead of the kernel parameters."""
+    n_in = 12
+    chain = W.Chain(
+        name="wide_concat", dtype="bf16", inputs=[[2, 16, 8, 8]] * n_in,
+        ops=[{"kind": "concat", "srcs": list(range(n_in)), "axis": 1}, {"kind": "transpose", "src": n_in, "perm": [0, 2, 3, 1]}],
+        values="normal",
+    )
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, plan = run_gpu(B, chain, xs)
+    assert plan.stats()["n_pieces"] == n_in and plan.stats()["n_launches"] == 1
+    assert np.array_equal(got, want.reshape(-1))
+
+
 def test_three_guards_in_one_piece(B):
     """A 3-D window gather written as one raw guarded statement: three guards, so the kernels' larger
     constraint variant runs."""

@@ -36,7 +36,9 @@ def test_static_table_matches_amap_execute_on_calls_in_a_row():
 
     cfg = W.reduced_configs()
     # different maps one after the other: each call finds the previous call's descriptors in the table
-    for name in ("c3", "c4_odd", "c5", "c1", "c3"):
+    # every kernel family reads its descriptors from the fixed table here: copy, aligned / narrow / realigning /
+    # shifted transposes with fills, window gather, element-wise gather
+    for name in ("c3", "c4", "c2_fwd_narrow", "c2_fwd", "c2_inv", "c4_odd", "c5", "c1", "c3"):
         ref, out, dry, dev, stream = _both_ways(B, torch, cfg[name])
         ptrs = [d.data_ptr() for d in dev]
         assert torch.equal(ref, out), name  # pure copies: bit-exact
