@@ -255,7 +255,10 @@ int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void 
  * the output and waits.  Uses device staging memory owned by the plan
  * (allocated on first use).  src_host_ptrs: host array of n_inputs HOST
  * pointers; dst_host_ptr: HOST.  Pinned host memory makes the copies faster
- * but is not required. */
+ * but is not required.  When the outermost loop of the whole map is a batch
+ * loop (slab k of the output needs only slab k of every input) the call works
+ * slab by slab on two more streams of its own, so that upload, kernel and
+ * download overlap; the result is the same. */
 int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------

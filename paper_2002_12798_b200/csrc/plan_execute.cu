@@ -63,6 +63,14 @@ struct amap_plan_t {
   // staging for amap_execute_host (allocated on first use)
   std::vector<void *> stage_in;
   void *stage_out = nullptr;
+  // amap_execute_host pipelines batch slabs when every piece's outermost loop is one batch loop that cuts the
+  // inputs and the output into independent slabs: a second plan for one slab, run once per slab
+  amap_plan_t *slab_plan = nullptr;
+  int n_slabs = 0;
+  std::vector<int64_t> slab_in_bytes;
+  int64_t slab_out_bytes = 0;
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  std::vector<cudaEvent_t> events;  // [0] start, then per slab: input ready, kernel done; last: output done
 };
 
 static FastDiv make_fastdiv(uint32_t d) {
@@ -679,7 +687,63 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
   return AMAP_OK;
 }
 
-extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts, amap_plan_t **out_plan) {
+// ---------------------------------------------------------------------------
+// Batch slabs for amap_execute_host.  If the outermost loop of every piece is the same batch loop, advancing it
+// moves every input and the output by one whole slab and nothing else of a piece leaves its slab, then slab k of
+// the output needs only slab k of the inputs: the host entry point can upload, run and download slab by slab and
+// overlap the three (PCIe is full duplex).  Guarded pieces are left alone (their unguarded offsets may point
+// outside the slab).
+// ---------------------------------------------------------------------------
+static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts, bool allow_slabs, amap_plan_t **out_plan);
+
+static void plan_slabs(const Map &m, int device, const amap_plan_opts &o, amap_plan_t *pl) {
+  if (m.stages.size() != 1 || m.pieces.empty() || m.out_numel == 0) return;
+  const int64_t N = m.pieces[0].n() > 0 ? m.pieces[0].ext[0] : 0;
+  if (N < 2 || m.out_numel % N) return;
+  const int64_t DS = m.out_numel / N;
+  for (int64_t n : m.in_numel)
+    if (n % N) return;
+  auto inside = [](const Aff &a, const std::vector<int64_t> &ext, int64_t slab) {
+    Aff rest = a;
+    rest.c[0] = 0;
+    int64_t lo, hi;
+    aff_range(rest, ext, &lo, &hi);
+    return lo >= 0 && hi < slab;
+  };
+  for (const Piece &p : m.pieces) {
+    if (p.n() < 1 || p.ext[0] != N || !p.guards.empty() || !p.domain.empty()) return;
+    if (p.dst.c[0] != DS || !inside(p.dst, p.ext, DS)) return;
+    if (p.src != AMAP_CONST) {
+      const int64_t SS = m.in_numel[p.src] / N;
+      if (p.srcoff.c[0] != SS || !inside(p.srcoff, p.ext, SS)) return;
+    }
+  }
+  int slabs = 1;
+  for (int g = 2; g <= 8; ++g)
+    if (N % g == 0) slabs = g;
+  if (slabs < 2) return;
+  const int64_t per = N / slabs;
+  const int es = m.elem_size;
+  amap_map sub;
+  sub.m = m;
+  sub.m.guard_views.clear();
+  sub.m.domain_views.clear();
+  for (Piece &p : sub.m.pieces) p.ext[0] = per;
+  sub.m.out_numel = DS * per;
+  sub.m.stages[0].numel = sub.m.out_numel;
+  for (size_t q = 0; q < m.in_numel.size(); ++q) sub.m.in_numel[q] = m.in_numel[q] / N * per;
+  if ((sub.m.out_numel * es) % pl->pointer_align) return;
+  for (int64_t n : sub.m.in_numel)
+    if ((n * es) % pl->pointer_align) return;
+  amap_plan_t *sp = nullptr;
+  if (plan_impl(&sub, device, &o, false, &sp) != AMAP_OK) return;
+  pl->slab_plan = sp;
+  pl->n_slabs = slabs;
+  pl->slab_out_bytes = sub.m.out_numel * es;
+  for (int64_t n : sub.m.in_numel) pl->slab_in_bytes.push_back(n * es);
+}
+
+static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts, bool allow_slabs, amap_plan_t **out_plan) {
   if (!map || !out_plan) return AMAP_EINVAL;
   amap_plan_opts o;
   memset(&o, 0, sizeof o);
@@ -801,8 +865,13 @@ extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *
     amap_plan_destroy(pl);
     return rc;
   }
+  if (allow_slabs) plan_slabs(m, device, o, pl);  // best effort: without it amap_execute_host copies in one piece
   *out_plan = pl;
   return AMAP_OK;
+}
+
+extern "C" int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts, amap_plan_t **out_plan) {
+  return plan_impl(map, device, opts, true, out_plan);
 }
 
 extern "C" void amap_plan_destroy(amap_plan_t *plan) {
@@ -820,6 +889,10 @@ extern "C" void amap_plan_destroy(amap_plan_t *plan) {
   for (void *p : plan->stage_in)
     if (p) cudaFree(p);
   if (plan->stage_out) cudaFree(plan->stage_out);
+  if (plan->slab_plan) amap_plan_destroy(plan->slab_plan);
+  if (plan->h2d_stream) cudaStreamDestroy(plan->h2d_stream);
+  if (plan->d2h_stream) cudaStreamDestroy(plan->d2h_stream);
+  for (cudaEvent_t ev : plan->events) cudaEventDestroy(ev);
   cudaSetDevice(prev);
   delete plan;
 }
@@ -1006,6 +1079,52 @@ extern "C" int amap_execute_host(amap_plan_t *plan, const void *const *src_host_
   for (size_t q = 0; q < plan->in_numel.size() && e == cudaSuccess; ++q)
     if (!plan->stage_in[q] && plan->in_numel[q] > 0) e = cudaMalloc(&plan->stage_in[q], plan->in_numel[q] * es);
   if (e == cudaSuccess && !plan->stage_out && plan->out_numel > 0) e = cudaMalloc(&plan->stage_out, plan->out_numel * es);
+  if (e == cudaSuccess && plan->slab_plan && plan->events.empty()) {  // the pipeline's streams and events, once
+    e = cudaStreamCreateWithFlags(&plan->h2d_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&plan->d2h_stream, cudaStreamNonBlocking);
+    for (int k = 0; k < 2 * plan->n_slabs + 2 && e == cudaSuccess; ++k) {
+      cudaEvent_t ev;
+      e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+      if (e == cudaSuccess) plan->events.push_back(ev);
+    }
+  }
+  if (e == cudaSuccess && plan->slab_plan) {
+    // upload slab k+1 while slab k runs and slab k-1 downloads; the caller's stream carries the kernels
+    const int S = plan->n_slabs;
+    cudaEvent_t *ev = plan->events.data();
+    e = cudaEventRecord(ev[0], s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(plan->h2d_stream, ev[0], 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(plan->d2h_stream, ev[0], 0);
+    std::vector<const void *> srcs(plan->in_numel.size());
+    for (int k = 0; k < S && e == cudaSuccess && rc == AMAP_OK; ++k) {
+      for (size_t q = 0; q < plan->in_numel.size() && e == cudaSuccess; ++q) {
+        const size_t off = (size_t)k * plan->slab_in_bytes[q];
+        srcs[q] = (const char *)plan->stage_in[q] + off;
+        if (plan->slab_in_bytes[q] > 0)
+          e = cudaMemcpyAsync((char *)plan->stage_in[q] + off, (const char *)src_host_ptrs[q] + off, plan->slab_in_bytes[q],
+                              cudaMemcpyHostToDevice, plan->h2d_stream);
+      }
+      if (e == cudaSuccess) e = cudaEventRecord(ev[1 + 2 * k], plan->h2d_stream);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ev[1 + 2 * k], 0);
+      char *out_k = (char *)plan->stage_out + (size_t)k * plan->slab_out_bytes;
+      if (e == cudaSuccess) rc = amap_execute(plan->slab_plan, srcs.data(), out_k, cuda_stream);
+      if (e == cudaSuccess && rc == AMAP_OK) e = cudaEventRecord(ev[2 + 2 * k], s);
+      if (e == cudaSuccess && rc == AMAP_OK) e = cudaStreamWaitEvent(plan->d2h_stream, ev[2 + 2 * k], 0);
+      if (e == cudaSuccess && rc == AMAP_OK)
+        e = cudaMemcpyAsync((char *)dst_host_ptr + (size_t)k * plan->slab_out_bytes, out_k, plan->slab_out_bytes,
+                            cudaMemcpyDeviceToHost, plan->d2h_stream);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ev[2 * S + 1], plan->d2h_stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, ev[2 * S + 1], 0);
+    // always drain what was enqueued, also after an error, before the buffers can be reused
+    cudaStreamSynchronize(plan->h2d_stream);
+    cudaStreamSynchronize(plan->d2h_stream);
+    const cudaError_t e2 = cudaStreamSynchronize(s);
+    if (e == cudaSuccess) e = e2;
+    cudaSetDevice(prev);
+    if (e != cudaSuccess) return cuda_fail(e, "amap_execute_host");
+    return rc;
+  }
   for (size_t q = 0; q < plan->in_numel.size() && e == cudaSuccess; ++q)
     if (plan->in_numel[q] > 0)
       e = cudaMemcpyAsync(plan->stage_in[q], src_host_ptrs[q], plan->in_numel[q] * es, cudaMemcpyHostToDevice, s);

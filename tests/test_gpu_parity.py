@@ -241,8 +241,13 @@ def test_other_element_sizes(B, dtype, es):
     assert np.array_equal(got, want.reshape(-1))
 
 
-def test_execute_host_matches(B):
-    chain = W.reduced_configs()["c4_odd"]
+@pytest.mark.parametrize("name", ["c4_odd", "c2_fwd_mid", "c3", "c4", "c5", "c1"])
+def test_execute_host_matches(B, name):
+    """Host buffers in, host buffers out.  Maps with an outer batch loop go slab by slab on extra streams
+    (c2, c3, c4); the others (guards, no batch loop) in one piece."""
+    import torch
+
+    chain = W.reduced_configs()[name]
     xs = W.make_inputs(chain)
     want = oracle.run_chain(chain, xs)
     m = B.compose_chain(chain)
@@ -250,9 +255,15 @@ def test_execute_host_matches(B):
     out = np.empty(m.out_numel, dtype=xs[0].dtype)
     plan.execute_host([np.ascontiguousarray(x) for x in xs], out)
     assert np.array_equal(out, want.reshape(-1))
-    out[:] = 0
-    plan.execute_host([np.ascontiguousarray(x) for x in xs], out)  # staging buffers are reused
-    assert np.array_equal(out, want.reshape(-1))
+    # pinned buffers (truly asynchronous copies), staging reused, a non-default stream
+    es = chain.elem_size
+    pins = [torch.from_numpy(np.ascontiguousarray(x).view(SIGNED[es])).pin_memory() for x in xs]
+    pout = torch.zeros(m.out_numel, dtype=pins[0].dtype).pin_memory()
+    stream = torch.cuda.Stream()
+    for _ in range(2):
+        pout.zero_()
+        plan.execute_host(pins, pout, stream.cuda_stream)
+        assert np.array_equal(pout.numpy().view(xs[0].dtype), want.reshape(-1))
 
 
 def test_misaligned_pointer_is_refused(B):
