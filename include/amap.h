@@ -227,7 +227,7 @@ typedef struct amap_stats {
   int32_t n_launches;     /* kernels one amap_execute enqueues                 */
   int32_t kernel_kind[4]; /* pieces planned per family: [0] gather [1] copy [2] transpose [3] fill */
   int32_t n_stages;       /* 1 unless the map keeps temporaries */
-  int32_t reserved[1];
+  int32_t n_descriptors;  /* launch descriptors behind the pieces (a piece may be cut into several)   */
 } amap_stats;
 
 int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts /* host, may be NULL */,

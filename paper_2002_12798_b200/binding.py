@@ -71,7 +71,7 @@ class _PlanOpts(Structure):
 class _Stats(Structure):
     _fields_ = [
         ("bytes_read", c_int64), ("bytes_written", c_int64), ("bytes_filled", c_int64), ("n_pieces", c_int32),
-        ("n_launches", c_int32), ("kernel_kind", c_int32 * 4), ("n_stages", c_int32), ("reserved", c_int32 * 1),
+        ("n_launches", c_int32), ("kernel_kind", c_int32 * 4), ("n_stages", c_int32), ("n_descriptors", c_int32),
     ]
 
 
@@ -288,7 +288,7 @@ class Plan:
         _check(_lib.amap_plan_stats(self._h, byref(s)), "amap_plan_stats")
         return {
             "bytes_read": s.bytes_read, "bytes_written": s.bytes_written, "bytes_filled": s.bytes_filled,
-            "n_pieces": s.n_pieces, "n_launches": s.n_launches, "n_stages": s.n_stages,
+            "n_pieces": s.n_pieces, "n_launches": s.n_launches, "n_stages": s.n_stages, "n_descriptors": s.n_descriptors,
             "kernels": {"gather": s.kernel_kind[0], "copy": s.kernel_kind[1], "transpose": s.kernel_kind[2], "fill": s.kernel_kind[3]},
         }
 

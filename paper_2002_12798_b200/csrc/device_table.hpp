@@ -75,10 +75,12 @@ struct DevPiece {
   int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
   int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less; 0: shifted rows, -1: realigned source rows
-  int32_t pad1_;
+  int32_t tile_ca;            // 16-byte kernel: 16-byte chunks of a per tile, 8 (by 128 elements of b) or 4 (by 256)
   int64_t src_bytes;          // size of the source tensor (shifted-row kernel: guards the last aligned chunk)
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b
+  uint32_t step_b;            // 16-byte kernel: elements of b between tiles (at most what a tile holds)
+  uint32_t pad1_;
   FastDiv fd_tiles_a, fd_tiles_b;
   FastDiv fd_a_in, fd_b_in;  // inner extents of the merged indices
   int64_t sa[2];             // source byte strides of (a_lo, a_hi)

@@ -256,12 +256,12 @@ __device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &p
 // bank-conflict-free.  Tiles on the ragged edge are predicated per chunk (the
 // planner only selects this kernel when both extents are multiples of 16/ES).
 // ---------------------------------------------------------------------------
-template <int ES>
+template <int ES, int CA = 8>
 __device__ __forceinline__ uint4 gather_column(const unsigned char *tile, int ca, int b_l) {
   constexpr int EPU = 16 / ES;
-  constexpr int RB = kTileB * ES;
+  constexpr int RB = kTileB * ES * (8 / CA);
   const int chunk = b_l / EPU;
-  const unsigned char *p = tile + (ca * EPU) * RB + ((chunk ^ ca) << 4) + (b_l % EPU) * ES;
+  const unsigned char *p = tile + (ca * EPU) * RB + ((chunk ^ (ca * (8 / CA))) << 4) + (b_l % EPU) * ES;
   uint4 out;
   if constexpr (ES == 1) {
     uint32_t w[4];
@@ -333,27 +333,24 @@ __device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
   }
 }
 
-struct LaunchDesc;
-__device__ __forceinline__ const DevPiece *piece_of_block(const LaunchDesc *ld, uint32_t block);
-
-template <int ES, typename OffT>
-__device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs, const LaunchDesc *ld) {
+// CA = 16-byte chunks of a per tile: 8 (128 bytes of a by 128 elements of b) or 4 (64 bytes of a by 256 elements
+// of b, for pieces or remainders at most 64 bytes long in a, which would leave the wide tile half empty).  The
+// planner may shorten the step along b (sp.step_b) so that the tiles of a row are evenly filled.
+template <int ES, typename OffT, int CA>
+__device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTable &ptrs, unsigned char *tile) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
-  constexpr int TA = 8 * EPU;      // rows of the tile: 128 bytes of destination run
-  constexpr int RB = kTileB * ES;  // bytes per row
+  constexpr int TA = CA * EPU;     // rows of the tile
+  constexpr int TB = kTileB * (8 / CA);  // elements of b a tile can hold
+  constexpr int RB = TB * ES;      // bytes per row
   constexpr int CB = RB / 16;      // chunks per row
+  constexpr int SW = 8 / CA;       // swizzle step: chunk index XOR (a / EPU) * SW
   constexpr int U = TA * CB / kTransposeThreads;
   static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB, "tile geometry");
-  __shared__ __align__(128) unsigned char tile[kTileBytes];
-  if (sp.kind != kDevTranspose) {  // block-uniform
-    pdl_wait();
-    fill_block(sp, ptrs.dst);
-    return;
-  }
 
+  const uint32_t step_b = sp.step_b;
   uint32_t t = blockIdx.x - sp.first_block;
   uint32_t q = fast_div(t, sp.fd_tiles_b);
-  const uint32_t b0 = (t - q * sp.tiles_b) * kTileB;
+  const uint32_t b0 = (t - q * sp.tiles_b) * step_b;
   t = q;
   q = fast_div(t, sp.fd_tiles_a);
   const uint32_t a0 = (t - q * sp.tiles_a) * TA;
@@ -368,20 +365,21 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
   }
   const char *src = ptrs.src[sp.input] + sbase;
   char *dst = ptrs.dst + dbase;
-  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  const uint32_t ext_a = sp.ext_a;
+  const uint32_t end_b = min(sp.ext_b, b0 + step_b);  // the tile's own end along b
   // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
   // reads nothing into the SM and is harmless whatever that kernel still writes); the loads after the wait
   // then start from L2 instead of paying a DRAM round trip with the memory system idle.
-  auto prefetch_rows = [&](const DevPiece &pp, const char *base, uint32_t pa0, uint32_t pb0) {
+  auto prefetch_rows = [&](const char *base, uint32_t pa0, uint32_t pb0) {
     const uint32_t a = pa0 + threadIdx.x;
-    if (a < pp.ext_a && pb0 < pp.ext_b) {
-      const uint32_t a_hi = fast_div(a, pp.fd_a_in);
-      const char *row = base + (int64_t)(a - a_hi * pp.fd_a_in.d) * pp.sa[0] + (int64_t)a_hi * pp.sa[1] + (int64_t)pb0 * ES;
-      const uint32_t bytes = min((uint32_t)kTileB, pp.ext_b - pb0) * ES;
+    if (a < ext_a && pb0 < sp.ext_b) {
+      const uint32_t a_hi = fast_div(a, sp.fd_a_in);
+      const char *row = base + (int64_t)(a - a_hi * sp.fd_a_in.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)pb0 * ES;
+      const uint32_t bytes = min(step_b, sp.ext_b - pb0) * ES;
       asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
     }
   };
-  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(sp, src, a0, b0);
+  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(src, a0, b0);
   pdl_wait();
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];
@@ -395,7 +393,7 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
       const int a_l = idx / CB, cb = idx % CB;
       const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
       v[u] = make_uint4(0, 0, 0, 0);
-      if (a < ext_a && b < ext_b) {
+      if (a < ext_a && b < end_b) {
         OffT off = (OffT)(b * ES);
         if (split) {
           const uint32_t a_hi = fast_div(a, fa);
@@ -408,41 +406,38 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
     }
     issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
     // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
-    // blocks further on in the grid): its loads will find their lines in L2.
+    // blocks further on in the grid): its loads will find their lines in L2.  Only within this piece: on a
+    // launch of several small pieces (measured on configuration 4) hints for another piece's tiles cost more
+    // than they save.
     if (sp.prefetch > 1 && threadIdx.x < TA) {
-      const uint32_t g = blockIdx.x + (uint32_t)sp.prefetch;
-      // only within this piece: on a launch of several small pieces (measured on configuration 4) hints for
-      // another piece's tiles cost more than they save
-      const DevPiece *np = (g - sp.first_block < sp.n_blocks) ? &sp : nullptr;
-      (void)ld;
-      if (np != nullptr && np->kind == kDevTranspose) {
-        uint32_t t2 = g - np->first_block;
-        uint32_t q2 = fast_div(t2, np->fd_tiles_b);
-        const uint32_t nb0 = (t2 - q2 * np->tiles_b) * kTileB;
+      uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
+      if (t2 < sp.n_blocks) {
+        uint32_t q2 = fast_div(t2, sp.fd_tiles_b);
+        const uint32_t nb0 = (t2 - q2 * sp.tiles_b) * step_b;
         t2 = q2;
-        q2 = fast_div(t2, np->fd_tiles_a);
-        const uint32_t na0 = (t2 - q2 * np->tiles_a) * TA;
+        q2 = fast_div(t2, sp.fd_tiles_a);
+        const uint32_t na0 = (t2 - q2 * sp.tiles_a) * TA;
         t2 = q2;
-        int64_t nbase = np->soff;
-        for (int k = np->n_loops - 1; k >= 0; --k) {
-          q2 = fast_div(t2, np->fd[k]);
-          nbase += (int64_t)(t2 - q2 * np->ext[k]) * np->sstride[k];
+        int64_t nbase = sp.soff;
+        for (int k = sp.n_loops - 1; k >= 0; --k) {
+          q2 = fast_div(t2, sp.fd[k]);
+          nbase += (int64_t)(t2 - q2 * sp.ext[k]) * sp.sstride[k];
           t2 = q2;
         }
-        prefetch_rows(*np, ptrs.src[np->input] + nbase, na0, nb0);
+        prefetch_rows(ptrs.src[sp.input] + nbase, na0, nb0);
       }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
       const int a_l = idx / CB, cb = idx % CB;
-      *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+      *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ (((a_l / EPU) * SW) & 7)) << 4)) = v[u];
     }
   }
   __syncthreads();
   // phase 2: shared -> global, 16 bytes along a
   const FastDiv fb = sp.fd_b_in;
-  const bool split_b = fb.d < ext_b;  // b merges two loops
+  const bool split_b = fb.d < sp.ext_b;  // b merges two loops
   const OffT db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
   auto dst_of = [&](uint32_t a, uint32_t b) -> char * {
     OffT off = (OffT)(a * ES);
@@ -459,10 +454,10 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
 #pragma unroll
     for (int u = 0; u < U / 2; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx & 7, b_l = (idx >> 3) * 2;
+      const int ca = idx % CA, b_l = (idx / CA) * 2;
       const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
-      if (a < ext_a && b < ext_b) {  // extents are even: b + 1 is inside too
-        const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ ca) << 4) + (b_l % EPU) * ES;
+      if (a < ext_a && b < end_b) {  // extents and steps are even: b + 1 is inside too
+        const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ (ca * SW)) << 4) + (b_l % EPU) * ES;
         uint32_t r[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * RB);
@@ -479,11 +474,23 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx & 7, b_l = idx >> 3;
+      const int ca = idx % CA, b_l = idx / CA;
       const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
-      if (a < ext_a && b < ext_b) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), gather_column<ES>(tile, ca, b_l));
+      if (a < ext_a && b < end_b) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), gather_column<ES, CA>(tile, ca, b_l));
     }
   }
+}
+
+template <int ES, typename OffT>
+__device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTable &ptrs) {
+  __shared__ __align__(128) unsigned char tile[kTileBytes];
+  if (sp.kind != kDevTranspose) {  // block-uniform
+    pdl_wait();
+    fill_block(sp, ptrs.dst);
+    return;
+  }
+  if (sp.tile_ca == 4) transpose_tile<ES, OffT, 4>(sp, ptrs, tile);
+  else transpose_tile<ES, OffT, 8>(sp, ptrs, tile);
 }
 
 // ---------------------------------------------------------------------------
@@ -875,21 +882,12 @@ __device__ __forceinline__ void transpose_realign_body(const DevPiece &sp, const
 // the *_table kernels read them from a descriptor table in global memory
 // (launches with more pieces, and amap_execute_static).
 // ---------------------------------------------------------------------------
-constexpr int kParamPieces = 8;
+constexpr int kParamPieces = 16;
 struct LaunchDesc {
   int32_t n_pieces;
   int32_t pad_;
   DevPiece piece[kParamPieces];
 };
-
-// the piece that owns block `block` of the launch, or null (past the end, or descriptors not in the parameters)
-__device__ __forceinline__ const DevPiece *piece_of_block(const LaunchDesc *ld, uint32_t block) {
-  if (ld == nullptr) return nullptr;
-  int p = 0;
-  while (p + 1 < ld->n_pieces && block >= ld->piece[p + 1].first_block) ++p;
-  const DevPiece *d = &ld->piece[p];
-  return (block - d->first_block < d->n_blocks) ? d : nullptr;
-}
 
 __device__ __forceinline__ const DevPiece &param_piece(const LaunchDesc &ld) {
   int p = 0;
@@ -929,7 +927,7 @@ template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_param(const __grid_constant__ LaunchDesc ld,
                                                                               PtrTable ptrs) {
   pdl_launch_dependents();
-  transpose_body<ES, OffT>(param_piece(ld), ptrs, &ld);
+  transpose_body<ES, OffT>(param_piece(ld), ptrs);
 }
 template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const DevPiece *__restrict__ table,
@@ -937,7 +935,7 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_table(const 
   __shared__ DevPiece sp;
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
-  transpose_body<ES, OffT>(sp, ptrs, nullptr);
+  transpose_body<ES, OffT>(sp, ptrs);
 }
 
 template <int ES, int UB, typename OffT>
@@ -986,7 +984,7 @@ __global__ void __launch_bounds__(kAffineThreads) amap_strip_one(const __grid_co
 template <int ES, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads, 8) amap_transpose_one(const __grid_constant__ DevPiece p, PtrTable ptrs) {
   pdl_launch_dependents();
-  transpose_body<ES, OffT>(p, ptrs, nullptr);
+  transpose_body<ES, OffT>(p, ptrs);
 }
 template <int ES, int UB, typename OffT>
 __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_narrow_one(const __grid_constant__ DevPiece p,

@@ -323,6 +323,51 @@ static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_
 // on that one side only (e.g. (h, w) is one run in an NCHW source but two
 // strides in a padded NHWC destination).
 // ---------------------------------------------------------------------------
+// Tile counts of a transpose descriptor whose extents and batch loops are set: tiles of `ca` 16-byte chunks of a
+// by up to kTileB * 8 / ca elements of b.  With `even` the step along b is shortened to the smallest multiple of
+// a chunk that still covers ext_b with the same number of tiles, so that no tile is left nearly empty
+// (784 = 7 x 112 instead of 6 x 128 + 16).
+static bool set_transpose_tiles(DevPiece *d, int ca, bool even) {
+  const int es = d->unit_bytes, epu = 16 / es;
+  const uint32_t ta = (uint32_t)(ca * epu), tb = (uint32_t)(kTileB * (8 / ca));
+  d->tile_ca = ca;
+  d->tiles_a = (d->ext_a + ta - 1) / ta;
+  d->tiles_b = (d->ext_b + tb - 1) / tb;
+  d->step_b = tb;
+  if (even) {
+    const uint32_t per = (d->ext_b + d->tiles_b - 1) / d->tiles_b;
+    d->step_b = std::min(tb, (per + epu - 1) / epu * epu);
+  }
+  d->fd_tiles_a = make_fastdiv(d->tiles_a);
+  d->fd_tiles_b = make_fastdiv(d->tiles_b);
+  unsigned __int128 blocks = (unsigned __int128)d->tiles_a * d->tiles_b;
+  for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
+  if (blocks > 0x7FFFFFFFull) return false;
+  d->n_blocks = (uint32_t)blocks;
+  d->n_items = (uint64_t)blocks;
+  return true;
+}
+
+// A 16-byte transpose piece whose extent along a leaves a remainder of at most half a tile is cut in two: whole
+// tiles, and the remainder as a piece of its own on the narrow tile (64 bytes of a by 256 elements of b), which
+// would otherwise travel in half-empty tiles.  Returns false when the piece stays as it is.
+static bool split_a_remainder(const DevPiece &d, DevPiece *whole, DevPiece *rest) {
+  const int es = d.unit_bytes, epu = 16 / es;
+  const uint32_t ta = (uint32_t)(8 * epu);
+  if (d.tr_unit != 16 || d.tile_ca != 8 || d.fd_a_in.d < d.ext_a) return false;  // a merges two loops: not cut
+  const uint32_t rem = d.ext_a % ta;
+  if (d.ext_a <= ta || rem == 0 || rem > ta / 2) return false;
+  *whole = d;
+  whole->ext_a = d.ext_a - rem;
+  whole->fd_a_in = make_fastdiv(whole->ext_a);
+  *rest = d;
+  rest->ext_a = rem;
+  rest->fd_a_in = make_fastdiv(rem);
+  rest->soff = d.soff + (int64_t)whole->ext_a * d.sa[0];
+  rest->doff = d.doff + (int64_t)whole->ext_a * es;
+  return set_transpose_tiles(whole, 8, true) && set_transpose_tiles(rest, 4, true);
+}
+
 static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t in_bytes, DevPiece *d) {
   if (es > 8 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
   const int n = p.n();
@@ -363,7 +408,6 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     bool aligned = (d->soff % ub == 0) && (d->doff % ub == 0) && (d->sa[0] % ub == 0) && (d->sa[1] % ub == 0) &&
                    (d->db[0] % ub == 0) && (d->db[1] % ub == 0);
     int j = 0;
-    unsigned __int128 batch = 1;
     for (int k = 0; k < n; ++k) {
       if (k == ia || k == a_hi || k == ib || k == b_hi) continue;
       if (j >= kDevMaxLoops) return false;
@@ -372,21 +416,12 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       d->sstride[j] = p.srcoff.c[k] * es;
       d->dstride[j] = p.dst.c[k] * es;
       if (d->sstride[j] % ub || d->dstride[j] % ub) aligned = false;
-      batch *= (uint64_t)p.ext[k];
       ++j;
     }
     if (!aligned) return false;
     d->n_loops = j;
-    const int ta = 8 * (16 / es);
-    d->tiles_a = (uint32_t)((ext_a + ta - 1) / ta);
-    d->tiles_b = (uint32_t)((ext_b + kTileB - 1) / kTileB);
-    d->fd_tiles_a = make_fastdiv(d->tiles_a);
-    d->fd_tiles_b = make_fastdiv(d->tiles_b);
-    const unsigned __int128 blocks = batch * d->tiles_a * d->tiles_b;
-    if (blocks > 0x7FFFFFFFull) return false;
-    d->n_blocks = (uint32_t)blocks;
-    d->n_items = (uint64_t)blocks;
-    return true;
+    // the 16-byte kernel takes the narrow tile (4 chunks of a) for pieces at most that long in a
+    return set_transpose_tiles(d, (ub == 16 && ext_a <= 4 * (16 / es)) ? 4 : 8, ub == 16);
   };
   // units of a single element gain nothing over the strip kernel's gather (measured): at least two per access
   for (int ub = 16; ub >= 2 * es; ub >>= 1) {
@@ -512,11 +547,15 @@ static bool check_realign_block(const DevPiece &d, uint32_t blk, int64_t in_byte
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   if (d.tr_unit < 0) return check_realign_block(d, blk, in_bytes, out_bytes);
-  const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
+  const int es = d.unit_bytes, epu = 16 / es, ca = d.tile_ca, ta = ca * epu, sw = 8 / ca;
+  if ((ca != 8 && !(ca == 4 && d.tr_unit == 16)) || d.step_b == 0 || d.step_b % epu || d.step_b > (uint32_t)(kTileB * sw) ||
+      (uint64_t)d.tiles_b * d.step_b < d.ext_b || (uint64_t)d.tiles_a * ta < d.ext_a)
+    return false;
   uint32_t t = blk;
   uint32_t q = host_fast_div(t, d.fd_tiles_b);
   if (q != t / d.tiles_b) return false;
-  const uint32_t b0 = (t - q * d.tiles_b) * kTileB;
+  const uint32_t b0 = (t - q * d.tiles_b) * d.step_b;
+  const uint32_t end_b = std::min<uint32_t>(d.ext_b, b0 + d.step_b);
   t = q;
   q = host_fast_div(t, d.fd_tiles_a);
   if (q != t / d.tiles_a) return false;
@@ -532,13 +571,13 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
     dbase += (int64_t)i * d.dstride[k];
   }
   if (t != 0) return false;
-  const int ub = d.tr_unit, epn = ub / es, rb = kTileB * es, cbu = rb / ub, nca = ta / epn;
-  auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ ((row / epu) & 7)) << 4) | (col & 15)); };
+  const int ub = d.tr_unit, epn = ub / es, rb = kTileB * sw * es, cbu = rb / ub, nca = ta / epn;
+  auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ (((row / epu) * sw) & 7)) << 4) | (col & 15)); };
   for (int idx = 0; idx < kTileBytes / ub; ++idx) {
     {  // phase 1
       const int a_l = idx / cbu, cu = idx % cbu;
       const uint32_t a = a0 + a_l, b = b0 + cu * epn;
-      if (a < d.ext_a && b < d.ext_b) {
+      if (a < d.ext_a && b < end_b) {
         const uint32_t a_hi = host_fast_div(a, d.fd_a_in);
         if (a_hi != a / d.fd_a_in.d) return false;
         const uint32_t a_lo = a - a_hi * d.fd_a_in.d;
@@ -551,7 +590,7 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
     {  // phase 2
       const int ca = idx % nca, b_l = idx / nca;
       const uint32_t a = a0 + ca * epn, b = b0 + b_l;
-      if (a < d.ext_a && b < d.ext_b) {
+      if (a < d.ext_a && b < end_b) {
         const uint32_t b_hi = host_fast_div(b, d.fd_b_in);
         if (b_hi != b / d.fd_b_in.d) return false;
         const uint32_t b_lo = b - b_hi * d.fd_b_in.d;
@@ -610,8 +649,8 @@ static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
 }
 
 // One launch of the transpose kernel per (access width, offset width) present.  Fill pieces with 16-byte units
-// and no constraints ride in the 16-byte launch (first: they only store and wait for nothing), so that padding
-// borders do not cost a launch of their own.
+// and no constraints ride in the 16-byte launch, so that padding borders do not cost a launch of their own; their
+// blocks come last (measured: 0.4 us faster on a 69 MB padded transpose than with the fills first).
 static int plan_stage_transposes(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
@@ -628,7 +667,14 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
         const bool needs_wide = (in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && access > 0;
         if ((int)needs_wide != wide) continue;
         if (!check_transpose_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
-        transposes.push_back(d);
+        DevPiece whole, rest;
+        if (split_a_remainder(d, &whole, &rest) && check_transpose_piece(whole, in_bytes, out_bytes) &&
+            check_transpose_piece(rest, in_bytes, out_bytes)) {
+          transposes.push_back(whole);
+          transposes.push_back(rest);
+        } else {
+          transposes.push_back(d);
+        }
         taken.push_back(q);
       }
       if (transposes.empty()) continue;
@@ -642,9 +688,9 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
         fills.push_back(d);
         taken.push_back(q);
       }
-      for (const DevPiece &d : fills)
-        if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
       for (const DevPiece &d : transposes)
+        if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
+      for (const DevPiece &d : fills)
         if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
       for (size_t q : taken) c.placed[q] = 1;
       c.pl->launches.push_back(L);
@@ -824,6 +870,7 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
     pl->stats.kernel_kind[slot]++;
   }
   pl->stats.n_launches = (int32_t)pl->launches.size();
+  pl->stats.n_descriptors = (int32_t)pl->table.size();
   pl->stats.n_stages = (int32_t)m.stages.size();
   {
     // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM)

@@ -273,6 +273,14 @@ def reduced_configs() -> dict:
         "c2_fwd_odd_f32b": c2_nchw_to_nhwc(N=2, C=36, H=7, W=9, dtype="fp32"),
         "c2_fwd_narrow": c2_nchw_to_nhwc(N=2, C=72, H=14, W=14),
         "c2_inv_narrow": c2_nhwc_to_nchw(N=2, C=68, H=14, W=14),
+        # 16-byte transposes whose extent along the destination run leaves at most half a tile (remainder pieces on
+        # the 64-byte tile), or is that short altogether; several tiles along the other index, evenly stepped
+        "c2_fwd_rem": c2_nchw_to_nhwc(N=2, C=96, H=20, W=26),
+        "c2_fwd_rem_f32": c2_nchw_to_nhwc(N=2, C=40, H=12, W=23, dtype="fp32"),
+        "c2_fwd_rem_u8": c2_nchw_to_nhwc(N=2, C=160, H=16, W=37, dtype="u8"),
+        "c2_fwd_rem_u64": c2_nchw_to_nhwc(N=2, C=20, H=10, W=53, dtype="u64"),
+        "c2_fwd_short": c2_nchw_to_nhwc(N=2, C=24, H=20, W=26),
+        "c2_inv_rem": c2_nhwc_to_nchw(N=2, C=280, H=8, W=12),
         "c3": c3_head_split(B=2, S=80, heads=3, D=128, keep=50),
         "c3_odd": c3_head_split(B=2, S=33, heads=5, D=24, keep=17),
         "c3_merge": c3_head_merge(B=2, S=70, heads=3, D=128),

@@ -175,9 +175,9 @@ def test_offsets_beyond_4_gib(B):
 
 
 def test_launch_with_more_pieces_than_fit_the_kernel_parameters(B):
-    """Twelve operands joined and transposed: twelve pieces in one launch, so the kernels read their descriptors
+    """Twenty operands joined and transposed: twenty pieces in one launch, so the kernels read their descriptors
     from the plan's table in device memory instead of the kernel parameters."""
-    n_in = 12
+    n_in = 20
     chain = W.Chain(
         name="wide_concat", dtype="bf16", inputs=[[2, 16, 8, 8]] * n_in,
         ops=[{"kind": "concat", "srcs": list(range(n_in)), "axis": 1}, {"kind": "transpose", "src": n_in, "perm": [0, 2, 3, 1]}],

@@ -51,6 +51,21 @@ def test_shifted_transpose_for_misaligned_destination_rows():
     assert k["gather"] == 1
 
 
+def test_remainders_of_at_most_half_a_tile_become_pieces_of_their_own():
+    """The 16-byte transpose kernel's tile spans 128 bytes of the destination run.  An extent that leaves at most
+    64 bytes over is cut: whole tiles, plus the remainder on the 64-byte tile."""
+    def descriptors(chain):
+        return B.compose_chain(chain).plan(device=-1).stats()["n_descriptors"]
+
+    assert descriptors(W.c2_nchw_to_nhwc(N=2, C=128, H=20, W=26)) == 1  # whole tiles only
+    assert descriptors(W.c2_nchw_to_nhwc(N=2, C=96, H=20, W=26)) == 2   # 64 + 32 channels
+    assert descriptors(W.c2_nchw_to_nhwc(N=2, C=112, H=20, W=26)) == 1  # 48 left over: more than half a tile
+    assert descriptors(W.c2_nchw_to_nhwc(N=2, C=24, H=20, W=26)) == 1   # shorter than half a tile altogether
+    assert descriptors(W.c2_nchw_to_nhwc(N=2, C=40, H=12, W=23, dtype="fp32")) == 2  # 32 + 8 four-byte elements
+    # configuration 4: operands of 64, 96, 128, 32 channels -> five transpose descriptors and four border fills
+    assert descriptors(W.full_configs()["c4"]) == 9
+
+
 def test_unfused_chain_has_one_stage_per_operator_and_moves_more_bytes():
     c3 = W.full_configs()["c3"]
     fused = B.compose_chain(c3).plan(device=-1).stats()
