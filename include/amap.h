@@ -119,6 +119,14 @@ int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int32_t kw, in
                         int32_t *out);
 /* broadcast: out[o] = in[o mod in.shape] with out.shape[d] = reps[d]*in.shape[d] (the paper's repeat/tile family) */
 int amap_builder_tile(amap_builder *b, int32_t src, int32_t rank, const int64_t *reps, int32_t *out);
+/* every element `count` times in a row along `axis`: out[.., i*count + j, ..] = in[.., i, ..] (a load that ignores
+ * one loop; Section 2.1 names repeat among the operators whose copies are eliminated) */
+int amap_builder_repeat(amap_builder *b, int32_t src, int32_t axis, int64_t count, int32_t *out);
+/* cut `src` along `axis` into n_parts consecutive tensors of the given sizes (they must add up to the extent;
+ * Section 2.1 names split); outs receives n_parts tensor ids (host array, caller-owned).  Each part is a tensor
+ * of its own: compose once per part that is wanted as an output. */
+int amap_builder_split(amap_builder *b, int32_t src, int32_t axis, int32_t n_parts, const int64_t *sizes,
+                       int32_t *outs);
 /* declare a tensor that raw statements will define */
 int amap_builder_tensor(amap_builder *b, int32_t rank, const int64_t *shape, int32_t *out);
 /* append one raw statement (deep-copied) */

@@ -223,6 +223,92 @@ int oracle_window_gather(const void *in, void *out, const int64_t *in_shape /* N
   return 0;
 }
 
+/* tile(reps): the whole tensor laid side by side reps[d] times along every
+ * axis (Section 2.1 names tile and repeat among the pure copies):
+ * out.shape[d] = reps[d]*in.shape[d], out[o] = in[j] with j[d] = o[d] mod in.shape[d]. */
+int oracle_tile(const void *in, void *out, int rank, const int64_t *in_shape, const int64_t *reps, int es,
+                int nt) {
+  if (bad_common(rank, in_shape, es) || !reps) return -1;
+  int64_t out_shape[ORACLE_MAX_RANK];
+  for (int d = 0; d < rank; ++d) {
+    if (reps[d] < 1) return -2;
+    out_shape[d] = reps[d] * in_shape[d];
+  }
+  if (numel(rank, in_shape) == 0) return 0;
+  const unsigned char *src = (const unsigned char *)in;
+  unsigned char *dst = (unsigned char *)out;
+#pragma omp parallel for num_threads(nt) schedule(static)
+  for (int64_t o0 = 0; o0 < out_shape[0]; ++o0) {
+    int64_t o[ORACLE_MAX_RANK] = {0}, j[ORACLE_MAX_RANK];
+    o[0] = o0;
+    do {
+      for (int d = 0; d < rank; ++d) j[d] = o[d] % in_shape[d];
+      copy_elem(dst, flat_of(rank, out_shape, o), src, flat_of(rank, in_shape, j), es);
+    } while (next_index(1, rank, out_shape, o));
+  }
+  return 0;
+}
+
+/* repeat(axis, count): every element count times in a row along one axis:
+ * out.shape[axis] = count*in.shape[axis], out[o] = in[j] with
+ * j[axis] = o[axis] div count and j[d] = o[d] elsewhere. */
+int oracle_repeat(const void *in, void *out, int rank, const int64_t *in_shape, int axis, int64_t count,
+                  int es, int nt) {
+  if (bad_common(rank, in_shape, es) || axis < 0 || axis >= rank || count < 1) return -1;
+  int64_t out_shape[ORACLE_MAX_RANK];
+  for (int d = 0; d < rank; ++d) out_shape[d] = in_shape[d];
+  out_shape[axis] = count * in_shape[axis];
+  if (numel(rank, in_shape) == 0) return 0;
+  const unsigned char *src = (const unsigned char *)in;
+  unsigned char *dst = (unsigned char *)out;
+#pragma omp parallel for num_threads(nt) schedule(static)
+  for (int64_t o0 = 0; o0 < out_shape[0]; ++o0) {
+    int64_t o[ORACLE_MAX_RANK] = {0}, j[ORACLE_MAX_RANK];
+    o[0] = o0;
+    do {
+      for (int d = 0; d < rank; ++d) j[d] = o[d];
+      j[axis] = o[axis] / count;
+      copy_elem(dst, flat_of(rank, out_shape, o), src, flat_of(rank, in_shape, j), es);
+    } while (next_index(1, rank, out_shape, o));
+  }
+  return 0;
+}
+
+/* split(axis, sizes): the tensor cut into consecutive parts along one axis;
+ * this writes part `part`: out.shape[axis] = sizes[part],
+ * out[o] = in[j] with j[axis] = o[axis] + sizes[0] + ... + sizes[part-1].
+ * The sizes must add up to in.shape[axis]. */
+int oracle_split_part(const void *in, void *out, int rank, const int64_t *in_shape, int axis, int n_parts,
+                      const int64_t *sizes, int part, int es, int nt) {
+  if (bad_common(rank, in_shape, es) || axis < 0 || axis >= rank || n_parts < 1 || !sizes || part < 0 ||
+      part >= n_parts)
+    return -1;
+  int64_t total = 0, first = 0;
+  for (int q = 0; q < n_parts; ++q) {
+    if (sizes[q] < 0) return -2;
+    if (q < part) first += sizes[q];
+    total += sizes[q];
+  }
+  if (total != in_shape[axis]) return -2;
+  int64_t out_shape[ORACLE_MAX_RANK];
+  for (int d = 0; d < rank; ++d) out_shape[d] = in_shape[d];
+  out_shape[axis] = sizes[part];
+  if (numel(rank, out_shape) == 0) return 0;
+  const unsigned char *src = (const unsigned char *)in;
+  unsigned char *dst = (unsigned char *)out;
+#pragma omp parallel for num_threads(nt) schedule(static)
+  for (int64_t o0 = 0; o0 < out_shape[0]; ++o0) {
+    int64_t o[ORACLE_MAX_RANK] = {0}, j[ORACLE_MAX_RANK];
+    o[0] = o0;
+    do {
+      for (int d = 0; d < rank; ++d) j[d] = o[d];
+      j[axis] = o[axis] + first;
+      copy_elem(dst, flat_of(rank, out_shape, o), src, flat_of(rank, in_shape, j), es);
+    } while (next_index(1, rank, out_shape, o));
+  }
+  return 0;
+}
+
 /* One load/store pair in the paper's form (Section 2, equations (load),
  * (store); Section 2.1's pair pattern): for every i in the box
  * 0 <= i_j < bounds[j], in lexicographic order,

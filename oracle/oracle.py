@@ -144,6 +144,42 @@ def window(x, kh, kw, stride, padding, nt=1):
     return out
 
 
+def tile(x, reps, nt=1):
+    x = _raw(x)
+    if len(reps) != x.ndim:
+        raise ValueError("reps rank")
+    out = np.empty([int(r) * n for r, n in zip(reps, x.shape)], dtype=x.dtype)
+    _check(lib().oracle_tile(_ptr(x), _ptr(out), x.ndim, _i64(x.shape), _i64(reps), x.itemsize, nt), "tile")
+    return out
+
+
+def repeat(x, axis, count, nt=1):
+    x = _raw(x)
+    shape = list(x.shape)
+    shape[axis] *= int(count)
+    out = np.empty(shape, dtype=x.dtype)
+    _check(
+        lib().oracle_repeat(_ptr(x), _ptr(out), x.ndim, _i64(x.shape), int(axis), ctypes.c_int64(int(count)), x.itemsize, nt),
+        "repeat",
+    )
+    return out
+
+
+def split_part(x, axis, sizes, part, nt=1):
+    """Part number `part` of x cut along `axis` into consecutive parts of the given sizes."""
+    x = _raw(x)
+    shape = list(x.shape)
+    shape[axis] = int(sizes[part])
+    out = np.empty(shape, dtype=x.dtype)
+    _check(
+        lib().oracle_split_part(
+            _ptr(x), _ptr(out), x.ndim, _i64(x.shape), int(axis), len(sizes), _i64(sizes), int(part), x.itemsize, nt
+        ),
+        "split",
+    )
+    return out
+
+
 def affine_stmt(dst, bounds, load, store, guarded=False, fill=0):
     """Run one load/store pair in the paper's form in place on `dst`.
 
@@ -197,6 +233,12 @@ def run_chain(chain, inputs, nt=1, keep_intermediates=False):
             t = pad(tensors[op["src"]], op["lo"], op["hi"], nt)
         elif kind == "window":
             t = window(tensors[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"], nt)
+        elif kind == "tile":
+            t = tile(tensors[op["src"]], op["reps"], nt)
+        elif kind == "repeat":
+            t = repeat(tensors[op["src"]], op["axis"], op["count"], nt)
+        elif kind == "split":
+            t = split_part(tensors[op["src"]], op["axis"], op["sizes"], op["part"], nt)
         elif kind == "stmts":
             # elements no statement writes stay at a recognisable poison value
             t = np.full(op["shape"], 0xA5, dtype=np.uint8).astype(tensors[0].dtype)

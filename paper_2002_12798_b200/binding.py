@@ -24,7 +24,8 @@ KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
 EXPORTS = [
     "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",
     "amap_builder_transpose", "amap_builder_slice", "amap_builder_concat", "amap_builder_pad",
-    "amap_builder_window", "amap_builder_tile", "amap_builder_tensor", "amap_builder_stmt",
+    "amap_builder_window", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
+    "amap_builder_stmt",
     "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
@@ -169,6 +170,16 @@ class Builder:
     def tile(self, src, reps):
         o = c_int32()
         return self._out(_lib.amap_builder_tile(self._h, src, len(reps), _i64(reps), byref(o)), "amap_builder_tile", o)
+
+    def repeat(self, src, axis, count):
+        out = c_int32()
+        return self._out(_lib.amap_builder_repeat(self._h, src, int(axis), c_int64(int(count)), byref(out)), "amap_builder_repeat", out)
+
+    def split(self, src, axis, sizes):
+        """The ids of the parts, in order."""
+        outs = (c_int32 * len(sizes))()
+        _check(_lib.amap_builder_split(self._h, src, int(axis), len(sizes), _i64(sizes), outs), "amap_builder_split")
+        return list(outs)
 
     def stmt(self, bounds, load, store, guarded=False, fill_bits=0):
         """One raw statement.  load = None | (tensor, C rows, b); store = (tensor, C rows, b)."""
@@ -372,6 +383,10 @@ def build_chain(chain) -> tuple:
             t = b.window(ids[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"])
         elif k == "tile":
             t = b.tile(ids[op["src"]], op["reps"])
+        elif k == "repeat":
+            t = b.repeat(ids[op["src"]], op["axis"], op["count"])
+        elif k == "split":
+            t = b.split(ids[op["src"]], op["axis"], op["sizes"])[op["part"]]
         elif k == "stmts":
             t = b.tensor(op["shape"])
             for st in op["stmts"]:

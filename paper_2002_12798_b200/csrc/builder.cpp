@@ -367,6 +367,68 @@ extern "C" int amap_builder_tile(amap_builder *b, int32_t src, int32_t rank, con
   return AMAP_OK;
 }
 
+extern "C" int amap_builder_repeat(amap_builder *b, int32_t src, int32_t axis, int64_t count, int32_t *out) {
+  GUARD_BUILDER(b, out);
+  if (!b->valid(src) || count < 1) return AMAP_EINVAL;
+  const std::vector<int64_t> in = b->shapes[src];
+  const int rank = (int)in.size();
+  if (axis < 0 || axis >= rank || rank + 1 > AMAP_MAX_LOOPS) return AMAP_EINVAL;
+  std::vector<int64_t> ou = in;
+  ou[axis] = count * in[axis];
+  StmtRec r;  // loops (i_0, ..., i_axis, j, ..., i_{rank-1}): the load ignores the copy loop j
+  const int n = rank + 1;
+  r.lC.assign((size_t)rank * n, 0);
+  r.sC.assign((size_t)rank * n, 0);
+  for (int d = 0; d < rank; ++d) {
+    const int k = d <= axis ? d : d + 1;  // loop of i_d
+    r.lC[(size_t)d * n + k] = 1;
+    r.sC[(size_t)d * n + k] = d == axis ? count : 1;
+  }
+  r.sC[(size_t)axis * n + axis + 1] = 1;
+  for (int k = 0; k < n; ++k) r.bounds.push_back(k == axis + 1 ? count : in[k <= axis ? k : k - 1]);
+  r.lb.assign(rank, 0);
+  r.sb.assign(rank, 0);
+  r.load_tensor = src;
+  r.load_rank = r.store_rank = rank;
+  r.store_tensor = b->add_tensor(ou);
+  *out = r.store_tensor;
+  b->stmts.push_back(std::move(r));
+  return AMAP_OK;
+}
+
+extern "C" int amap_builder_split(amap_builder *b, int32_t src, int32_t axis, int32_t n_parts, const int64_t *sizes,
+                                  int32_t *outs) {
+  GUARD_BUILDER(b, outs);
+  if (!b->valid(src) || !sizes || n_parts < 1) return AMAP_EINVAL;
+  const std::vector<int64_t> in = b->shapes[src];
+  const int rank = (int)in.size();
+  if (axis < 0 || axis >= rank) return AMAP_EINVAL;
+  int64_t total = 0;
+  for (int q = 0; q < n_parts; ++q) {
+    if (sizes[q] < 0) return AMAP_EINVAL;
+    total += sizes[q];
+  }
+  if (total != in[axis]) return AMAP_EINVAL;
+  int64_t off = 0;
+  for (int q = 0; q < n_parts; ++q) {  // one statement and one tensor per part, loops = the part's own index
+    StmtRec r;
+    r.bounds = in;
+    r.bounds[axis] = sizes[q];
+    r.lC = identity_rows(rank, rank);
+    r.lb.assign(rank, 0);
+    r.lb[axis] = off;
+    off += sizes[q];
+    r.sC = identity_rows(rank, rank);
+    r.sb.assign(rank, 0);
+    r.load_tensor = src;
+    r.load_rank = r.store_rank = rank;
+    r.store_tensor = b->add_tensor(r.bounds);
+    outs[q] = r.store_tensor;
+    b->stmts.push_back(std::move(r));
+  }
+  return AMAP_OK;
+}
+
 extern "C" int amap_builder_chain(amap_builder *b, int32_t output, const amap_chain **out) {
   GUARD_BUILDER(b, out);
   if (!b->valid(output)) return AMAP_EINVAL;

@@ -18,6 +18,9 @@ Chain format
   {"kind": "concat",    "srcs": [t0, t1, ...], "axis": a}
   {"kind": "pad",       "src": t, "lo": [...], "hi": [...]}          zero fill
   {"kind": "window",    "src": t, "kh":, "kw":, "stride":, "pad":}   NHWC im2col, column order (r, s, c)
+  {"kind": "tile",      "src": t, "reps": [...]}                     the whole tensor reps[d] times along axis d
+  {"kind": "repeat",    "src": t, "axis": a, "count": c}             every element c times in a row along axis a
+  {"kind": "split",     "src": t, "axis": a, "sizes": [...], "part": k}   part k of t cut along axis a
   {"kind": "stmts",     "shape": [...], "stmts": [ {...}, ... ]}     raw load/store pairs in the paper's form:
         {"bounds": [...], "load": None | (tensor, C rows, b), "store": (C rows, b),
          "guarded": bool, "fill": int}
@@ -233,6 +236,39 @@ def c5_im2col(N=64, H=56, W=56, C=128, k=3, stride=1, pad=1, dtype="fp16") -> Ch
         ops=[{"kind": "window", "src": 0, "kh": k, "kw": k, "stride": stride, "pad": pad}],
         values="uniform_pm1",
         seed=BASE_SEED + 5,
+    )
+
+
+def upsample_nhwc(N=32, H=56, W=56, C=256, factor=2, dtype="fp16") -> Chain:
+    """Nearest-neighbour upsampling of NHWC activations: every pixel `factor` times along H and along W."""
+    return Chain(
+        name="upsample_nhwc",
+        dtype=dtype,
+        inputs=[[N, H, W, C]],
+        ops=[
+            {"kind": "repeat", "src": 0, "axis": 1, "count": factor},
+            {"kind": "repeat", "src": 1, "axis": 2, "count": factor},
+        ],
+        values="uniform_pm1",
+        seed=BASE_SEED + 6,
+    )
+
+
+def qkv_split(B=16, S=2048, heads=32, D=128, part=0, dtype="bf16") -> Chain:
+    """The output [B,S,3*heads*D] of a fused QKV projection cut into three on the last axis; part `part`
+    reshaped to [B,S,heads,D] and moved to [B,heads,S,D]."""
+    hd = heads * D
+    return Chain(
+        name="qkv_split_%d" % part,
+        dtype=dtype,
+        inputs=[[B, S, 3 * hd]],
+        ops=[
+            {"kind": "split", "src": 0, "axis": 2, "sizes": [hd, hd, hd], "part": part},
+            {"kind": "reshape", "src": 1, "shape": [B, S, heads, D]},
+            {"kind": "transpose", "src": 2, "perm": [0, 2, 1, 3]},
+        ],
+        values="normal",
+        seed=BASE_SEED + 7,
     )
 
 

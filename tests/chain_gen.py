@@ -12,7 +12,7 @@ def random_chain(r, n_ops=4, max_extent=5, max_rank=4):
     ops = []
     cur, cur_shape = 0, list(shape)
     for _ in range(n_ops):
-        kind = r.choice(["reshape", "transpose", "slice", "pad", "concat"])
+        kind = r.choice(["reshape", "transpose", "slice", "pad", "concat", "tile", "repeat", "split"])
         tid = len(inputs) + len(ops)
         if kind == "reshape":
             n = int(np.prod(cur_shape))
@@ -45,6 +45,25 @@ def random_chain(r, n_ops=4, max_extent=5, max_rank=4):
             hi = [int(r.integers(0, 2)) for _ in cur_shape]
             ops.append({"kind": "pad", "src": cur, "lo": lo, "hi": hi})
             cur_shape = [a + n + b for a, n, b in zip(lo, cur_shape, hi)]
+        elif kind == "tile":
+            reps = [int(r.integers(1, 3)) for _ in cur_shape]
+            ops.append({"kind": "tile", "src": cur, "reps": reps})
+            cur_shape = [a * n for a, n in zip(reps, cur_shape)]
+        elif kind == "repeat":
+            axis = int(r.integers(0, len(cur_shape)))
+            count = int(r.integers(1, 4))
+            ops.append({"kind": "repeat", "src": cur, "axis": axis, "count": count})
+            cur_shape = list(cur_shape)
+            cur_shape[axis] *= count
+        elif kind == "split":
+            axis = int(r.integers(0, len(cur_shape)))
+            n = cur_shape[axis]
+            cut = sorted(int(c) for c in r.integers(0, n + 1, size=2))
+            sizes = [cut[0], cut[1] - cut[0], n - cut[1]]
+            part = int(r.choice([k for k in range(3) if sizes[k] > 0]))
+            ops.append({"kind": "split", "src": cur, "axis": axis, "sizes": sizes, "part": part})
+            cur_shape = list(cur_shape)
+            cur_shape[axis] = sizes[part]
         else:  # concat the current tensor with itself or with the first input when shapes allow
             axis = int(r.integers(0, len(cur_shape)))
             other = cur

@@ -130,6 +130,31 @@ def test_tile_broadcast(B):
     assert np.array_equal(got.reshape(80, 15), np.tile(xs[0], (5, 2)).T)
 
 
+def test_repeat_upsamples(B):
+    """Nearest-neighbour 2x upsampling of NHWC activations: repeat on H, then on W, one composed copy."""
+    chain = W.upsample_nhwc(N=2, H=9, W=7, C=40, factor=2)
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    for force in (0, 1):
+        got, plan = run_gpu(B, chain, xs, force=force)
+        assert plan.stats()["n_stages"] == 1
+        assert np.array_equal(got, want.reshape(-1))
+    assert np.array_equal(want, np.repeat(np.repeat(xs[0], 2, axis=1), 2, axis=2))
+
+
+def test_split_parts_each_compose_to_one_copy(B):
+    """A fused QKV projection output cut into q, k, v, each moved to [B, heads, S, D]: one plan per part."""
+    for part in range(3):
+        chain = W.qkv_split(B=2, S=24, heads=3, D=16, part=part)
+        xs = W.make_inputs(chain)
+        want = oracle.run_chain(chain, xs)
+        got, plan = run_gpu(B, chain, xs)
+        assert plan.stats()["n_stages"] == 1 and plan.stats()["n_launches"] == 1
+        assert np.array_equal(got, want.reshape(-1))
+        x = xs[0].reshape(2, 24, 3, 3, 16)  # [B, S, part, heads, D]
+        assert np.array_equal(want, x[:, :, part].transpose(0, 2, 1, 3))
+
+
 def test_random_statement_chains(B):
     """Raw load/store statements with arbitrary small affine maps (interleaved and merged stores, guards,
     temporaries where a pair cannot be eliminated)."""

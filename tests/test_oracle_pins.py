@@ -292,6 +292,74 @@ def test_operator_families_as_load_store_pairs():
 
 
 # ---------------------------------------------------------------------------
+# tile, repeat, split (the broadcast and cutting operators Section 2.1 names)
+# ---------------------------------------------------------------------------
+def test_tile_matches_numpy_and_counts_every_element():
+    x = rand_u((3, 4, 5))
+    reps = [2, 1, 3]
+    y = oracle.tile(x, reps)
+    assert y.shape == (6, 4, 15)
+    assert np.array_equal(y, np.tile(x, reps))
+    # each copy, cut back out by slicing, is the input; every value appears prod(reps) times as often
+    for r0 in range(2):
+        for r2 in range(3):
+            part = oracle.slice_(y, [3 * r0, 0, 5 * r2], [3 * r0 + 3, 4, 5 * r2 + 5], [1, 1, 1])
+            assert np.array_equal(part, x)
+    vals, counts = np.unique(x, return_counts=True)
+    vals_y, counts_y = np.unique(y, return_counts=True)
+    assert np.array_equal(vals, vals_y) and np.array_equal(counts_y, 6 * counts)
+    assert np.array_equal(oracle.tile(x, [1, 1, 1]), x)
+    with pytest.raises(ValueError):
+        oracle.tile(x, [1, 0, 1])
+
+
+def test_repeat_matches_numpy_and_differs_from_tile():
+    x = rand_u((3, 4, 5))
+    for axis, count in ((0, 2), (1, 3), (2, 4)):
+        y = oracle.repeat(x, axis, count)
+        assert np.array_equal(y, np.repeat(x, count, axis=axis))
+        # picking every count-th element along the axis, from any phase, gives the input back
+        for phase in range(count):
+            start = [0, 0, 0]
+            start[axis] = phase
+            assert np.array_equal(oracle.slice_(y, start, list(y.shape), [count if d == axis else 1 for d in range(3)]), x)
+    # on the flat index of a rank-1 tensor: out[k] = in[k div count], not in[k mod n]
+    v = np.arange(1, 6, dtype=np.uint16)
+    assert oracle.repeat(v, 0, 3).tolist() == [1, 1, 1, 2, 2, 2, 3, 3, 3, 4, 4, 4, 5, 5, 5]
+    assert oracle.tile(v, [3]).tolist() == [1, 2, 3, 4, 5] * 3
+    assert np.array_equal(oracle.repeat(x, 1, 1), x)
+
+
+def test_split_parts_match_numpy_and_join_back():
+    x = rand_u((4, 9, 3))
+    sizes = [2, 0, 3, 4]
+    parts = [oracle.split_part(x, 1, sizes, k) for k in range(4)]
+    want = np.split(x, np.cumsum(sizes)[:-1], axis=1)
+    for got, w in zip(parts, want):
+        assert got.shape == w.shape and np.array_equal(got, w)
+    assert np.array_equal(oracle.concat(parts, 1), x)  # concat is the inverse of split
+    with pytest.raises(ValueError):
+        oracle.split_part(x, 1, [2, 3], 0)  # sizes do not add up to the extent
+
+
+def test_broadcast_and_split_as_load_store_pairs():
+    """tile, repeat and split written in the paper's form agree with the operators' own loop nests."""
+    x = rand_u((3, 4), np.uint32)
+    # tile(2, 3): loops (r0, i0, r1, i1); the load ignores the repetition loops
+    y = np.zeros((6, 12), np.uint32)
+    oracle.affine_stmt(y, [2, 3, 3, 4], (x, [[0, 1, 0, 0], [0, 0, 0, 1]], [0, 0]), ([[3, 1, 0, 0], [0, 0, 4, 1]], [0, 0]))
+    assert np.array_equal(y, oracle.tile(x, [2, 3]))
+    # repeat(axis 1, 3): loops (i0, i1, j)
+    y = np.zeros((3, 12), np.uint32)
+    oracle.affine_stmt(y, [3, 4, 3], (x, [[1, 0, 0], [0, 1, 0]], [0, 0]), ([[1, 0, 0], [0, 3, 1]], [0, 0]))
+    assert np.array_equal(y, oracle.repeat(x, 1, 3))
+    # split(axis 1, [1, 3]) part 1: loops = part index, load offset 1
+    y = np.zeros((3, 3), np.uint32)
+    oracle.affine_stmt(y, [3, 3], (x, [[1, 0], [0, 1]], [0, 1]), ([[1, 0], [0, 1]], [0, 0]))
+    assert np.array_equal(y, oracle.split_part(x, 1, [1, 3], 1))
+
+
+# ---------------------------------------------------------------------------
 # brute force on tiny random chains
 # ---------------------------------------------------------------------------
 def _python_chain(chain, inputs):
@@ -308,6 +376,12 @@ def _python_chain(chain, inputs):
             t = np.concatenate([ts[s] for s in op["srcs"]], op["axis"])
         elif k == "pad":
             t = np.pad(ts[op["src"]], list(zip(op["lo"], op["hi"])))
+        elif k == "tile":
+            t = np.tile(ts[op["src"]], op["reps"])
+        elif k == "repeat":
+            t = np.repeat(ts[op["src"]], op["count"], axis=op["axis"])
+        elif k == "split":
+            t = np.split(ts[op["src"]], np.cumsum(op["sizes"])[:-1], axis=op["axis"])[op["part"]]
         ts.append(np.ascontiguousarray(t))
     return ts[-1]
 
