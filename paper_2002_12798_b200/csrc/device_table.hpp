@@ -75,7 +75,7 @@ struct DevPiece {
   int32_t ku_coef[kDevMaxCons];
   // --- transpose kernel only -------------------------------------------
   int32_t tr_unit;            // bytes per global access: 16, or less for pieces aligned to less; 0: shifted rows, -1: realigned source rows
-  int32_t tile_ca;            // 16-byte kernel: 16-byte chunks of a per tile, 8 (by 128 elements of b) or 4 (by 256)
+  int32_t tile_ca;            // 16-byte kernel: 16-byte chunks of a per tile: 8 (by 128 elements of b), 4 (by 256), 16 (by 64), 32 (by 32)
   int64_t src_bytes;          // size of the source tensor (shifted-row kernel: guards the last aligned chunk)
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b

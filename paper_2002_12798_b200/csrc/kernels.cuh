@@ -256,12 +256,18 @@ __device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &p
 // bank-conflict-free.  Tiles on the ragged edge are predicated per chunk (the
 // planner only selects this kernel when both extents are multiples of 16/ES).
 // ---------------------------------------------------------------------------
+// the 16-byte chunk index within a tile row is XOR-ed with this function of the row's chunk of a
+template <int CA>
+__device__ __forceinline__ int tile_swizzle(int ca) {
+  return CA >= 8 ? (ca & 7) : ca * (8 / CA);
+}
+
 template <int ES, int CA = 8>
 __device__ __forceinline__ uint4 gather_column(const unsigned char *tile, int ca, int b_l) {
   constexpr int EPU = 16 / ES;
-  constexpr int RB = kTileB * ES * (8 / CA);
+  constexpr int RB = kTileB * ES * 8 / CA;
   const int chunk = b_l / EPU;
-  const unsigned char *p = tile + (ca * EPU) * RB + ((chunk ^ (ca * (8 / CA))) << 4) + (b_l % EPU) * ES;
+  const unsigned char *p = tile + (ca * EPU) * RB + ((chunk ^ tile_swizzle<CA>(ca)) << 4) + (b_l % EPU) * ES;
   uint4 out;
   if constexpr (ES == 1) {
     uint32_t w[4];
@@ -333,19 +339,36 @@ __device__ __forceinline__ void fill_block(const DevPiece &sp, char *dst) {
   }
 }
 
-// CA = 16-byte chunks of a per tile: 8 (128 bytes of a by 128 elements of b) or 4 (64 bytes of a by 256 elements
-// of b, for pieces or remainders at most 64 bytes long in a, which would leave the wide tile half empty).  The
-// planner may shorten the step along b (sp.step_b) so that the tiles of a row are evenly filled.
+// CA = 16-byte chunks of a per tile; the tile always holds 1024 chunks:
+//    8   128 bytes of a by 128 elements of b, the general shape;
+//    4   64 bytes of a by 256 elements of b, for pieces or remainders at most 64 bytes long in a;
+//   16   256 bytes of a by 64 elements of b, and
+//   32   512 bytes of a by 32 elements of b, for pieces that short in b (NHWC -> NCHW with 64 or 32 channels);
+//        rows must stay at least 128 bytes long for the swizzle, so 16 needs ES >= 2 and 32 needs ES >= 4.
+// Either way a short extent no longer leaves the tile half empty.  The planner may also shorten the step along b
+// (sp.step_b) so that the tiles of a row are evenly filled.
 template <int ES, typename OffT, int CA>
 __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTable &ptrs, unsigned char *tile) {
   constexpr int EPU = 16 / ES;     // elements per 16-byte chunk
   constexpr int TA = CA * EPU;     // rows of the tile
-  constexpr int TB = kTileB * (8 / CA);  // elements of b a tile can hold
+  constexpr int TB = kTileB * 8 / CA;    // elements of b a tile can hold
   constexpr int RB = TB * ES;      // bytes per row
   constexpr int CB = RB / 16;      // chunks per row
-  constexpr int SW = 8 / CA;       // swizzle step: chunk index XOR (a / EPU) * SW
+  constexpr int G = CA >= 8 ? CA / 8 : 1;  // phase 2 walks a in groups of 8 chunks (one 128-byte line per row of lanes)
   constexpr int U = TA * CB / kTransposeThreads;
-  static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB, "tile geometry");
+  static_assert(TA * RB == kTileBytes && U * kTransposeThreads == TA * CB && RB >= 128, "tile geometry");
+  // phase 2: which chunk of a and which b (ES == 2: which pair of b) work item idx takes.  The 8 lanes that share a
+  // b take 8 consecutive chunks of a (a full line of the destination), the 4 groups of 8 lanes 4 consecutive b.
+  auto phase2_item = [](int idx, int *ca, int *bq) {
+    if constexpr (CA >= 8) {
+      const int lane = idx & 31, w = idx >> 5;
+      *ca = (lane & 7) + 8 * (w % G);
+      *bq = (lane >> 3) + 4 * (w / G);
+    } else {
+      *ca = idx % CA;
+      *bq = idx / CA;
+    }
+  };
 
   const uint32_t step_b = sp.step_b;
   uint32_t t = blockIdx.x - sp.first_block;
@@ -431,7 +454,7 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
       const int a_l = idx / CB, cb = idx % CB;
-      *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ (((a_l / EPU) * SW) & 7)) << 4)) = v[u];
+      *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ tile_swizzle<CA>(a_l / EPU)) << 4)) = v[u];
     }
   }
   __syncthreads();
@@ -454,10 +477,12 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
 #pragma unroll
     for (int u = 0; u < U / 2; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx % CA, b_l = (idx / CA) * 2;
+      int ca, b_l;
+      phase2_item(idx, &ca, &b_l);
+      b_l *= 2;
       const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
       if (a < ext_a && b < end_b) {  // extents and steps are even: b + 1 is inside too
-        const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ (ca * SW)) << 4) + (b_l % EPU) * ES;
+        const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ tile_swizzle<CA>(ca)) << 4) + (b_l % EPU) * ES;
         uint32_t r[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * RB);
@@ -474,7 +499,8 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx % CA, b_l = idx / CA;
+      int ca, b_l;
+      phase2_item(idx, &ca, &b_l);
       const uint32_t a = a0 + ca * EPU, b = b0 + b_l;
       if (a < ext_a && b < end_b) __stcs(reinterpret_cast<uint4 *>(dst_of(a, b)), gather_column<ES, CA>(tile, ca, b_l));
     }
@@ -489,8 +515,23 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
     fill_block(sp, ptrs.dst);
     return;
   }
-  if (sp.tile_ca == 4) transpose_tile<ES, OffT, 4>(sp, ptrs, tile);
-  else transpose_tile<ES, OffT, 8>(sp, ptrs, tile);
+  if (sp.tile_ca == 4) {
+    transpose_tile<ES, OffT, 4>(sp, ptrs, tile);
+    return;
+  }
+  if constexpr (ES >= 2) {
+    if (sp.tile_ca == 16) {
+      transpose_tile<ES, OffT, 16>(sp, ptrs, tile);
+      return;
+    }
+  }
+  if constexpr (ES >= 4) {
+    if (sp.tile_ca == 32) {
+      transpose_tile<ES, OffT, 32>(sp, ptrs, tile);
+      return;
+    }
+  }
+  transpose_tile<ES, OffT, 8>(sp, ptrs, tile);
 }
 
 // ---------------------------------------------------------------------------

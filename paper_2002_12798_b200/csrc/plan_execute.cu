@@ -324,12 +324,12 @@ static bool check_affine_piece(const DevPiece &d, int64_t in_bytes, int64_t out_
 // strides in a padded NHWC destination).
 // ---------------------------------------------------------------------------
 // Tile counts of a transpose descriptor whose extents and batch loops are set: tiles of `ca` 16-byte chunks of a
-// by up to kTileB * 8 / ca elements of b.  With `even` the step along b is shortened to the smallest multiple of
+// by up to kTileB * 8 / ca elements of b (1024 chunks either way).  With `even` the step along b is shortened to the smallest multiple of
 // a chunk that still covers ext_b with the same number of tiles, so that no tile is left nearly empty
 // (784 = 7 x 112 instead of 6 x 128 + 16).
 static bool set_transpose_tiles(DevPiece *d, int ca, bool even) {
   const int es = d->unit_bytes, epu = 16 / es;
-  const uint32_t ta = (uint32_t)(ca * epu), tb = (uint32_t)(kTileB * (8 / ca));
+  const uint32_t ta = (uint32_t)(ca * epu), tb = (uint32_t)(kTileB * 8 / ca);
   d->tile_ca = ca;
   d->tiles_a = (d->ext_a + ta - 1) / ta;
   d->tiles_b = (d->ext_b + tb - 1) / tb;
@@ -420,8 +420,15 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     }
     if (!aligned) return false;
     d->n_loops = j;
-    // the 16-byte kernel takes the narrow tile (4 chunks of a) for pieces at most that long in a
-    return set_transpose_tiles(d, (ub == 16 && ext_a <= 4 * (16 / es)) ? 4 : 8, ub == 16);
+    // the 16-byte kernel has tile shapes for pieces that are short in a (4 chunks of a by 256 elements of b) or in
+    // b (16 chunks by 64 elements, 32 chunks by 32 elements; their rows must stay 128 bytes long)
+    int ca = 8;
+    if (ub == 16) {
+      if (ext_a <= 4 * (16 / es)) ca = 4;
+      else if (ext_b <= 32 && es >= 4) ca = 32;
+      else if (ext_b <= 64 && es >= 2) ca = 16;
+    }
+    return set_transpose_tiles(d, ca, ub == 16);
   };
   // units of a single element gain nothing over the strip kernel's gather (measured): at least two per access
   for (int ub = 16; ub >= 2 * es; ub >>= 1) {
@@ -547,8 +554,9 @@ static bool check_realign_block(const DevPiece &d, uint32_t blk, int64_t in_byte
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   if (d.tr_unit < 0) return check_realign_block(d, blk, in_bytes, out_bytes);
-  const int es = d.unit_bytes, epu = 16 / es, ca = d.tile_ca, ta = ca * epu, sw = 8 / ca;
-  if ((ca != 8 && !(ca == 4 && d.tr_unit == 16)) || d.step_b == 0 || d.step_b % epu || d.step_b > (uint32_t)(kTileB * sw) ||
+  const int es = d.unit_bytes, epu = 16 / es, ca = d.tile_ca, ta = ca * epu;
+  const bool shape_ok = ca == 8 || (d.tr_unit == 16 && (ca == 4 || (ca == 16 && es >= 2) || (ca == 32 && es >= 4)));
+  if (!shape_ok || d.step_b == 0 || d.step_b % epu || d.step_b > (uint32_t)(kTileB * 8 / ca) ||
       (uint64_t)d.tiles_b * d.step_b < d.ext_b || (uint64_t)d.tiles_a * ta < d.ext_a)
     return false;
   uint32_t t = blk;
@@ -571,8 +579,11 @@ static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_by
     dbase += (int64_t)i * d.dstride[k];
   }
   if (t != 0) return false;
-  const int ub = d.tr_unit, epn = ub / es, rb = kTileB * sw * es, cbu = rb / ub, nca = ta / epn;
-  auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ (((row / epu) * sw) & 7)) << 4) | (col & 15)); };
+  const int ub = d.tr_unit, epn = ub / es, rb = kTileB * 8 / ca * es, cbu = rb / ub, nca = ta / epn;
+  auto swizzle = [&](int chunk_a) { return ca >= 8 ? (chunk_a & 7) : chunk_a * (8 / ca); };
+  auto tile_off = [&](int row, int col) { return row * rb + ((((col >> 4) ^ swizzle(row / epu)) << 4) | (col & 15)); };
+  // phase 2 below visits the kernel's (chunk of a, b) pairs in plain order; the kernel deals the same pairs out to
+  // its lanes in another order
   for (int idx = 0; idx < kTileBytes / ub; ++idx) {
     {  // phase 1
       const int a_l = idx / cbu, cu = idx % cbu;

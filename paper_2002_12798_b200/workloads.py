@@ -317,6 +317,13 @@ def reduced_configs() -> dict:
         "c2_fwd_rem_u64": c2_nchw_to_nhwc(N=2, C=20, H=10, W=53, dtype="u64"),
         "c2_fwd_short": c2_nchw_to_nhwc(N=2, C=24, H=20, W=26),
         "c2_inv_rem": c2_nhwc_to_nchw(N=2, C=280, H=8, W=12),
+        # 16-byte transposes that are short along the source run (64 or 32 channels in NHWC): wide, flat tiles
+        "c2_inv_c64": c2_nhwc_to_nchw(N=2, C=64, H=24, W=20),
+        "c2_inv_c48": c2_nhwc_to_nchw(N=2, C=48, H=24, W=20),
+        "c2_inv_c32_f32": c2_nhwc_to_nchw(N=2, C=32, H=12, W=23, dtype="fp32"),
+        "c2_inv_c64_f32": c2_nhwc_to_nchw(N=2, C=64, H=12, W=23, dtype="fp32"),
+        "c2_inv_c24_u64": c2_nhwc_to_nchw(N=2, C=24, H=10, W=27, dtype="u64"),
+        "c2_fwd_hw64": c2_nchw_to_nhwc(N=2, C=200, H=8, W=8),
         "c3": c3_head_split(B=2, S=80, heads=3, D=128, keep=50),
         "c3_odd": c3_head_split(B=2, S=33, heads=5, D=24, keep=17),
         "c3_merge": c3_head_merge(B=2, S=70, heads=3, D=128),
