@@ -121,7 +121,7 @@ class Builder:
         self.elem_size = elem_size
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:  # module globals are gone at interpreter shutdown
             _lib.amap_builder_destroy(self._h)
             self._h = None
 
@@ -230,7 +230,7 @@ class Map:
         self.elem_size = es.value
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:  # module globals are gone at interpreter shutdown
             _lib.amap_map_destroy(self._h)
             self._h = None
 
@@ -290,7 +290,7 @@ class Plan:
         self.map = amap
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:  # module globals are gone at interpreter shutdown
             _lib.amap_plan_destroy(self._h)
             self._h = None
 
