@@ -80,7 +80,7 @@ struct DevPiece {
   uint32_t ext_a, ext_b;      // merged extents, in elements
   uint32_t tiles_a, tiles_b;  // tiles along a / b
   uint32_t step_b;            // 16-byte kernel: elements of b between tiles (at most what a tile holds)
-  uint32_t pad1_;
+  uint32_t shift_wrap;        // shifted-row kernel: 1 when destination row b + 1 starts where row b ends
   FastDiv fd_tiles_a, fd_tiles_b;
   FastDiv fd_a_in, fd_b_in;  // inner extents of the merged indices
   int64_t sa[2];             // source byte strides of (a_lo, a_hi)

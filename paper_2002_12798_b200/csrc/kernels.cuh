@@ -626,24 +626,36 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
 // ---------------------------------------------------------------------------
 // The tiled transpose for pieces whose DESTINATION rows are not 16-byte aligned
 // but whose source rows are (NHWC -> NCHW with an odd H*W).  Phase 1 is the
-// aligned kernel's.  In phase 2 the eight lanes that share a destination row b
-// each gather their 16 bytes of the tile's run (a0 + 8ca ...), then build the
-// ALIGNED 16-byte slot of the destination that starts inside their predecessor's
-// bytes: the last s bytes of lane ca-1's vector and the first 16-s of their own
-// (s = destination address mod 16; one shuffle per word, a word select and a
-// funnel shift).  Slots that are not wholly inside the tile's run -- the first
-// and, through lane 7, a ninth one, and whatever crosses the end of the row --
-// are stored element by element; the neighbouring tile writes their other part.
+// aligned kernel's, over a taller tile.  Phase 2 works on the destination's
+// own 16-byte grid: in row b the aligned slots start at the elements
+// a = head + k * EPU, head = the elements from the row's start to the next
+// 16-byte boundary, and the tile at a0 owns the eight slots that START inside
+// [a0, a0 + TA).  A slot that starts near the end of that range needs up to
+// EPU - 1 source rows beyond it, so the tile loads TA + EPU rows.  A slot that
+// straddles the END of row b continues with the first elements of row b + 1
+// when the rows follow each other in memory; those come from EPU more "wrap"
+// rows (source rows 0 .. EPU-1), which a tile that can hold a row's end loads
+// as well, and from column b + 1.  Every store is then a whole aligned 16-byte
+// slot, except where the neighbour column is not in the tile: the last column
+// of a tile stores its part of the straddling slot element by element, and the
+// tile at a0 = 0 does the same for the head of its first column (both do it for
+// every column when the rows do not follow each other).
 // ---------------------------------------------------------------------------
 template <int ES>
 __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const PtrTable &ptrs) {
   constexpr int EPU = 16 / ES;
-  constexpr int TA = 8 * EPU;
-  constexpr int RB = kTileB * ES;
+  constexpr int TA = 8 * EPU;            // slot starts a tile owns: a0 .. a0 + TA - 1
+  constexpr int ROWS = TA + 2 * EPU;     // + EPU rows beyond that range + EPU wrap rows
+  constexpr int RB = kTileB * ES;        // bytes per shared-memory row
   constexpr int CB = RB / 16;
-  constexpr int U = TA * CB / kTransposeThreads;
+  constexpr int U = ROWS * CB / kTransposeThreads;
+  static_assert(U * kTransposeThreads == ROWS * CB, "tile geometry");
   using E = typename Unit<ES>::T;
-  __shared__ __align__(128) unsigned char tile[kTileBytes];
+  union Slot {
+    uint4 vec;
+    E e[EPU];
+  };
+  __shared__ __align__(128) unsigned char tile[ROWS * RB];
 
   uint32_t t = blockIdx.x - sp.first_block;
   uint32_t q = fast_div(t, sp.fd_tiles_b);
@@ -662,20 +674,23 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
   }
   const char *src = ptrs.src[sp.input] + sbase;
   char *dst = ptrs.dst;  // dbase stays a byte offset: the slots are aligned relative to the tensor's start
-  const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
+  const uint32_t ext_a = sp.ext_a;
+  const uint32_t end_b = min(sp.ext_b, b0 + kTileB);
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
-  const int na = (int)min((uint32_t)TA, ext_a - a0);  // rows of the tile that exist
+  const bool holds_row_end = a0 + TA + EPU > ext_a;  // this tile may own the slot that straddles the end of a row
+  const bool rows_follow = sp.shift_wrap != 0;       // row b + 1 starts where row b ends
   pdl_wait();
 
-  // phase 1: as in the aligned kernel (rows past the end of a stay unwritten and are never stored)
+  // phase 1: rows [a0, a0 + TA + EPU) of the source, then (wrap) rows [0, EPU); 16-byte chunks along b
   uint4 v[U];
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     const int idx = threadIdx.x + u * kTransposeThreads;
-    const int a_l = idx / CB, cb = idx % CB;
-    const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
+    const int r = idx / CB, cb = idx % CB;
+    const uint32_t a = r < TA + EPU ? a0 + r : (uint32_t)(r - (TA + EPU)), b = b0 + cb * EPU;
+    const bool wanted = r < TA + EPU ? a < ext_a : (holds_row_end && rows_follow && a < ext_a);
     v[u] = make_uint4(0, 0, 0, 0);
-    if (a < ext_a && b < ext_b) {
+    if (wanted && b < end_b) {
       const uint32_t a_hi = fast_div(a, fa);
       v[u] = load_16(src + (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)b * ES);
     }
@@ -684,85 +699,95 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     const int idx = threadIdx.x + u * kTransposeThreads;
-    const int a_l = idx / CB, cb = idx % CB;
-    *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+    const int r = idx / CB, cb = idx % CB;
+    *reinterpret_cast<uint4 *>(tile + r * RB + ((cb ^ ((r / EPU) & 7)) << 4)) = v[u];
   }
   __syncthreads();
 
-  // one destination row: lane ca of the row's eight lanes holds run bytes [16 ca, 16 ca + 16) in `own`
-  auto emit_row = [&](uint4 own, int ca, uint32_t b, bool row_ok) {
-    const uint32_t b_hi = fast_div(b, fb);
-    const int64_t D = dbase + (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1] + (int64_t)a0 * ES;
-    const int sh = (int)(D & 15);
-    uint32_t w[9];
-    w[0] = __shfl_up_sync(0xFFFFFFFFu, own.x, 1, 8);
-    w[1] = __shfl_up_sync(0xFFFFFFFFu, own.y, 1, 8);
-    w[2] = __shfl_up_sync(0xFFFFFFFFu, own.z, 1, 8);
-    w[3] = __shfl_up_sync(0xFFFFFFFFu, own.w, 1, 8);
-    w[4] = own.x, w[5] = own.y, w[6] = own.z, w[7] = own.w, w[8] = 0;
-    // slot `s` = run bytes [16 s - sh, 16 s - sh + 16); lane 7 also owns slot 8 (its own tail)
+  auto element = [&](int r, int b_l) -> E {  // tile row r, column b_l
+    const int col = b_l * ES;
+    return *reinterpret_cast<const E *>(tile + r * RB + ((((col >> 4) ^ ((r / EPU) & 7)) << 4) | (col & 15)));
+  };
+  // a slot that straddles the end of its row: elements a .. of column b_l, then rows wrap0 .. of column b_l + 1 if
+  // that column is in the tile (whole store), else only the row's own elements, one by one
+  auto straddling_slot = [&](char *p, uint32_t a, int r, int b_l, int wrap0, bool next_col) {
+    Slot out;
 #pragma unroll
-    for (int pass = 0; pass < 2; ++pass) {
-      const int s = ca + pass;
-      if (pass == 1) {
-        if (ca != 7 || sh == 0) break;
-        w[0] = own.x, w[1] = own.y, w[2] = own.z, w[3] = own.w, w[4] = w[5] = w[6] = w[7] = 0;
-      }
-      const int first = 16 - sh;  // where the slot starts inside the 32-byte window
-      const int o = first >> 2, bits = (first & 3) * 8;
-      // z[i] = w[i + o], o in 0..4, by a three-stage word select (w[8] = 0 pads the window)
-      uint32_t x[8], y[6], z[5];
+    for (int e = 0; e < EPU; ++e) {
+      if (a + e < ext_a) out.e[e] = element(r + e, b_l);
+      else if (next_col) out.e[e] = element(wrap0 + (int)(a + e - ext_a), b_l + 1);
+    }
+    if (next_col) {
+      __stcs(reinterpret_cast<uint4 *>(p), out.vec);
+    } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] = (o & 4) ? (i + 4 <= 8 ? w[i + 4 <= 8 ? i + 4 : 8] : 0u) : w[i];
-#pragma unroll
-      for (int i = 0; i < 6; ++i) y[i] = (o & 2) ? x[i + 2] : x[i];
-#pragma unroll
-      for (int i = 0; i < 5; ++i) z[i] = (o & 1) ? y[i + 1] : y[i];
-      union {
-        uint4 vec;
-        E e[EPU];
-      } out;
-      out.vec.x = __funnelshift_r(z[0], z[1], bits);
-      out.vec.y = __funnelshift_r(z[1], z[2], bits);
-      out.vec.z = __funnelshift_r(z[2], z[3], bits);
-      out.vec.w = __funnelshift_r(z[3], z[4], bits);
-      if (!row_ok) continue;
-      const int rel0 = (16 * s - sh) / ES;  // tile row of the slot's first element (negative for slot 0 when sh > 0)
-      const int64_t A = D - sh + 16 * s;
-      if (rel0 >= 0 && rel0 + EPU <= na) {
-        __stcs(reinterpret_cast<uint4 *>(dst + A), out.vec);
-      } else {
-#pragma unroll
-        for (int e = 0; e < EPU; ++e)
-          if (rel0 + e >= 0 && rel0 + e < na) store_unit<ES>(dst + A + e * ES, out.e[e]);
-      }
+      for (int e = 0; e < EPU; ++e)
+        if (a + e < ext_a) store_unit<ES>(p + e * ES, out.e[e]);
     }
   };
 
-  if constexpr (ES == 2) {
+  // Short rows (a whole row fits the tile, rows follow each other): the tile's destination is ONE contiguous
+  // range, rows b0 .. end_b - 1, and an item is one aligned slot of that range, wherever it falls in a row.
+  if (sp.tiles_a == 1 && rows_follow && fa.d >= ext_a) {
+    const int64_t D0 = dbase + (int64_t)b0 * sp.db[0];  // start of row b0
+    const uint32_t head0 = (uint32_t)((16 - (int)(D0 & 15)) & 15) / ES;
+    const uint32_t n_flat = (end_b - b0) * ext_a;  // elements of the range
+    if (threadIdx.x == 0)  // the elements before the first slot: the tile before this one could not store them
+      for (uint32_t f = 0; f < head0 && f < n_flat; ++f) store_unit<ES>(dst + D0 + (int64_t)f * ES, element((int)f, 0));
+    for (uint32_t f = head0 + threadIdx.x * EPU; f < n_flat; f += kTransposeThreads * EPU) {
+      const uint32_t b_l = fast_div(f, fa), a = f - b_l * ext_a;
+      char *p = dst + D0 + (int64_t)f * ES;
+      if (a + EPU <= ext_a) {
+        // EPU consecutive tile rows from row a on: they cross into the next group of EPU rows (the next swizzle)
+        // after EPU - a % EPU of them
+        const int col = (int)b_l * ES, chunk = col >> 4, g = (int)a / EPU;
+        const unsigned char *base = tile + (int)a * RB + (col & 15);
+        const int off_lo = (chunk ^ (g & 7)) << 4, off_hi = (chunk ^ ((g + 1) & 7)) << 4;
+        const int split = EPU - (int)a % EPU;
+        Slot out;
 #pragma unroll
-    for (int u = 0; u < U / 2; ++u) {
-      const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx & 7, b_l = (idx >> 3) * 2;
-      const uint32_t b = b0 + b_l;
-      const unsigned char *p = tile + (ca * EPU) * RB + (((b_l / EPU) ^ ca) << 4) + (b_l % EPU) * ES;
-      uint32_t r[8];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(p + j * RB);
-      uint4 lo, hi;
-      lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
-      lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
-      lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
-      lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
-      emit_row(lo, ca, b, b < ext_b);
-      emit_row(hi, ca, b + 1, b + 1 < ext_b);
+        for (int e = 0; e < EPU; ++e) out.e[e] = *reinterpret_cast<const E *>(base + e * RB + (e < split ? off_lo : off_hi));
+        __stcs(reinterpret_cast<uint4 *>(p), out.vec);
+      } else {
+        straddling_slot(p, a, (int)a, (int)b_l, 0, b0 + b_l + 1 < end_b);
+      }
     }
-  } else {
+    return;
+  }
+
+  // phase 2: one item = one destination slot: slot k (0..7) of column b_l.  The eight lanes that share a column
+  // take its eight slots (128 contiguous bytes); the four columns of a warp are two apart, so that their
+  // elements sit in different shared-memory words.
+#pragma unroll 2
+  for (int idx = threadIdx.x; idx < 8 * kTileB; idx += kTransposeThreads) {
+    const int k = idx & 7, sel = idx >> 3;
+    const int b_l = ((sel & 3) << 1) + ((sel >> 2) & 1) + ((sel >> 3) << 3);
+    const uint32_t b = b0 + b_l;
+    if (b >= end_b) continue;
+    const uint32_t b_hi = fast_div(b, fb);
+    const int64_t D = dbase + (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1];  // row start
+    const uint32_t head = (uint32_t)((16 - (int)(D & 15)) & 15) / ES;  // elements before the row's first slot
+    // the head of the row belongs to the slot that straddles the end of the row before; this tile stores it
+    // only when that slot's owner cannot (its column is the first of this tile, or rows do not follow each other)
+    if (k == 0 && a0 == 0 && head > 0 && !(rows_follow && b_l > 0)) {
+      for (uint32_t a = 0; a < head && a < ext_a; ++a) store_unit<ES>(dst + D + (int64_t)a * ES, element((int)a, b_l));
+    }
+    const uint32_t a_s = a0 + head + (uint32_t)k * EPU;  // first element of the slot
+    if (a_s >= ext_a) continue;
+    char *p = dst + D + (int64_t)a_s * ES;
+    if (a_s + EPU <= ext_a) {
+      // the slot lies inside the row (nearly all do): EPU consecutive tile rows from row head + k * EPU on, which
+      // cross into the next group of EPU rows (the next swizzle) after EPU - head of them
+      const int col = b_l * ES, chunk = col >> 4;
+      const unsigned char *base = tile + (int)(head + (uint32_t)k * EPU) * RB + (col & 15);
+      const int off_lo = (chunk ^ (k & 7)) << 4, off_hi = (chunk ^ ((k + 1) & 7)) << 4;
+      const int split = EPU - (int)head;
+      Slot out;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int idx = threadIdx.x + u * kTransposeThreads;
-      const int ca = idx & 7, b_l = idx >> 3;
-      emit_row(gather_column<ES>(tile, ca, b_l), ca, b0 + b_l, b0 + b_l < ext_b);
+      for (int e = 0; e < EPU; ++e) out.e[e] = *reinterpret_cast<const E *>(base + e * RB + (e < split ? off_lo : off_hi));
+      __stcs(reinterpret_cast<uint4 *>(p), out.vec);
+    } else {
+      straddling_slot(p, a_s, (int)(a_s - a0), b_l, TA + EPU, rows_follow && b + 1 < end_b);
     }
   }
 }

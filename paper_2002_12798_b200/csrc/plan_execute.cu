@@ -460,16 +460,18 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       }
     }
   }
-  // destination rows misaligned, source rows aligned: the shifted-destination kernel (tr_unit = 0; the aligned
-  // kernel's tile, destination slots realigned in registers)
+  // destination rows misaligned, source rows aligned: the shifted-destination kernel (tr_unit = 0; it stores whole
+  // slots of the destination's own 16-byte grid; rows at least one slot long, so that a slot spans two rows at most)
   if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_b % (16 / es) == 0 && d->soff % 16 == 0 &&
-      d->sa[0] % 16 == 0 && d->sa[1] % 16 == 0) {
+      d->sa[0] % 16 == 0 && d->sa[1] % 16 == 0 && d->ext_a >= (uint32_t)(16 / es)) {
     bool src_aligned = true;
     for (int j = 0; j < d->n_loops; ++j) src_aligned = src_aligned && d->sstride[j] % 16 == 0;
     if (src_aligned) {
       d->tr_unit = 0;
       d->src_bytes = in_bytes;
-      return true;  // tiles and blocks as try_build computed them: 8 chunks of a by kTileB of b
+      // row b + 1 follows row b in memory (b is one loop whose destination stride is the row's length)
+      d->shift_wrap = (d->fd_b_in.d >= d->ext_b && d->db[0] == (int64_t)d->ext_a * es) ? 1 : 0;
+      return true;  // tiles and blocks as try_build computed them: slot starts in 8 chunks of a by kTileB of b
     }
   }
   return false;
@@ -478,7 +480,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
 // the shifted-destination kernel's address arithmetic for one block, replayed on the host
 static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   const int es = d.unit_bytes, epu = 16 / es, ta = 8 * epu;
-  if (d.ext_b % epu) return false;
+  if (d.ext_b % epu || d.ext_a < (uint32_t)epu) return false;
   uint32_t t = blk;
   uint32_t q = t / d.tiles_b;
   const uint32_t b0 = (t - q * d.tiles_b) * kTileB;
@@ -494,22 +496,39 @@ static bool check_shifted_block(const DevPiece &d, uint32_t blk, int64_t in_byte
     t = q;
   }
   if (t != 0 || a0 >= d.ext_a || b0 >= d.ext_b) return false;
-  const int na = (int)std::min<uint32_t>(ta, d.ext_a - a0);
-  for (int a_l = 0; a_l < na; ++a_l)  // aligned 16-byte loads along b
-    for (uint32_t b = b0; b < std::min<uint32_t>(b0 + kTileB, d.ext_b); b += epu) {
-      const uint32_t a = a0 + a_l, a_hi = a / d.fd_a_in.d;
-      const int64_t s = sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
-      if (s % 16 || s < 0 || s + 16 > in_bytes) return false;
-    }
-  for (uint32_t b = b0; b < std::min<uint32_t>(b0 + kTileB, d.ext_b); ++b) {
+  const uint32_t end_b = std::min<uint32_t>(b0 + kTileB, d.ext_b);
+  const bool holds_row_end = a0 + ta + epu > d.ext_a, rows_follow = d.shift_wrap != 0;
+  auto src_ok = [&](uint32_t a, uint32_t b) {  // an aligned 16-byte load of the source
+    const uint32_t a_hi = a / d.fd_a_in.d;
+    const int64_t s = sbase + (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1] + (int64_t)b * es;
+    return s % 16 == 0 && s >= 0 && s + 16 <= in_bytes;
+  };
+  for (int r = 0; r < ta + 2 * epu; ++r) {
+    const uint32_t a = r < ta + epu ? a0 + r : (uint32_t)(r - (ta + epu));
+    const bool wanted = r < ta + epu ? a < d.ext_a : (holds_row_end && rows_follow && a < d.ext_a);
+    for (uint32_t b = b0; wanted && b < end_b; b += epu)
+      if (!src_ok(a, b)) return false;
+  }
+  auto row_start = [&](uint32_t b) {
     const uint32_t b_hi = b / d.fd_b_in.d;
-    const int64_t D = dbase + (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1] + (int64_t)a0 * es;
-    if (D < 0 || D % es || D + (int64_t)na * es > out_bytes) return false;
-    const int sh = (int)(D & 15);
-    for (int s = 0; s <= 8; ++s) {  // every slot: whole ones are aligned and inside, partial ones store valid elements only
-      const int rel0 = (16 * s - sh) / es;
-      const int64_t A = D - sh + 16 * s;
-      if (rel0 >= 0 && rel0 + epu <= na && (A % 16 || A < 0 || A + 16 > out_bytes)) return false;
+    return dbase + (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1];
+  };
+  // the slots of a row are the same whether the kernel walks them row by row or, for short rows, along the flat range
+  for (uint32_t b = b0; b < end_b; ++b) {
+    const int64_t D = row_start(b);
+    if (D < 0 || D % es || D + (int64_t)d.ext_a * es > out_bytes) return false;
+    if (rows_follow && b + 1 < end_b && row_start(b + 1) != D + (int64_t)d.ext_a * es) return false;
+    const uint32_t head = (uint32_t)((16 - (int)(D & 15)) & 15) / es;
+    for (int k = 0; k < 8; ++k) {
+      const uint32_t a_s = a0 + head + (uint32_t)k * epu;
+      if (a_s >= d.ext_a) continue;
+      const bool next_col = rows_follow && b + 1 < end_b;
+      if (a_s + epu > d.ext_a && next_col && !holds_row_end) return false;  // would read wrap rows that were not loaded
+      if (a_s + epu <= d.ext_a || next_col) {  // a whole slot: aligned and inside
+        const int64_t A = D + (int64_t)a_s * es;
+        if (A % 16 || A < 0 || A + 16 > out_bytes) return false;
+      }
+      if (a_s - a0 + epu > (uint32_t)(ta + epu)) return false;  // beyond the rows the tile holds
     }
   }
   return true;

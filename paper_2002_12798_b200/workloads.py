@@ -305,6 +305,19 @@ def reduced_configs() -> dict:
         "c2_inv_odd_big": c2_nhwc_to_nchw(N=2, C=256, H=27, W=27),
         "c2_fwd_odd_big": c2_nchw_to_nhwc(N=2, C=256, H=27, W=27),
         "c2_fwd_odd_gather": c2_nchw_to_nhwc(N=2, C=255, H=27, W=27),
+        # misaligned destination rows: shorter than a tile, just longer than one, of 4- and 1-byte elements, and
+        # with a gap after every row (so that a row does not continue where the one before ends)
+        "c2_inv_7x7": c2_nhwc_to_nchw(N=3, C=136, H=7, W=7),
+        "c2_inv_67": c2_nhwc_to_nchw(N=2, C=40, H=67, W=1),
+        "c2_inv_65": c2_nhwc_to_nchw(N=2, C=24, H=5, W=13),
+        "c2_inv_33_f32": c2_nhwc_to_nchw(N=2, C=20, H=3, W=11, dtype="fp32"),
+        "c2_inv_131_u8": c2_nhwc_to_nchw(N=2, C=48, H=131, W=1, dtype="u8"),
+        "c2_inv_gap": Chain(
+            name="c2_inv_gap", dtype="bf16", inputs=[[2, 5, 25, 48]],
+            ops=[{"kind": "transpose", "src": 0, "perm": [0, 3, 1, 2]},
+                 {"kind": "pad", "src": 1, "lo": [0, 0, 0, 0], "hi": [0, 0, 0, 2]}],
+            values="normal", seed=BASE_SEED + 2,
+        ),
         "c2_fwd_odd_u8": c2_nchw_to_nhwc(N=2, C=64, H=11, W=13, dtype="u8"),
         "c2_fwd_odd_f32b": c2_nchw_to_nhwc(N=2, C=36, H=7, W=9, dtype="fp32"),
         "c2_fwd_narrow": c2_nchw_to_nhwc(N=2, C=72, H=14, W=14),
