@@ -430,14 +430,20 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     }
     return set_transpose_tiles(d, ca, ub == 16);
   };
-  // units of a single element gain nothing over the strip kernel's gather (measured): at least two per access
-  for (int ub = 16; ub >= 2 * es; ub >>= 1) {
-    if (ub > ptr_align) continue;
+  // Accesses of `ub` bytes on both sides.  Units of a single element gain nothing over the strip kernel's gather
+  // (measured): at least two per access.
+  auto try_unit = [&](int ub) -> bool {
+    if (ub > ptr_align || ub < 2 * es) return false;
     if (try_build(ia_hi, ib_hi, ub)) return true;
     if (ib_hi >= 0 && try_build(ia_hi, -1, ub)) return true;
     if (ia_hi >= 0 && try_build(-1, ib_hi, ub)) return true;
     if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1, ub)) return true;
-  }
+    return false;
+  };
+  // Order of preference, as measured on 2-byte elements (TB/s): 16-byte units on both sides 6.5; one side
+  // misaligned: the realigning kernel 4.0-4.5 for the source, 8-byte units 3.4-4.4 or the shifted-destination
+  // kernel 3.2-4.2 for the destination; 4-byte units 2.9.
+  if (try_unit(16)) return true;
   // source rows misaligned, destination rows aligned: the realigning kernel (tr_unit = -1; tile 8 x 14 chunks)
   if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_a % (16 / es) == 0 && d->doff % 16 == 0 &&
       d->db[0] % 16 == 0 && d->db[1] % 16 == 0) {
@@ -460,6 +466,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       }
     }
   }
+  if (try_unit(8)) return true;
   // destination rows misaligned, source rows aligned: the shifted-destination kernel (tr_unit = 0; it stores whole
   // slots of the destination's own 16-byte grid; rows at least one slot long, so that a slot spans two rows at most)
   if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_b % (16 / es) == 0 && d->soff % 16 == 0 &&
@@ -474,6 +481,8 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       return true;  // tiles and blocks as try_build computed them: slot starts in 8 chunks of a by kTileB of b
     }
   }
+  if (try_unit(4)) return true;
+  if (try_unit(2)) return true;
   return false;
 }
 

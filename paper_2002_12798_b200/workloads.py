@@ -322,6 +322,9 @@ def reduced_configs() -> dict:
         "c2_fwd_odd_f32b": c2_nchw_to_nhwc(N=2, C=36, H=7, W=9, dtype="fp32"),
         "c2_fwd_narrow": c2_nchw_to_nhwc(N=2, C=72, H=14, W=14),
         "c2_inv_narrow": c2_nhwc_to_nchw(N=2, C=68, H=14, W=14),
+        # rows aligned to 4 bytes only, on both sides: 4-byte units
+        "c2_fwd_both4": c2_nchw_to_nhwc(N=2, C=70, H=6, W=9),
+        "c2_inv_both4": c2_nhwc_to_nchw(N=2, C=70, H=6, W=9),
         # 16-byte transposes whose extent along the destination run leaves at most half a tile (remainder pieces on
         # the 64-byte tile), or is that short altogether; several tiles along the other index, evenly stepped
         "c2_fwd_rem": c2_nchw_to_nhwc(N=2, C=96, H=20, W=26),
