@@ -390,6 +390,11 @@ def all_configs(torch, B, device, stream, l2, peak, only=None, iters=None, warmu
     # is read once and written four times) and a fused QKV tensor cut in three, each part to [B, heads, S, D]
     # (split: one composed copy per part, three launches over the same input)
     configs["upsample2x"] = W.upsample_nhwc()
+    # layout changes whose rows are not 16-byte aligned on one side (Inception's 35x35x288 maps, ResNet's 14x14x1024):
+    # the realigning, shifted-destination and narrow-unit transpose kernels
+    configs["odd35_fwd"] = W.c2_nchw_to_nhwc(N=64, C=288, H=35, W=35)
+    configs["odd35_inv"] = W.c2_nhwc_to_nchw(N=64, C=288, H=35, W=35)
+    configs["map14_inv"] = W.c2_nhwc_to_nchw(N=64, C=1024, H=14, W=14)
     configs["qkv_split"] = [W.qkv_split(part=k) for k in range(3)]
     for name, chain in configs.items():
         if name == "c1" or (only and name != only):

@@ -266,7 +266,9 @@ int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void 
  * but is not required.  When the outermost loop of the whole map is a batch
  * loop (slab k of the output needs only slab k of every input) the call works
  * slab by slab on two more streams of its own, so that upload, kernel and
- * download overlap; the result is the same. */
+ * download overlap; the result is the same.  The staging memory and the extra
+ * streams belong to the plan: calls on ONE plan must not run at the same time
+ * (amap_execute on the same plan is unaffected). */
 int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------
