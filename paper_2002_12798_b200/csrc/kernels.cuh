@@ -167,10 +167,24 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
   }
   T val[U];
   const T fill = fill_unit<V>(sp);
+  // A contiguous piece (one loop of 16-byte units, a plain copy): the block's source bytes are one range.  While the
+  // kernel before this one on the stream drains, ask L2 for them, and after the loads for the range of the block
+  // that will take this block's place (`prefetch` blocks further on), as the transpose kernel does for its tiles.
+  constexpr uint32_t kBlockBytes = kAffineThreads * U * V;
+  const bool hint = V == 16 && NC == 0 && sp.prefetch && n == 1 && src != nullptr && sp.sstride[0] == V && threadIdx.x < 8;
+  auto prefetch_block = [&](uint64_t block) {
+    const uint64_t first = block * kBlockBytes + threadIdx.x * (kBlockBytes / 8), end = sp.n_items * V;
+    if (first < end) {
+      const uint32_t bytes = (uint32_t)min((uint64_t)(kBlockBytes / 8), end - first);
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src + sp.soff + first), "r"(bytes) : "memory");
+    }
+  };
+  if (hint) prefetch_block(blockIdx.x - sp.first_block);
   pdl_wait();
 #pragma unroll
   for (int u = 0; u < U; ++u) val[u] = load[u] ? load_unit<V>(src + so[u]) : fill;
   issue_barrier();  // every load is issued before the first store
+  if (hint && sp.prefetch > 1) prefetch_block((uint64_t)(blockIdx.x - sp.first_block) + (uint32_t)sp.prefetch);
 #pragma unroll
   for (int u = 0; u < U; ++u)
     if (live[u]) store_unit<V>(dst + doff[u], val[u]);
