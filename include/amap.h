@@ -16,7 +16,8 @@
  *    bytes (1, 2, 4, 8 or 16).  No floating-point arithmetic happens anywhere.
  *  - Every function returns AMAP_OK (0) or a negative amap_status.  Out-handles
  *    are written only on success.  Nothing throws, exits or prints (unless the
- *    environment variable AMAP_LOG is set, which prints composed pieces).
+ *    environment variable AMAP_LOG is set to something other than 0, which
+ *    prints composed pieces and the reason of a failure to stderr).
  *  - Host arrays passed in are read during the call and copied; the caller
  *    keeps ownership.  Handles returned are owned by the library until the
  *    matching *_destroy call.  Device buffers are always the caller's.

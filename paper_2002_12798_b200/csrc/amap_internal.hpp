@@ -6,7 +6,15 @@
 
 #include "amap.h"
 
+#include <cstdlib>
+
 namespace amap {
+
+// AMAP_LOG set to anything but "" or "0": print composed pieces and failures to stderr
+inline bool log_enabled() {
+  const char *v = getenv("AMAP_LOG");
+  return v != nullptr && v[0] != '\0' && !(v[0] == '0' && v[1] == '\0');
+}
 
 // c0 + sum_k c[k] * i_k over a piece's loops
 struct Aff {

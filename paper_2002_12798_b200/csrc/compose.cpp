@@ -734,7 +734,7 @@ extern "C" int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map
     s.code = AMAP_ENOMEM;
   }
   if (!s.ok()) {
-    if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] compose failed: %s\n", s.msg.c_str());
+    if (log_enabled()) fprintf(stderr, "[amap] compose failed: %s\n", s.msg.c_str());
     delete m;
     return s.code;
   }
@@ -745,7 +745,7 @@ extern "C" int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map
     for (auto &g : mm.pieces[q].guards) mm.guard_views[q].push_back({g.e.c.data(), g.e.c0, g.extent});
     for (auto &g : mm.pieces[q].domain) mm.domain_views[q].push_back({g.e.c.data(), g.e.c0, g.extent});
   }
-  if (getenv("AMAP_LOG")) log_map(mm);
+  if (log_enabled()) log_map(mm);
   *out_map = m;
   return AMAP_OK;
 }

@@ -674,7 +674,7 @@ struct PlanCtx {
 };
 
 static int plan_fail(int rc, size_t piece) {
-  if (getenv("AMAP_LOG")) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", piece, rc);
+  if (log_enabled()) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", piece, rc);
   return rc;
 }
 
