@@ -347,4 +347,6 @@ def reduced_configs() -> dict:
         "c4_odd": c4_inception_concat(N=3, channels=(8, 24, 40, 16), H=7, W=9),
         "c5": c5_im2col(N=2, H=14, W=12, C=128),
         "c5_odd": c5_im2col(N=2, H=9, W=7, C=24, k=3, stride=2, pad=1),
+        "c5_5x5": c5_im2col(N=2, H=10, W=9, C=24, k=5, stride=1, pad=2),
+        "c5_5x5_wide": c5_im2col(N=1, H=12, W=11, C=128, k=5, stride=2, pad=2),
     }

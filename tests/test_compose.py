@@ -149,6 +149,17 @@ def test_window_over_a_transposed_input_stays_one_guarded_piece():
     assert np.array_equal(eval_map(m, [xin]), want.reshape(-1))
 
 
+def test_a_5x5_window_is_one_guarded_piece():
+    """A 5x5 window with stride 1 and padding 2 composes to one piece with two guards (as the 3x3 one does)."""
+    b = B.Builder(2)
+    x = b.input([2, 9, 8, 4])
+    m = b.compose(b.window(x, 5, 5, 1, 2))
+    ps = m.pieces()
+    assert len(ps) == 1 and len(ps[0]["guards"]) == 2
+    xin = np.random.default_rng(4).integers(1, 60000, size=(2, 9, 8, 4)).astype(np.uint16)
+    assert np.array_equal(eval_map(m, [xin]), oracle.window(xin, 5, 5, 1, 2).reshape(-1))
+
+
 def test_tile_is_a_broadcast_load():
     b = B.Builder(4)
     x = b.input([2, 3])
