@@ -233,30 +233,18 @@ __device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &p
 #pragma unroll
   for (int u = 0; u < kStrip; ++u) {
     live[u] = (uint32_t)u < left;
-    load[u] = src != nullptr;
-  }
-  if constexpr (NC > 0) {
-    // constraint by constraint (the branches are the same for every thread of the launch): one that does not
-    // depend on the strip's loop (a 3x3 window walked along w: the guard on h) is evaluated once, not per unit
-    const int ng = sp.n_guards, nc = sp.n_guards + sp.n_domain;
+    load[u] = live[u] && (src != nullptr);
+    if constexpr (NC > 0) {
+      const int ng = sp.n_guards, nc = sp.n_guards + sp.n_domain;
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      if (c >= nc) break;
-      const uint32_t extent = (uint32_t)sp.cons[c].extent;
-      const int32_t step = sp.ku_coef[c];
-      bool *flag = c < ng ? load : live;  // a failed guard stores the fill value, a failed domain constraint nothing
-      if (step == 0) {
-        const bool ok = (uint32_t)acc[c] < extent;
-#pragma unroll
-        for (int u = 0; u < kStrip; ++u) flag[u] = flag[u] && ok;
-      } else {
-#pragma unroll
-        for (int u = 0; u < kStrip; ++u) flag[u] = flag[u] && (uint32_t)(acc[c] + u * step) < extent;
+      for (int c = 0; c < NC; ++c) {
+        const bool ok = (c >= nc) || ((uint32_t)(acc[c] + u * sp.ku_coef[c]) < (uint32_t)sp.cons[c].extent);
+        if (c < ng) load[u] = load[u] && ok;
+        else live[u] = live[u] && ok;
       }
+      load[u] = load[u] && live[u];
     }
   }
-#pragma unroll
-  for (int u = 0; u < kStrip; ++u) load[u] = load[u] && live[u];
   T val[kStrip];
   const T fill = fill_unit<V>(sp);
   pdl_wait();
