@@ -160,6 +160,25 @@ def test_a_5x5_window_is_one_guarded_piece():
     assert np.array_equal(eval_map(m, [xin]), oracle.window(xin, 5, 5, 1, 2).reshape(-1))
 
 
+def test_an_intermediate_with_two_readers_is_eliminated_for_both():
+    """A small DAG: one transposed tensor feeds a slice and a pad, whose results are joined again.  The shared
+    intermediate has two readers; each is rewritten against it (Section 2.1, equation (2), per reader)."""
+    b = B.Builder(2)
+    x = b.input([6, 10])
+    t = b.transpose(x, [1, 0])                        # [10, 6], read twice below
+    left = b.slice(t, [0, 0], [10, 4], [1, 2])        # [10, 2]
+    right = b.pad(t, [0, 0], [0, 3])                  # [10, 9]
+    m = b.compose(b.concat([left, right, left], 1))   # [10, 13]
+    assert len(m.stages()) == 1
+    xin = np.random.default_rng(11).integers(1, 60000, size=(6, 10)).astype(np.uint16)
+    tt = xin.T
+    want = np.concatenate([tt[:, 0:4:2], np.pad(tt, [(0, 0), (0, 3)]), tt[:, 0:4:2]], 1)
+    assert np.array_equal(eval_map(m, [xin]), want.reshape(-1))
+    ot = oracle.transpose(xin, [1, 0])
+    ol = oracle.slice_(ot, [0, 0], [10, 4], [1, 2])
+    assert np.array_equal(oracle.concat([ol, oracle.pad(ot, [0, 0], [0, 3]), ol], 1), want)
+
+
 def test_tile_is_a_broadcast_load():
     b = B.Builder(4)
     x = b.input([2, 3])

@@ -155,6 +155,25 @@ def test_split_parts_each_compose_to_one_copy(B):
         assert np.array_equal(want, x[:, :, part].transpose(0, 2, 1, 3))
 
 
+def test_dag_with_a_shared_intermediate(B):
+    """One transposed tensor feeds a slice and a pad that are joined again: two readers of one intermediate."""
+    chain = W.Chain(
+        name="dag", dtype="bf16", inputs=[[48, 200]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},                                           # 1: [200, 48]
+            {"kind": "slice", "src": 1, "start": [0, 0], "stop": [200, 32], "step": [1, 2]},           # 2: [200, 16]
+            {"kind": "pad", "src": 1, "lo": [0, 0], "hi": [0, 16]},                                    # 3: [200, 64]
+            {"kind": "concat", "srcs": [2, 3, 2], "axis": 1},                                          # 4: [200, 96]
+        ],
+        values="normal",
+    )
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, plan = run_gpu(B, chain, xs)
+    assert plan.stats()["n_stages"] == 1
+    assert np.array_equal(got, want.reshape(-1))
+
+
 def test_random_statement_chains(B):
     """Raw load/store statements with arbitrary small affine maps (interleaved and merged stores, guards,
     temporaries where a pair cannot be eliminated)."""
