@@ -171,6 +171,10 @@ typedef struct amap_constraint {
   int64_t extent;
 } amap_constraint;
 
+/* One piece of a composed map: a loop nest in the paper's form (Section 2, equations (load)/(store)) after
+ * Section 2.1's rewrite, i.e. the reader's store with the load g' = f_l o f_s' o f_l' of equation (2) put in its
+ * place.  It differs from amap_stmt only in that both tensors are addressed through their flat views (rank 1,
+ * so C_l and C_s are single rows and b_l, b_s scalars) and that guards / domain constraints are spelled out. */
 typedef struct amap_piece {
   int32_t n_loops;
   const int64_t *bounds; /* n_loops (host, owned by the map)                                   */
@@ -186,15 +190,24 @@ typedef struct amap_piece {
   uint64_t fill_bits;
 } amap_piece;
 
+/* number of pieces of the composed map (all stages): the load/store pairs that are left once Section 2.1's
+ * elimination has reached its fixpoint */
 int amap_map_num_pieces(const amap_map *map, int32_t *n);
-/* *out receives views into the map, valid until amap_map_destroy */
+/* piece k in the form above (Section 2.1, equation (2): the rewritten reader); *out receives views into the
+ * map, valid until amap_map_destroy.  host pointers. */
 int amap_map_get_piece(const amap_map *map, int32_t k, amap_piece *out);
-/* element counts of the external inputs (n_inputs entries written to in_numel) and of the output */
+/* element counts of the external inputs (n_inputs entries written to in_numel, a host array of the caller) and of
+ * the output: the tensors t_l and t_s of Section 2 that survive the elimination and must exist in device memory */
 int amap_map_sizes(const amap_map *map, int32_t *n_inputs, int64_t *in_numel /* may be NULL */, int64_t *out_numel,
                    int32_t *elem_size);
 
 /* ---------------------------------------------------------------------------
  * amap_plan: choose a kernel family per piece and build the launch table.
+ * (Section 2.2 of the paper: the memory references that remain after the
+ * elimination are compulsory, and the way they are laid out and issued must
+ * let them use the available memory bandwidth in full.  There that is a
+ * mapping of tensors to scratchpad banks; here it is the choice of access
+ * width, tile shape and loop order per piece.)
  * `device` is a CUDA ordinal: the call makes it current, uploads a small
  * descriptor table to device memory owned by the plan, and restores the
  * previous device.  device = -1 gives a dry plan (no CUDA call at all) whose
@@ -242,6 +255,8 @@ typedef struct amap_stats {
 int amap_plan(const amap_map *map, int device, const amap_plan_opts *opts /* host, may be NULL */,
               amap_plan_t **out_plan);
 void amap_plan_destroy(amap_plan_t *plan);
+/* the compulsory traffic of the plan (Section 2.2: what cannot be eliminated): each unique source byte once,
+ * each output byte once; also how many kernels an execute enqueues and the family chosen per piece */
 int amap_plan_stats(const amap_plan_t *plan, amap_stats *out /* host */);
 /* kernel family chosen for piece k (an amap_kernel_kind) */
 int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
@@ -252,8 +267,9 @@ int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
  *   src_dev_ptrs  host array of n_inputs DEVICE pointers, in amap_chain.inputs order
  *   dst_dev_ptr   DEVICE pointer to the output (out_numel * elem_size bytes)
  *   cuda_stream   a cudaStream_t (NULL = the legacy default stream)
- * Enqueues the plan's kernel(s) and returns without synchronising or
- * allocating.  Source and destination must not overlap (AMAP_EINVAL if the
+ * Enqueues the plan's kernel(s) -- one per kernel family present in the map,
+ * one in all for each of the common operator chains -- and returns without
+ * synchronising or allocating.  Source and destination must not overlap (AMAP_EINVAL if the
  * byte ranges do).  Pointers must be
  * aligned to the plan's pointer_align, else AMAP_EALIGN and nothing is
  * enqueued.  Launch failures give AMAP_ECUDA.
@@ -285,25 +301,35 @@ int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void 
  * Instead of the plan's own table in cudaMalloc'ed memory, the kernels read
  * their descriptors from a fixed array that is part of the library image
  * (64 descriptors, about 70 KB; every GPU on which the library is loaded
- * holds it until the process exits).  The call copies the plan's descriptors
- * into that array on `cuda_stream` and enqueues the same kernels as
- * amap_execute behind the copy.  It calls no cudaMalloc / cudaFree and no
- * allocating library routine, and does not synchronise.
+ * holds it until the process exits).  The call enqueues, on `cuda_stream`,
+ * small kernels that carry the plan's descriptors in their parameters and
+ * write them into that array, and behind them the same kernels as
+ * amap_execute.  It calls no cudaMalloc / cudaFree, no allocating library
+ * routine and no host-to-device copy, and waits for nothing: neither the host
+ * nor the stream is synchronised.
  *
  *  - Runs on the CURRENT device; src/dst pointers and the stream must belong
- *    to it.  Arguments and alignment rules are those of amap_execute.
+ *    to it.  Arguments, alignment rules and refusals (null pointers, AMAP_EALIGN,
+ *    AMAP_EINVAL for source and destination byte ranges that overlap) are those
+ *    of amap_execute.  A plan made for another device gives AMAP_EINVAL.
  *  - A plan with more than 64 descriptors is refused with AMAP_ETOOLARGE and
  *    nothing is enqueued (compose fewer operators per call, or use amap_execute).
  *    A plan whose map keeps temporaries (more than one stage) is refused with
  *    AMAP_EUNSUPPORTED: temporaries need device memory.
  *  - The first call on each device looks up the array's device address
- *    (cudaGetSymbolAddress); make that first call before starting any stream
- *    capture on that device.
+ *    (cudaGetSymbolAddress) and the device's multiprocessor count and keeps
+ *    both for later calls; make that first call before starting any stream
+ *    capture on that device.  cudaDeviceReset invalidates what was kept: do not
+ *    call this function again in a process that has reset the device.
  *  - All calls on one device share the one array, which still holds the
- *    previous call's descriptors until the next copy overwrites them.  Calls
- *    are safe back to back on ONE stream.  Two calls that can overlap on the
- *    GPU (different streams without an ordering between them) race on the
- *    array: order them with events or use amap_execute for one of them.
+ *    previous call's descriptors until the next call's upload kernels overwrite
+ *    them.  Calls are safe back to back on ONE stream, issued by one host thread
+ *    at a time (two threads enqueueing on the same stream could interleave their
+ *    uploads and copies).  Two calls that can overlap on the GPU (different
+ *    streams without an ordering between them) race on the array: order them
+ *    with events or use amap_execute for one of them.
+ *  - A dry plan assumes a 148-multiprocessor device for its L2 look-ahead
+ *    distances; this call rescales them to the device it runs on.
  * ------------------------------------------------------------------------- */
 int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, void *cuda_stream);
 

@@ -84,6 +84,7 @@ static FastDiv make_fastdiv(uint32_t d) {
   return f;
 }
 
+static const int kDefaultSms = 148;  // B200; only dry plans rely on it
 static const int kUnroll = kStrip;  // units per thread in the affine kernel
 
 // largest power-of-two unit (<= 16 bytes) in which the piece is still an affine loop nest
@@ -912,9 +913,11 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
   pl->stats.n_descriptors = (int32_t)pl->table.size();
   pl->stats.n_stages = (int32_t)m.stages.size();
   {
-    // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM)
-    int sms = 148;
-    if (device >= 0) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    // prefetch distance for the transpose kernel: the number of blocks resident at once (8 per SM).  A dry plan
+    // knows no device: it assumes kDefaultSms, and amap_execute_static rescales the distances for the device it
+    // runs on.
+    int sms = kDefaultSms;
+    if (device >= 0 && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) sms = kDefaultSms;
     const char *dist = getenv("AMAP_PREFETCH_DISTANCE");
     const int ahead = dist ? atoi(dist) : 8 * sms;
     for (DevPiece &d : pl->table)
@@ -1118,27 +1121,36 @@ static cudaError_t enqueue(const DescSource &ds, const Launch &L, const PtrTable
   return cudaGetLastError();
 }
 
-extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
-                            void *cuda_stream) {
-  if (!plan || plan->device < 0 || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
-  if (plan->out_numel == 0) return AMAP_OK;
+// Argument checks shared by amap_execute and amap_execute_static: null pointers, alignment to the plan's
+// pointer_align, and no overlap between any source's byte range and the destination's.  Fills pt->src for the
+// external inputs.
+static int bind_buffers(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, PtrTable *pt) {
+  if (!src_dev_ptrs && !plan->in_numel.empty()) return AMAP_EINVAL;
   if (!dst_dev_ptr) return AMAP_EINVAL;
-  PtrTable pt;
-  memset(&pt, 0, sizeof pt);
+  memset(pt, 0, sizeof *pt);
   const uintptr_t mask = (uintptr_t)plan->pointer_align - 1;
-  const size_t n_in = plan->in_numel.size();
-  for (size_t q = 0; q < n_in; ++q) {
+  const uintptr_t d0 = (uintptr_t)dst_dev_ptr, d1 = d0 + (uintptr_t)plan->out_numel * plan->elem_size;
+  for (size_t q = 0; q < plan->in_numel.size(); ++q) {
     if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
     if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
-    {  // source and destination ranges must not overlap
-      const uintptr_t s0 = (uintptr_t)src_dev_ptrs[q], s1 = s0 + (uintptr_t)plan->in_numel[q] * plan->elem_size;
-      const uintptr_t d0 = (uintptr_t)dst_dev_ptr, d1 = d0 + (uintptr_t)plan->out_numel * plan->elem_size;
-      if (s0 < d1 && d0 < s1) return AMAP_EINVAL;
-    }
-    pt.src[q] = (const char *)src_dev_ptrs[q];
+    const uintptr_t s0 = (uintptr_t)src_dev_ptrs[q], s1 = s0 + (uintptr_t)plan->in_numel[q] * plan->elem_size;
+    if (s0 < d1 && d0 < s1) return AMAP_EINVAL;  // source and destination ranges must not overlap
+    pt->src[q] = (const char *)src_dev_ptrs[q];
   }
+  if (d0 & mask) return AMAP_EALIGN;
+  pt->dst = (char *)dst_dev_ptr;
+  return AMAP_OK;
+}
+
+extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
+                            void *cuda_stream) {
+  if (!plan || plan->device < 0) return AMAP_EINVAL;
+  if (plan->out_numel == 0) return AMAP_OK;
+  PtrTable pt;
+  const int brc = bind_buffers(plan, src_dev_ptrs, dst_dev_ptr, &pt);
+  if (brc != AMAP_OK) return brc;
+  const size_t n_in = plan->in_numel.size();
   for (size_t k = 0; k < plan->temps.size(); ++k) pt.src[n_in + k] = (const char *)plan->temps[k];
-  if ((uintptr_t)dst_dev_ptr & mask) return AMAP_EALIGN;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   int prev = 0;
   CUDA_TRY(cudaGetDevice(&prev));
@@ -1242,6 +1254,14 @@ extern "C" int amap_execute_host(amap_plan_t *plan, const void *const *src_host_
 static const int kStaticMaxPieces = 64;
 static __device__ __align__(256) unsigned char g_static_table[kStaticMaxPieces * sizeof(DevPiece)];
 
+// writes descriptors [first, first + ld.n_pieces) of the fixed array (device code names the array directly)
+__global__ void amap_static_table_store(const __grid_constant__ LaunchDesc ld, int first) {
+  const uint32_t *src = reinterpret_cast<const uint32_t *>(ld.piece);
+  uint32_t *dst = reinterpret_cast<uint32_t *>(g_static_table + (size_t)first * sizeof(DevPiece));
+  const int words = ld.n_pieces * (int)(sizeof(DevPiece) / 4);
+  for (int w = threadIdx.x; w < words; w += blockDim.x) dst[w] = src[w];
+}
+
 static const int kStaticMaxDevices = 64;
 static void *g_static_table_addr[kStaticMaxDevices];  // device address of g_static_table, per device, 0 = not set up
 
@@ -1260,24 +1280,27 @@ static int static_table_address(int device, void **out) {
   return AMAP_OK;
 }
 
+// multiprocessors of the current device, looked up once per device (the look-ahead distance of a dry plan is
+// set for the device the call runs on)
+static int g_static_sms[kStaticMaxDevices];
+static int static_device_sms(int device) {
+  int n = __atomic_load_n(&g_static_sms[device], __ATOMIC_ACQUIRE);
+  if (n <= 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = kDefaultSms;
+    __atomic_store_n(&g_static_sms[device], n, __ATOMIC_RELEASE);
+  }
+  return n;
+}
+
 extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
                                    void *cuda_stream) {
-  if (!plan || (!src_dev_ptrs && !plan->in_numel.empty())) return AMAP_EINVAL;
+  if (!plan) return AMAP_EINVAL;
   if (plan->table.size() > (size_t)kStaticMaxPieces) return AMAP_ETOOLARGE;
   if (!plan->temp_numel.empty()) return AMAP_EUNSUPPORTED;  // temporaries would need device memory
   if (plan->out_numel == 0) return AMAP_OK;
-  if (!dst_dev_ptr) return AMAP_EINVAL;
   PtrTable pt;
-  memset(&pt, 0, sizeof pt);
-  const uintptr_t mask = (uintptr_t)plan->pointer_align - 1;
-  for (size_t q = 0; q < plan->in_numel.size(); ++q) {
-    if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
-    if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
-    if (src_dev_ptrs[q] == dst_dev_ptr) return AMAP_EINVAL;
-    pt.src[q] = (const char *)src_dev_ptrs[q];
-  }
-  if ((uintptr_t)dst_dev_ptr & mask) return AMAP_EALIGN;
-  pt.dst = (char *)dst_dev_ptr;
+  const int brc = bind_buffers(plan, src_dev_ptrs, dst_dev_ptr, &pt);  // the same refusals as amap_execute
+  if (brc != AMAP_OK) return brc;
   int device = 0;
   CUDA_TRY(cudaGetDevice(&device));
   if (plan->device >= 0 && plan->device != device) return AMAP_EINVAL;
@@ -1285,12 +1308,35 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
   const int rc = static_table_address(device, &table);
   if (rc != AMAP_OK) return rc;
   cudaStream_t s = (cudaStream_t)cuda_stream;
-  // the part of the array this plan uses is overwritten in full; nothing in it needs to start at zero
-  CUDA_TRY(cudaMemcpyAsync(table, plan->table.data(), plan->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice, s));
+  // The descriptors travel to the array in the parameters of small kernels, kParamPieces at a time: nothing is
+  // copied from host memory, so neither the host nor the stream is made to wait.  A dry plan was made without
+  // knowing the device: its look-ahead distances assume kDefaultSms multiprocessors and are rescaled here.
+  const int sms = static_device_sms(device);
+  const bool rescale = plan->device < 0 && sms != kDefaultSms;
+  for (size_t first = 0; first < plan->table.size(); first += kParamPieces) {
+    LaunchDesc ld;
+    memset(&ld, 0, sizeof ld);
+    ld.n_pieces = (int32_t)std::min<size_t>(kParamPieces, plan->table.size() - first);
+    for (int q = 0; q < ld.n_pieces; ++q) {
+      ld.piece[q] = plan->table[first + q];
+      if (rescale && ld.piece[q].prefetch > 1)
+        ld.piece[q].prefetch = std::max(2, (int)((int64_t)ld.piece[q].prefetch * sms / kDefaultSms));
+    }
+    // a plain launch: it starts only after everything before it on the stream (an earlier call's kernels, which
+    // still read the array) has finished
+    amap_static_table_store<<<1, 256, 0, s>>>(ld, (int)first);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: descriptor upload");
+  }
+  bool first_launch = true;
   for (const Launch &L : plan->launches) {
     const DescSource ds{nullptr, (const DevPiece *)table};  // always through the fixed table
-    const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl);
+    // The first copy kernel must not start before the upload kernels have completed (it reads its descriptor ahead
+    // of its grid-dependency wait), so it is launched without programmatic dependent launch; the later ones only
+    // follow kernels that leave the array alone.
+    const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl && !first_launch);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute_static: kernel launch");
+    first_launch = false;
   }
   return AMAP_OK;
 }

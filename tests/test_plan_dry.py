@@ -88,3 +88,56 @@ def test_bad_plan_options():
         with pytest.raises(B.AmapError) as e:
             m.plan(**{"device": -1, **kw})
         assert e.value.code == -1, kw
+
+
+def test_execute_entry_points_refuse_bad_buffers_before_any_cuda_call():
+    """amap_execute_static shares amap_execute's argument checks: they come before the first CUDA call, so a dry
+    plan and made-up addresses show them without a GPU."""
+    chain = W.reduced_configs()["c2_fwd_rag"]
+    m = B.compose_chain(chain)
+    dry = m.plan(device=-1)
+    nbytes = m.out_numel * 2
+    src = 0x7F0000000000
+    codes = {}
+    for name, (s, d) in {
+        "overlap_equal": (src, src),
+        "overlap_partial": (src, src + 64),              # the output starts inside the input
+        "overlap_from_below": (src, src - nbytes + 32),  # the output's last bytes reach into the input
+        "misaligned_src": (src + 2, src + 4 * nbytes),
+        "misaligned_dst": (src, src + 4 * nbytes + 8),
+        "null_dst": (src, 0),
+    }.items():
+        with pytest.raises(B.AmapError) as e:
+            dry.execute_static_ptrs([s], d, 0)
+        codes[name] = e.value.code
+    assert codes == {"overlap_equal": -1, "overlap_partial": -1, "overlap_from_below": -1, "misaligned_src": -7,
+                     "misaligned_dst": -7, "null_dst": -1}
+    # amap_execute refuses a dry plan outright
+    with pytest.raises(B.AmapError) as e:
+        dry.execute_ptrs([src], src + 4 * nbytes, 0)
+    assert e.value.code == -1
+
+
+def test_static_entry_point_refuses_temporaries_and_oversized_plans():
+    awkward = W.Chain(
+        name="awkward", dtype="bf16", inputs=[[40, 24]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},
+            {"kind": "reshape", "src": 1, "shape": [64, 15]},
+            {"kind": "transpose", "src": 2, "perm": [1, 0]},
+        ],
+        values="normal",
+    )
+    m = B.compose_chain(awkward, B.COMPOSE_NO_FUSE)
+    dry = m.plan(device=-1)
+    assert dry.stats()["n_stages"] > 1
+    with pytest.raises(B.AmapError) as e:
+        dry.execute_static_ptrs([0x7F0000000000], 0x7F0000100000, 0)
+    assert e.value.code == -9  # temporaries need device memory
+    b = B.Builder(2)
+    ids = [b.input([4, 8]) for _ in range(22)]
+    big = b.compose(b.concat([b.pad(t, [1, 1], [1, 1]) for t in ids], 0)).plan(device=-1)
+    assert big.stats()["n_descriptors"] > 64
+    with pytest.raises(B.AmapError) as e:
+        big.execute_static_ptrs([0x7F0000000000 + 4096 * k for k in range(22)], 0x7F0000100000, 0)
+    assert e.value.code == -11

@@ -1,11 +1,13 @@
 """amap_execute_static: the entry point for callers that may not allocate device memory
 (a plug-in inside a framework that owns the GPU's memory, a serving loop that cannot
 afford cudaMalloc's device-wide synchronisation).  It must produce exactly what
-amap_execute produces, call after call, although every call reuses one fixed descriptor
-table inside the library.  Collected last on purpose (file name)."""
+amap_execute produces -- and what the CPU oracle computes -- call after call, although
+every call reuses one fixed descriptor table inside the library.  Collected last on
+purpose (file name)."""
 import numpy as np
 import pytest
 
+from oracle import oracle
 from paper_2002_12798_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -26,6 +28,8 @@ def _both_ways(B, torch, chain):
     dry = m.plan(device=-1)  # a plan made without touching CUDA
     dry.execute_static_ptrs(ptrs, out.data_ptr(), stream)
     torch.cuda.synchronize()
+    want = oracle.run_chain(chain, xs).reshape(-1)  # the independent opinion: pure copies, so bit for bit
+    assert np.array_equal(out.cpu().numpy().view(want.dtype), want), chain.name
     return ref, out, dry, dev, stream  # dev is returned so that the inputs stay allocated
 
 
@@ -48,6 +52,25 @@ def test_static_table_matches_amap_execute_on_calls_in_a_row():
         dry.execute_static_ptrs(ptrs, again.data_ptr(), stream)
         torch.cuda.synchronize()
         assert torch.equal(ref, again), name
+
+
+def test_static_table_accepts_a_plan_made_for_the_current_device():
+    import torch
+
+    from paper_2002_12798_b200 import binding as B
+
+    chain = W.reduced_configs()["c4_odd"]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs).reshape(-1)
+    m = B.compose_chain(chain)
+    plan = m.plan(device=0)  # not a dry plan: it owns a table in device memory, which this entry point ignores
+    dev = [torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).cuda() for x in xs]
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(2):
+        out = torch.full((m.out_numel,), 0x33, dtype=torch.int16, device="cuda")
+        plan.execute_static_ptrs([d.data_ptr() for d in dev], out.data_ptr(), stream)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy().view(np.uint16), want)
 
 
 def test_static_table_refuses_a_plan_that_does_not_fit():
