@@ -223,6 +223,38 @@ int oracle_window_gather(const void *in, void *out, const int64_t *in_shape /* N
   return 0;
 }
 
+/* The window gather with dilated taps and a choice of column order (the im2col families of the common
+ * frameworks; the paper's Section 2.1 treats all of them as load/store pairs with a non-injective load):
+ *   tap (r, s) of output pixel (ho, wo) reads in[n, ho*stride + r*dilation, wo*stride + s*dilation, c],
+ *   Ho = (Hp - dilation*(kh-1) - 1)/stride + 1, likewise Wo,
+ *   column = (r*kw + s)*C + c   when crs_order == 0  (channel fastest, NHWC style),
+ *   column = (c*kh + r)*kw + s  when crs_order != 0  (tap fastest, NCHW style).
+ * The zero border comes from oracle_pad, run as its own operator before. */
+int oracle_window_gather_ex(const void *in, void *out, const int64_t *in_shape /* N,Hp,Wp,C */, int64_t kh,
+                            int64_t kw, int64_t stride, int64_t dilation, int crs_order, int es, int nt) {
+  if (bad_common(4, in_shape, es) || kh < 1 || kw < 1 || stride < 1 || dilation < 1) return -1;
+  const int64_t N = in_shape[0], Hp = in_shape[1], Wp = in_shape[2], C = in_shape[3];
+  const int64_t span_h = dilation * (kh - 1) + 1, span_w = dilation * (kw - 1) + 1;
+  if (Hp < span_h || Wp < span_w) return -2;
+  const int64_t Ho = (Hp - span_h) / stride + 1, Wo = (Wp - span_w) / stride + 1;
+  const int64_t cols = kh * kw * C;
+  const unsigned char *src = (const unsigned char *)in;
+  unsigned char *dst = (unsigned char *)out;
+#pragma omp parallel for num_threads(nt) schedule(static)
+  for (int64_t n = 0; n < N; ++n)
+    for (int64_t ho = 0; ho < Ho; ++ho)
+      for (int64_t wo = 0; wo < Wo; ++wo)
+        for (int64_t r = 0; r < kh; ++r)
+          for (int64_t s = 0; s < kw; ++s)
+            for (int64_t c = 0; c < C; ++c) {
+              int64_t row = (n * Ho + ho) * Wo + wo;
+              int64_t col = crs_order ? (c * kh + r) * kw + s : (r * kw + s) * C + c;
+              int64_t h = ho * stride + r * dilation, w = wo * stride + s * dilation;
+              copy_elem(dst, row * cols + col, src, ((n * Hp + h) * Wp + w) * C + c, es);
+            }
+  return 0;
+}
+
 /* tile(reps): the whole tensor laid side by side reps[d] times along every
  * axis (Section 2.1 names tile and repeat among the pure copies):
  * out.shape[d] = reps[d]*in.shape[d], out[o] = in[j] with j[d] = o[d] mod in.shape[d]. */

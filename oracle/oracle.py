@@ -131,16 +131,31 @@ def pad(x, lo, hi, nt=1):
     return out
 
 
-def window(x, kh, kw, stride, padding, nt=1):
-    """NHWC im2col = zero pad on H and W, then the window gather: two operators."""
+def window(x, kh, kw, stride, padding, nt=1, dilation=1, order="rsc"):
+    """NHWC im2col = zero pad on H and W, then the window gather: two operators.  `order`: "rsc" (column
+    (r*kw+s)*C+c) or "crs" (column (c*kh+r)*kw+s); taps are `dilation` pixels apart."""
     x = _raw(x)
     if x.ndim != 4:
         raise ValueError("window wants NHWC")
+    if order not in ("rsc", "crs"):
+        raise ValueError("window column order")
     xp = pad(x, [0, padding, padding, 0], [0, padding, padding, 0], nt)
     N, Hp, Wp, C = xp.shape
-    Ho, Wo = (Hp - kh) // stride + 1, (Wp - kw) // stride + 1
+    if dilation == 1 and order == "rsc":
+        Ho, Wo = (Hp - kh) // stride + 1, (Wp - kw) // stride + 1
+        out = np.empty([N * Ho * Wo, kh * kw * C], dtype=x.dtype)
+        _check(lib().oracle_window_gather(_ptr(xp), _ptr(out), _i64(xp.shape), kh, kw, stride, x.itemsize, nt), "window")
+        return out
+    Ho = (Hp - dilation * (kh - 1) - 1) // stride + 1
+    Wo = (Wp - dilation * (kw - 1) - 1) // stride + 1
     out = np.empty([N * Ho * Wo, kh * kw * C], dtype=x.dtype)
-    _check(lib().oracle_window_gather(_ptr(xp), _ptr(out), _i64(xp.shape), kh, kw, stride, x.itemsize, nt), "window")
+    _check(
+        lib().oracle_window_gather_ex(
+            _ptr(xp), _ptr(out), _i64(xp.shape), ctypes.c_int64(kh), ctypes.c_int64(kw), ctypes.c_int64(stride),
+            ctypes.c_int64(dilation), int(order == "crs"), x.itemsize, nt,
+        ),
+        "window",
+    )
     return out
 
 
@@ -232,7 +247,8 @@ def run_chain(chain, inputs, nt=1, keep_intermediates=False):
         elif kind == "pad":
             t = pad(tensors[op["src"]], op["lo"], op["hi"], nt)
         elif kind == "window":
-            t = window(tensors[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"], nt)
+            t = window(tensors[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"], nt, op.get("dilation", 1),
+                       op.get("order", "rsc"))
         elif kind == "tile":
             t = tile(tensors[op["src"]], op["reps"], nt)
         elif kind == "repeat":

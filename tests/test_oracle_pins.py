@@ -213,6 +213,39 @@ def test_window_matches_torch_unfold(k, stride, padding):
     assert np.array_equal(y.astype(np.float32), u.numpy())
 
 
+@pytest.mark.parametrize("k,stride,padding,dilation", [(3, 1, 2, 2), (3, 2, 2, 2), (2, 1, 1, 3), (3, 1, 1, 1), (5, 1, 4, 2)])
+@pytest.mark.parametrize("order", ["rsc", "crs"])
+def test_dilated_window_and_column_orders_match_torch_unfold(k, stride, padding, dilation, order):
+    """torch's unfold has the dilation argument and produces the (c, r, s) column order natively."""
+    torch = pytest.importorskip("torch")
+    N, H, Wd, C = 2, 11, 9, 5
+    x = rng.integers(1, 2000, size=(N, H, Wd, C)).astype(np.uint32)
+    y = oracle.window(x, k, k, stride, padding, dilation=dilation, order=order)
+    xt = torch.from_numpy(x.astype(np.float32)).permute(0, 3, 1, 2)  # NCHW
+    u = torch.nn.functional.unfold(xt, k, dilation=dilation, padding=padding, stride=stride)  # [N, C*k*k, L]
+    L = u.shape[-1]
+    if order == "crs":
+        want = u.permute(0, 2, 1).reshape(N * L, C * k * k)  # unfold's own order
+    else:
+        want = u.reshape(N, C, k, k, L).permute(0, 4, 2, 3, 1).reshape(N * L, k * k * C)
+    assert y.shape == tuple(want.shape)
+    assert np.array_equal(y.astype(np.float32), want.numpy())
+
+
+def test_dilated_window_spot_values():
+    """Tap (r, s) of output pixel (ho, wo) reads in[ho*stride + r*dilation - pad, wo*stride + s*dilation - pad]."""
+    N, H, Wd, C = 1, 10, 12, 3
+    x = (np.arange(N * H * Wd * C, dtype=np.uint32) + 1).reshape(N, H, Wd, C)
+    k, stride, padding, dil = 3, 2, 2, 2
+    Ho, Wo = (H + 2 * padding - dil * (k - 1) - 1) // stride + 1, (Wd + 2 * padding - dil * (k - 1) - 1) // stride + 1
+    y = oracle.window(x, k, k, stride, padding, dilation=dil, order="rsc").reshape(Ho, Wo, k, k, C)
+    z = oracle.window(x, k, k, stride, padding, dilation=dil, order="crs").reshape(Ho, Wo, C, k, k)
+    for ho, wo, r, s_, c in [(0, 0, 0, 0, 0), (1, 2, 2, 1, 2), (Ho - 1, Wo - 1, 2, 2, 1), (2, 3, 1, 1, 0)]:
+        h, w = ho * stride + r * dil - padding, wo * stride + s_ * dil - padding
+        want = x[0, h, w, c] if 0 <= h < H and 0 <= w < Wd else 0
+        assert y[ho, wo, r, s_, c] == want and z[ho, wo, c, r, s_] == want
+
+
 # ---------------------------------------------------------------------------
 # the generic load/store statement
 # ---------------------------------------------------------------------------
