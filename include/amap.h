@@ -118,6 +118,15 @@ int amap_builder_pad(amap_builder *b, int32_t src, int32_t rank, const int64_t *
  * in[n, ho*stride+r-pad, wo*stride+s-pad, c], zero outside (one guarded, non-injective load) */
 int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
                         int32_t *out);
+/* The same gather with taps `dilation` pixels apart and a choice of column order: tap (r, s) of output pixel
+ * (ho, wo) reads in[n, ho*stride + r*dilation - pad, wo*stride + s*dilation - pad, c], zero outside;
+ * Ho = (H + 2*pad - dilation*(kh-1) - 1)/stride + 1, likewise Wo.  AMAP_WINDOW_COLS_RSC: column (r*kw+s)*C+c
+ * (channel fastest, as amap_builder_window); AMAP_WINDOW_COLS_CRS: column (c*kh+r)*kw+s (tap fastest, the order
+ * of NCHW im2col).  Still one guarded load/store pair in the paper's form (Section 2.1). */
+#define AMAP_WINDOW_COLS_RSC 0
+#define AMAP_WINDOW_COLS_CRS 1
+int amap_builder_window_ex(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                           int32_t dilation, int32_t column_order, int32_t *out);
 /* broadcast: out[o] = in[o mod in.shape] with out.shape[d] = reps[d]*in.shape[d] (the paper's repeat/tile family) */
 int amap_builder_tile(amap_builder *b, int32_t src, int32_t rank, const int64_t *reps, int32_t *out);
 /* every element `count` times in a row along `axis`: out[.., i*count + j, ..] = in[.., i, ..] (a load that ignores

@@ -24,7 +24,7 @@ KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
 EXPORTS = [
     "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",
     "amap_builder_transpose", "amap_builder_slice", "amap_builder_concat", "amap_builder_pad",
-    "amap_builder_window", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
+    "amap_builder_window", "amap_builder_window_ex", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
     "amap_builder_stmt",
     "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
@@ -163,9 +163,14 @@ class Builder:
             "amap_builder_pad", o,
         )
 
-    def window(self, src, kh, kw, stride, pad):
+    def window(self, src, kh, kw, stride, pad, dilation=1, order="rsc"):
         o = c_int32()
-        return self._out(_lib.amap_builder_window(self._h, src, kh, kw, stride, pad, byref(o)), "amap_builder_window", o)
+        if dilation == 1 and order == "rsc":
+            return self._out(_lib.amap_builder_window(self._h, src, kh, kw, stride, pad, byref(o)), "amap_builder_window", o)
+        return self._out(
+            _lib.amap_builder_window_ex(self._h, src, kh, kw, stride, pad, dilation, {"rsc": 0, "crs": 1}[order], byref(o)),
+            "amap_builder_window_ex", o,
+        )
 
     def tile(self, src, reps):
         o = c_int32()
@@ -380,7 +385,7 @@ def build_chain(chain) -> tuple:
         elif k == "pad":
             t = b.pad(ids[op["src"]], op["lo"], op["hi"], 0)
         elif k == "window":
-            t = b.window(ids[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"])
+            t = b.window(ids[op["src"]], op["kh"], op["kw"], op["stride"], op["pad"], op.get("dilation", 1), op.get("order", "rsc"))
         elif k == "tile":
             t = b.tile(ids[op["src"]], op["reps"])
         elif k == "repeat":

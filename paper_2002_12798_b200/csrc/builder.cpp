@@ -301,32 +301,41 @@ extern "C" int amap_builder_pad(amap_builder *b, int32_t src, int32_t rank, cons
   return AMAP_OK;
 }
 
-extern "C" int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
-                                   int32_t *out) {
+extern "C" int amap_builder_window_ex(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                                      int32_t dilation, int32_t column_order, int32_t *out) {
   GUARD_BUILDER(b, out);
-  if (!b->valid(src) || b->shapes[src].size() != 4 || kh < 1 || kw < 1 || stride < 1 || pad < 0) return AMAP_EINVAL;
+  if (!b->valid(src) || b->shapes[src].size() != 4 || kh < 1 || kw < 1 || stride < 1 || pad < 0 || dilation < 1 ||
+      (column_order != AMAP_WINDOW_COLS_RSC && column_order != AMAP_WINDOW_COLS_CRS))
+    return AMAP_EINVAL;
   const std::vector<int64_t> in = b->shapes[src];
   const int64_t N = in[0], H = in[1], W = in[2], C = in[3];
-  if (H + 2 * pad < kh || W + 2 * pad < kw) return AMAP_EINVAL;
-  const int64_t Ho = (H + 2 * pad - kh) / stride + 1, Wo = (W + 2 * pad - kw) / stride + 1;
+  const int64_t span_h = (int64_t)dilation * (kh - 1) + 1, span_w = (int64_t)dilation * (kw - 1) + 1;
+  if (H + 2 * pad < span_h || W + 2 * pad < span_w) return AMAP_EINVAL;
+  const int64_t Ho = (H + 2 * pad - span_h) / stride + 1, Wo = (W + 2 * pad - span_w) / stride + 1;
   StmtRec r;  // loops (n, ho, wo, r, s, c)
   r.bounds = {N, Ho, Wo, kh, kw, C};
   const int n = 6;
   r.lC.assign(4 * n, 0);
   r.lC[0 * n + 0] = 1;
   r.lC[1 * n + 1] = stride;
-  r.lC[1 * n + 3] = 1;
+  r.lC[1 * n + 3] = dilation;
   r.lC[2 * n + 2] = stride;
-  r.lC[2 * n + 4] = 1;
+  r.lC[2 * n + 4] = dilation;
   r.lC[3 * n + 5] = 1;
   r.lb = {0, -(int64_t)pad, -(int64_t)pad, 0};
   r.sC.assign(2 * n, 0);
   r.sC[0 * n + 0] = Ho * Wo;
   r.sC[0 * n + 1] = Wo;
   r.sC[0 * n + 2] = 1;
-  r.sC[1 * n + 3] = (int64_t)kw * C;
-  r.sC[1 * n + 4] = C;
-  r.sC[1 * n + 5] = 1;
+  if (column_order == AMAP_WINDOW_COLS_RSC) {  // column (r*kw + s)*C + c
+    r.sC[1 * n + 3] = (int64_t)kw * C;
+    r.sC[1 * n + 4] = C;
+    r.sC[1 * n + 5] = 1;
+  } else {  // column (c*kh + r)*kw + s
+    r.sC[1 * n + 3] = kw;
+    r.sC[1 * n + 4] = 1;
+    r.sC[1 * n + 5] = (int64_t)kh * kw;
+  }
   r.sb = {0, 0};
   r.guarded = 1;
   r.fill = 0;
@@ -337,6 +346,11 @@ extern "C" int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int
   *out = r.store_tensor;
   b->stmts.push_back(std::move(r));
   return AMAP_OK;
+}
+
+extern "C" int amap_builder_window(amap_builder *b, int32_t src, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                                   int32_t *out) {
+  return amap_builder_window_ex(b, src, kh, kw, stride, pad, 1, AMAP_WINDOW_COLS_RSC, out);
 }
 
 extern "C" int amap_builder_tile(amap_builder *b, int32_t src, int32_t rank, const int64_t *reps, int32_t *out) {

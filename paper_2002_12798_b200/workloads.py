@@ -17,7 +17,8 @@ Chain format
   {"kind": "slice",     "src": t, "start": [...], "stop": [...], "step": [...]}
   {"kind": "concat",    "srcs": [t0, t1, ...], "axis": a}
   {"kind": "pad",       "src": t, "lo": [...], "hi": [...]}          zero fill
-  {"kind": "window",    "src": t, "kh":, "kw":, "stride":, "pad":}   NHWC im2col, column order (r, s, c)
+  {"kind": "window",    "src": t, "kh":, "kw":, "stride":, "pad":}   NHWC im2col, column order (r, s, c);
+                        optional "dilation": d (taps d pixels apart), "order": "rsc" | "crs" (column order)
   {"kind": "tile",      "src": t, "reps": [...]}                     the whole tensor reps[d] times along axis d
   {"kind": "repeat",    "src": t, "axis": a, "count": c}             every element c times in a row along axis a
   {"kind": "split",     "src": t, "axis": a, "sizes": [...], "part": k}   part k of t cut along axis a
@@ -228,12 +229,17 @@ def c4_inception_concat(N=64, channels=(64, 96, 128, 32), H=28, W=28, dtype="fp1
     )
 
 
-def c5_im2col(N=64, H=56, W=56, C=128, k=3, stride=1, pad=1, dtype="fp16") -> Chain:
+def c5_im2col(N=64, H=56, W=56, C=128, k=3, stride=1, pad=1, dtype="fp16", dilation=1, order="rsc") -> Chain:
+    op = {"kind": "window", "src": 0, "kh": k, "kw": k, "stride": stride, "pad": pad}
+    if dilation != 1:
+        op["dilation"] = dilation
+    if order != "rsc":
+        op["order"] = order
     return Chain(
         name="c5_im2col",
         dtype=dtype,
         inputs=[[N, H, W, C]],
-        ops=[{"kind": "window", "src": 0, "kh": k, "kw": k, "stride": stride, "pad": pad}],
+        ops=[op],
         values="uniform_pm1",
         seed=BASE_SEED + 5,
     )
@@ -349,4 +355,9 @@ def reduced_configs() -> dict:
         "c5_odd": c5_im2col(N=2, H=9, W=7, C=24, k=3, stride=2, pad=1),
         "c5_5x5": c5_im2col(N=2, H=10, W=9, C=24, k=5, stride=1, pad=2),
         "c5_5x5_wide": c5_im2col(N=1, H=12, W=11, C=128, k=5, stride=2, pad=2),
+        # dilated taps and the (c, r, s) column order of NCHW im2col
+        "c5_dil2": c5_im2col(N=2, H=13, W=11, C=128, k=3, stride=1, pad=2, dilation=2),
+        "c5_dil3_s2": c5_im2col(N=2, H=14, W=15, C=24, k=3, stride=2, pad=3, dilation=3),
+        "c5_crs": c5_im2col(N=2, H=10, W=12, C=64, k=3, stride=1, pad=1, order="crs"),
+        "c5_crs_dil2_f32": c5_im2col(N=1, H=9, W=11, C=20, k=3, stride=2, pad=2, dilation=2, order="crs", dtype="fp32"),
     }
