@@ -249,7 +249,8 @@ def bench_configs():
     configs["odd35_fwd"] = W.c2_nchw_to_nhwc(N=64, C=288, H=35, W=35)
     configs["odd35_inv"] = W.c2_nhwc_to_nchw(N=64, C=288, H=35, W=35)
     configs["map14_inv"] = W.c2_nhwc_to_nchw(N=64, C=1024, H=14, W=14)
-    configs["qkv_split"] = [W.qkv_split(part=k) for k in range(3)]
+    configs["qkv_split"] = [W.qkv_split(part=k) for k in range(3)]   # three maps, three launches
+    configs["qkv_split_one_launch"] = W.qkv_split_all()               # one map with three outputs, one launch
     return configs
 
 
@@ -301,6 +302,31 @@ def typed(torch, t, dtype_name):
     return t.view({"bf16": torch.bfloat16, "fp16": torch.float16, "fp32": torch.float32}.get(dtype_name, t.dtype))
 
 
+class Case:
+    """One configuration set up on the device: composed maps, plans, rotating buffer sets and the bound calls."""
+
+    def __init__(self, torch, B, chain, device, stream, l2, flags=0):
+        self.parts = chain if isinstance(chain, list) else [chain]
+        self.chain = self.parts[0]
+        es = self.es = self.chain.elem_size
+        self.xs = W.make_inputs(self.chain)
+        self.maps = [B.compose_chain(c, outputs=c.meta.get("outputs")) for c in self.parts]
+        self.plans = [m.plan(device.index, flags=flags) for m in self.maps]
+        self.stats = [p.stats() for p in self.plans]
+        self.total = sum(t["bytes_read"] + t["bytes_written"] for t in self.stats)
+        foot = sum(x.nbytes for x in self.xs) + sum(sum(m.out_numels) for m in self.maps) * es
+        self.n_sets = n_sets = max(2, min(8, -(-4 * l2 // foot)))
+        self.ins = [[torch.from_numpy(x.view(SIGNED[es])).to(device) for x in self.xs] for _ in range(n_sets)]
+        dt = self.ins[0][0].dtype
+        # per buffer set and per map: one tensor, or a list of them when the map has several outputs
+        self.outs = [[[torch.empty(n, dtype=dt, device=device) for n in m.out_numels] if len(m.out_numels) > 1
+                      else torch.empty(m.out_numel, dtype=dt, device=device) for m in self.maps] for _ in range(n_sets)]
+        bound = [[p.bind(self.ins[i], self.outs[i][k], stream) for k, p in enumerate(self.plans)] for i in range(n_sets)]
+        self.calls = [(lambda b=b: [c() for c in b]) if len(b) > 1 else b[0] for b in bound]
+        self.launches = sum(t["n_launches"] for t in self.stats)
+        self.single = len(self.parts) == 1 and len(self.maps[0].out_numels) == 1
+
+
 def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False, oracle=None, reps=10):
     """One row per configuration: the composed copy (median of `reps` repetitions), a plain copy of the same number
     of bytes with the library's own copy kernel, and the view-aware torch chain.  With `extras`: the unfused
@@ -309,27 +335,15 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
     out = {}
     configs = bench_configs()
     for name in names:
-        chain = configs[name]
-        parts = chain if isinstance(chain, list) else [chain]
-        chain = parts[0]
-        es = chain.elem_size
-        xs = W.make_inputs(chain)
-        maps = [B.compose_chain(c) for c in parts]
-        plans = [m.plan(device.index, flags=flags) for m in maps]
-        sts = [p.stats() for p in plans]
-        total = sum(t["bytes_read"] + t["bytes_written"] for t in sts)
-        foot = sum(x.nbytes for x in xs) + sum(mm.out_numel for mm in maps) * es
-        n_sets = max(2, min(8, -(-4 * l2 // foot)))
-        ins = [[torch.from_numpy(x.view(SIGNED[es])).to(device) for x in xs] for _ in range(n_sets)]
-        outs = [[torch.empty(mm.out_numel, dtype=ins[0][0].dtype, device=device) for mm in maps] for _ in range(n_sets)]
-        bound = [[p.bind(ins[i], outs[i][k], stream) for k, p in enumerate(plans)] for i in range(n_sets)]
-        calls = [(lambda b=b: [c() for c in b]) if len(b) > 1 else b[0] for b in bound]
-        row = rate_fields(measure_calls(torch, calls, stream, total, device.index, reps=reps), peak)
+        case = Case(torch, B, configs[name], device, stream, l2, flags)
+        chain, es, xs, total, ins, outs, n_sets = case.chain, case.es, case.xs, case.total, case.ins, case.outs, case.n_sets
+        sts = case.stats
+        row = rate_fields(measure_calls(torch, case.calls, stream, total, device.index, reps=reps), peak)
         row["bytes"] = total
-        row["launches"] = sum(t["n_launches"] for t in sts)
+        row["launches"] = case.launches
         row["kernels"] = {k: sum(t["kernels"][k] for t in sts) for k in sts[0]["kernels"]}
         row["buffer_sets"] = n_sets
-        ours = outs[0][0].clone() if len(parts) == 1 else None
+        ours = outs[0][0].clone() if case.single else None
 
         # the library's own plain copy of the same number of bytes (practical ceiling at this size)
         if name != "plain_copy_512MB":
@@ -345,7 +359,7 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
             del cin, cout, ccalls, cplan
 
         # torch's own operators on the same GPU, views kept as views
-        fn = torch_view_chain(torch, name, chain) if len(parts) == 1 else None
+        fn = torch_view_chain(torch, name, chain) if case.single else None
         if fn is not None:
             tin = [[typed(torch, t.view(list(shape)), chain.dtype) for t, shape in zip(s, chain.inputs)] for s in ins]
             got = fn(tin[0])
@@ -358,7 +372,7 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
                                        "same_bits": same}
             del tin, tcalls
 
-        if extras and len(chain.ops) > 1 and len(parts) == 1:
+        if extras and len(chain.ops) > 1 and case.single:
             # the chain before data-movement elimination: one launch and one temporary per operator, same kernels
             uplan = B.compose_chain(chain, B.COMPOSE_NO_FUSE).plan(device.index, flags=flags)
             ucalls = [uplan.bind(ins[i], outs[i][0], stream) for i in range(n_sets)]
@@ -367,10 +381,10 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
             row["unfused"] = {"us": u["us"], "gbs_effective": u["gbs"], "bytes_moved": ust["bytes_read"] + ust["bytes_written"],
                               "stages": ust["n_stages"], "slowdown": round(u["us"] / row["us"], 2)}
             del uplan, ucalls
-        if extras and oracle is not None and len(parts) == 1:
+        if extras and oracle is not None and case.single:
             row["cpu_oracle"] = oracle_row(oracle, chain, xs, total, ours.cpu().numpy())
         out[name] = row
-        del ins, outs, bound, calls, ours
+        del ins, outs, case, ours
         torch.cuda.empty_cache()
     return out
 
@@ -611,7 +625,7 @@ def run_ours(args):
         torch.cuda.empty_cache()
         names = list(TABLE_CONFIGS)
         if args.all_configs:
-            names += ["upsample2x", "qkv_split", "plain_copy_512MB"]
+            names += ["upsample2x", "qkv_split", "qkv_split_one_launch", "plain_copy_512MB"]
         if not args.no_table:
             line["configs"] = config_rows(torch, B, device, stream, l2, peak, names, flags=args.plan_flags,
                                           extras=args.all_configs, oracle=oracle, reps=max(10, args.reps))
@@ -716,30 +730,20 @@ def run_one_config(args):
     torch.cuda.set_device(device)
     stream = torch.cuda.current_stream(device)
     l2 = torch.cuda.get_device_properties(device).L2_cache_size
-    chain = bench_configs()[args.config]
-    parts = chain if isinstance(chain, list) else [chain]
-    es = parts[0].elem_size
-    xs = W.make_inputs(parts[0])
-    maps = [B.compose_chain(c) for c in parts]
-    plans = [m.plan(0, flags=args.plan_flags) for m in maps]
-    total = sum(p.stats()["bytes_read"] + p.stats()["bytes_written"] for p in plans)
-    foot = sum(x.nbytes for x in xs) + sum(m.out_numel for m in maps) * es
-    n_sets = max(2, min(8, -(-4 * l2 // foot)))
-    ins = [[torch.from_numpy(x.view(SIGNED[es])).to(device) for x in xs] for _ in range(n_sets)]
-    outs = [[torch.empty(m.out_numel, dtype=ins[0][0].dtype, device=device) for m in maps] for _ in range(n_sets)]
-    calls = [[p.bind(ins[i], outs[i][k], stream) for k, p in enumerate(plans)] for i in range(n_sets)]
+    case = Case(torch, B, bench_configs()[args.config], device, stream, l2, args.plan_flags)
+    calls, n_sets, total = case.calls, case.n_sets, case.total
     for i in range(args.warmup):
-        [c() for c in calls[i % n_sets]]
+        calls[i % n_sets]()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     stream.synchronize()
     start.record(stream)
     for i in range(args.steps):
-        [c() for c in calls[i % n_sets]]
+        calls[i % n_sets]()
     stop.record(stream)
     stream.synchronize()
     sec = start.elapsed_time(stop) * 1e-3 / args.steps
     print(json.dumps({args.config: {"us": round(sec * 1e6, 2), "gbs": round(total / sec / 1e9, 1), "bytes": total,
-                                    "buffer_sets": n_sets, "launches": sum(p.stats()["n_launches"] for p in plans)}}))
+                                    "buffer_sets": n_sets, "launches": case.launches}}))
 
 
 def main():

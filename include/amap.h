@@ -137,6 +137,14 @@ int amap_builder_repeat(amap_builder *b, int32_t src, int32_t axis, int64_t coun
  * of its own: compose once per part that is wanted as an output. */
 int amap_builder_split(amap_builder *b, int32_t src, int32_t axis, int32_t n_parts, const int64_t *sizes,
                        int32_t *outs);
+/* A tensor computed by an operator that is NOT a layout operator (a convolution, a matmul, ...) from the tensors
+ * `ins` (host array of n_ins ids).  Data-movement elimination stops at such an operator (Section 2.1 eliminates
+ * load/store PAIRS; the paper's evaluation, Section 3, keeps what feeds compute): the new tensor is bound at execute
+ * time like an external input (its position in amap_chain.inputs follows the inputs declared before it), the
+ * statements behind it compose into reads of it, and the statements before it compose into the tensors in `ins`,
+ * which the caller asks for as outputs of a map of their own (amap_compose_multi) and hands to the operator. */
+int amap_builder_opaque(amap_builder *b, int32_t n_ins, const int32_t *ins, int32_t rank, const int64_t *shape,
+                        int32_t *out);
 /* declare a tensor that raw statements will define */
 int amap_builder_tensor(amap_builder *b, int32_t rank, const int64_t *shape, int32_t *out);
 /* append one raw statement (deep-copied) */
@@ -161,13 +169,25 @@ int amap_compose(const amap_chain *chain, amap_map **out_map);
  * chain operator by operator as the paper's Section 2.1 finds it before the optimisation (the comparison baseline). */
 #define AMAP_COMPOSE_NO_FUSE 1u
 int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map **out_map);
+/* Several results from one chain (Section 2.1 names split; its last paragraph repeats the elimination until no pair
+ * is left, over the whole graph): `outputs` (host array of n_outputs distinct tensor ids, 1..8; chain->output is
+ * ignored) are all composed back to the external inputs in ONE map.  Their pieces form the map's last stage side by
+ * side (amap_piece.output says which output a piece writes), so one amap_execute_multi launch writes all of them --
+ * the parts of a split cost one launch instead of one per part.  A tensor may be an output and be read by later
+ * statements as well. */
+int amap_compose_multi(const amap_chain *chain, int32_t n_outputs, const int32_t *outputs, uint32_t flags,
+                       amap_map **out_map);
+int amap_map_num_outputs(const amap_map *map, int32_t *n);
+/* elements of output k (amap_map_sizes reports output 0) */
+int amap_map_output_numel(const amap_map *map, int32_t k, int64_t *numel);
 void amap_map_destroy(amap_map *map);
 
 /* Stages.  A map normally has ONE stage: all intermediates are gone.  Where a load/store pair cannot be
  * eliminated affinely (Section 3 of the paper reports such a leftover pair too: 123 of 124), the intermediate
  * stays as a TEMPORARY: an earlier stage writes it and later stages read it.  Stage s owns pieces
  * [first_piece, first_piece + n_pieces) of the piece list and writes temporary *dst_temp (0-based) or, when
- * *dst_temp is -1, the output; an amap_piece.input >= n_inputs names temporary (input - n_inputs).
+ * *dst_temp is -1, the output(s) -- the last stage, whose pieces name their output in amap_piece.output; an
+ * amap_piece.input >= n_inputs names temporary (input - n_inputs).
  * Temporaries live in device memory that amap_plan allocates. */
 int amap_map_num_stages(const amap_map *map, int32_t *n);
 int amap_map_get_stage(const amap_map *map, int32_t s, int32_t *first_piece, int32_t *n_pieces, int32_t *dst_temp,
@@ -197,6 +217,7 @@ typedef struct amap_piece {
   int32_t n_domain; /* where any of these fails the loop point is not part of the piece        */
   const amap_constraint *domain;
   uint64_t fill_bits;
+  int32_t output; /* which output of the map the piece writes (0 unless amap_compose_multi named several) */
 } amap_piece;
 
 /* number of pieces of the composed map (all stages): the load/store pairs that are left once Section 2.1's
@@ -284,6 +305,12 @@ int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
  * enqueued.  Launch failures give AMAP_ECUDA.
  * ------------------------------------------------------------------------- */
 int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, void *cuda_stream);
+/* The same for a map with several outputs (amap_compose_multi): dst_dev_ptrs is a host array of n_outputs DEVICE
+ * pointers in the order the outputs were named.  No buffer may overlap another (sources with destinations,
+ * destinations with each other): AMAP_EINVAL.  amap_execute, amap_execute_host and amap_execute_static take plans
+ * of single-output maps only (AMAP_EINVAL otherwise). */
+int amap_execute_multi(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *const *dst_dev_ptrs,
+                       void *cuda_stream);
 
 /* Same copy with HOST buffers: uploads the inputs, runs the plan, downloads
  * the output and waits.  Uses device staging memory owned by the plan

@@ -26,7 +26,8 @@ EXPORTS = [
     "amap_builder_transpose", "amap_builder_slice", "amap_builder_concat", "amap_builder_pad",
     "amap_builder_window", "amap_builder_window_ex", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
     "amap_builder_stmt",
-    "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
+    "amap_builder_opaque", "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_compose_multi",
+    "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
@@ -61,7 +62,7 @@ class _Piece(Structure):
         ("n_loops", c_int32), ("bounds", POINTER(c_int64)), ("input", c_int32), ("C_l", POINTER(c_int64)),
         ("b_l", c_int64), ("C_s", POINTER(c_int64)), ("b_s", c_int64), ("n_guards", c_int32),
         ("guards", POINTER(_Constraint)), ("n_domain", c_int32), ("domain", POINTER(_Constraint)),
-        ("fill_bits", c_uint64),
+        ("fill_bits", c_uint64), ("output", c_int32),
     ]
 
 
@@ -90,6 +91,7 @@ def _load():
     lib.amap_plan_destroy.argtypes = [c_void_p]
     lib.amap_builder_pad.argtypes = [c_void_p, c_int32, c_int32, POINTER(c_int64), POINTER(c_int64), c_uint64, POINTER(c_int32)]
     lib.amap_execute.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
+    lib.amap_execute_multi.argtypes = [c_void_p, POINTER(c_void_p), POINTER(c_void_p), c_void_p]
     lib.amap_execute_host.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
     lib.amap_execute_static.argtypes = [c_void_p, POINTER(c_void_p), c_void_p, c_void_p]
     return lib
@@ -136,6 +138,14 @@ class Builder:
     def tensor(self, shape):
         o = c_int32()
         return self._out(_lib.amap_builder_tensor(self._h, len(shape), _i64(shape), byref(o)), "amap_builder_tensor", o)
+
+    def opaque(self, ins, shape):
+        """The result of an operator that is not a layout operator, computed from tensors `ins`: bound at execute
+        like an input."""
+        o = c_int32()
+        return self._out(
+            _lib.amap_builder_opaque(self._h, len(ins), _i32(ins), len(shape), _i64(shape), byref(o)), "amap_builder_opaque", o
+        )
 
     def reshape(self, src, shape):
         o = c_int32()
@@ -220,6 +230,16 @@ class Builder:
             _check(_lib.amap_compose(chain, byref(h)), "amap_compose")
         return Map(h)
 
+    def compose_multi(self, outputs, flags=0) -> "Map":
+        """One map with several outputs (amap_compose_multi)."""
+        chain = c_void_p()
+        _check(_lib.amap_builder_chain(self._h, outputs[0] if outputs else 0, byref(chain)), "amap_builder_chain")
+        h = c_void_p()
+        _check(
+            _lib.amap_compose_multi(chain, len(outputs), _i32(outputs), ctypes.c_uint32(flags), byref(h)), "amap_compose_multi"
+        )
+        return Map(h)
+
 
 class Map:
     """A composed map: amap_compose's result."""
@@ -233,6 +253,13 @@ class Map:
         self.in_numel = [ins[q] for q in range(n_in.value)]
         self.out_numel = out_numel.value
         self.elem_size = es.value
+        n_out = c_int32()
+        _check(_lib.amap_map_num_outputs(self._h, byref(n_out)), "amap_map_num_outputs")
+        self.out_numels = []
+        for k in range(n_out.value):
+            n = c_int64()
+            _check(_lib.amap_map_output_numel(self._h, k, byref(n)), "amap_map_output_numel")
+            self.out_numels.append(n.value)
 
     def __del__(self):
         if getattr(self, "_h", None) and _lib is not None:  # module globals are gone at interpreter shutdown
@@ -262,6 +289,7 @@ class Map:
                     "guards": cons(p.guards, p.n_guards),
                     "domain": cons(p.domain, p.n_domain),
                     "fill_bits": p.fill_bits,
+                    "output": p.output,
                 }
             )
         return out
@@ -320,6 +348,12 @@ class Plan:
         arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
         _check(_lib.amap_execute(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute")
 
+    def execute_multi_ptrs(self, src_ptrs, dst_ptrs, stream=0):
+        """amap_execute_multi: one destination pointer per output of the map."""
+        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        darr = (c_void_p * max(len(dst_ptrs), 1))(*[c_void_p(p) for p in dst_ptrs])
+        _check(_lib.amap_execute_multi(self._h, arr, darr, c_void_p(stream)), "amap_execute_multi")
+
     def execute_static_ptrs(self, src_ptrs, dst_ptr, stream=0):
         """amap_execute_static: no device allocation; the descriptors go through the library's fixed table."""
         arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
@@ -330,9 +364,15 @@ class Plan:
         Keeps `srcs` and `dst` alive.  For loops that launch the same plan on the same buffers many times."""
         import torch
 
-        s = (stream or torch.cuda.current_stream(dst.device)).cuda_stream
         arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(t.data_ptr()) for t in srcs])
-        h, d, st, fn = self._h, c_void_p(dst.data_ptr()), c_void_p(s), _lib.amap_execute
+        if isinstance(dst, (list, tuple)):  # a map with several outputs
+            s = (stream or torch.cuda.current_stream(dst[0].device)).cuda_stream
+            d = (c_void_p * len(dst))(*[c_void_p(t.data_ptr()) for t in dst])
+            fn = _lib.amap_execute_multi
+        else:
+            s = (stream or torch.cuda.current_stream(dst.device)).cuda_stream
+            d, fn = c_void_p(dst.data_ptr()), _lib.amap_execute
+        h, st = self._h, c_void_p(s)
         keep = (list(srcs), dst, self)
 
         def call():
@@ -404,9 +444,14 @@ def build_chain(chain) -> tuple:
         else:
             raise ValueError("unknown operator kind %r" % k)
         ids.append(t)
+    b.ids = ids  # tensor id of every input and operator result, in the chain's numbering
     return b, ids[-1]
 
 
-def compose_chain(chain, flags=0) -> Map:
+def compose_chain(chain, flags=0, outputs=None) -> Map:
+    """`outputs`: tensor numbers of the chain (inputs first, then one per operator) wanted as results; default the
+    last operator's."""
     b, out = build_chain(chain)
-    return b.compose(out, flags)
+    if outputs is None:
+        return b.compose(out, flags)
+    return b.compose_multi([b.ids[t] for t in outputs], flags)

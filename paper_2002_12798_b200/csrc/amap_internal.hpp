@@ -38,6 +38,7 @@ struct Piece {
   std::vector<Con> guards;
   std::vector<Con> domain;
   uint64_t fill = 0;
+  int out = 0;  // which output of the map the piece writes (final stage of a map with several outputs)
   int n() const { return (int)ext.size(); }
 };
 
@@ -75,14 +76,15 @@ Status canonicalise(std::vector<Piece> &pieces);
 // temporary: an earlier stage writes it, later stages read it like an input (piece.src = n_inputs + temporary).
 struct StageInfo {
   int first_piece = 0, n_pieces = 0;
-  int dst_temp = -1;  // -1: the stage writes the output
-  int64_t numel = 0;
+  int dst_temp = -1;  // -1: the stage writes the output(s): every piece names its output in Piece::out
+  int64_t numel = 0;  // elements of the temporary written; of output 0 for the final stage
 };
 
 struct Map {
   int elem_size = 0;
   std::vector<int64_t> in_numel;
-  int64_t out_numel = 0;
+  int64_t out_numel = 0;             // output 0
+  std::vector<int64_t> out_numels;   // every output
   std::vector<int64_t> temp_numel;
   std::vector<StageInfo> stages;
   std::vector<Piece> pieces;  // all stages, in execution order

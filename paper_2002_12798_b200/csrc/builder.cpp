@@ -73,6 +73,18 @@ extern "C" int amap_builder_input(amap_builder *b, int32_t rank, const int64_t *
   return AMAP_OK;
 }
 
+extern "C" int amap_builder_opaque(amap_builder *b, int32_t n_ins, const int32_t *ins, int32_t rank, const int64_t *shape,
+                                   int32_t *out) {
+  GUARD_BUILDER(b, out);
+  if (n_ins < 0 || (n_ins > 0 && !ins) || !good_shape(rank, shape)) return AMAP_EINVAL;
+  for (int32_t k = 0; k < n_ins; ++k)
+    if (!b->valid(ins[k])) return AMAP_EINVAL;
+  // to the host algebra the operator's result is one more external tensor
+  *out = b->add_tensor(std::vector<int64_t>(shape, shape + rank));
+  b->inputs.push_back(*out);
+  return AMAP_OK;
+}
+
 extern "C" int amap_builder_tensor(amap_builder *b, int32_t rank, const int64_t *shape, int32_t *out) {
   GUARD_BUILDER(b, out);
   if (!good_shape(rank, shape)) return AMAP_EINVAL;

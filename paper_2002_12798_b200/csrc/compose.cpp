@@ -514,14 +514,21 @@ static int64_t unique_reads(const Piece &p0, int64_t in_numel) {
   return std::min(bound, in_numel);
 }
 
-static Status compose_chain(const amap_chain *ch, uint32_t flags, Map *out) {
+// `outputs`: the tensors wanted as results (one: the chain's own output).  Each becomes a set of pieces of the
+// final stage; a tensor may be both an output and read by later statements.
+static Status compose_chain(const amap_chain *ch, const std::vector<int> &outputs, uint32_t flags, Map *out) {
   if (!ch) return err(AMAP_EINVAL, "null chain");
   const int es = ch->elem_size;
   if (!(es == 1 || es == 2 || es == 4 || es == 8 || es == 16)) return err(AMAP_EINVAL, "elem_size must be 1, 2, 4, 8 or 16");
   if (ch->n_tensors < 1 || !ch->tensors || ch->n_stmts < 0 || (ch->n_stmts > 0 && !ch->stmts) || ch->n_inputs < 0 ||
       (ch->n_inputs > 0 && !ch->inputs))
     return err(AMAP_EINVAL, "bad chain header");
-  if (ch->output < 0 || ch->output >= ch->n_tensors) return err(AMAP_EINVAL, "bad output tensor id");
+  if (outputs.empty() || outputs.size() > 8) return err(AMAP_EINVAL, "a map has 1 to 8 outputs");
+  for (size_t k = 0; k < outputs.size(); ++k) {
+    if (outputs[k] < 0 || outputs[k] >= ch->n_tensors) return err(AMAP_EINVAL, "bad output tensor id");
+    for (size_t j = 0; j < k; ++j)
+      if (outputs[j] == outputs[k]) return err(AMAP_EINVAL, "an output tensor is named twice");
+  }
 
   std::vector<TensorInfo> T(ch->n_tensors);
   for (int t = 0; t < ch->n_tensors; ++t) {
@@ -543,15 +550,16 @@ static Status compose_chain(const amap_chain *ch, uint32_t flags, Map *out) {
     if (t < 0 || t >= ch->n_tensors || T[t].input_slot >= 0) return err(AMAP_EINVAL, "bad or repeated input tensor id");
     T[t].input_slot = q;
   }
-  if (T[ch->output].input_slot >= 0) return err(AMAP_EINVAL, "the output tensor is an input");
+  for (int t : outputs)
+    if (T[t].input_slot >= 0) return err(AMAP_EINVAL, "the output tensor is an input");
 
   std::vector<TensorState> S(ch->n_tensors);
   out->elem_size = es;
   out->in_numel.resize(ch->n_inputs);
   for (int q = 0; q < ch->n_inputs; ++q) out->in_numel[q] = T[ch->inputs[q]].numel;
 
-  // closes the definitions of tensor t into a stage that writes temporary `temp` (-1: the output)
-  auto finish_stage = [&](int t, int temp) -> Status {
+  // closes the definitions of tensor t: canonical pieces that write temporary `temp`, or (temp < 0) output `out_k`
+  auto close_tensor = [&](int t, int temp, int out_k, std::vector<Piece> *done) -> Status {
     std::vector<Piece> pieces = S[t].defs;
     int64_t covered = 0;
     for (auto &p : pieces) {
@@ -565,9 +573,18 @@ static Status compose_chain(const amap_chain *ch, uint32_t flags, Map *out) {
                  temp < 0 ? "some output elements are never written" : "a partly written intermediate cannot be kept as a temporary");
     Status s = canonicalise(pieces);
     if (!s.ok()) return s;
-    for (auto &p : pieces)
+    for (auto &p : pieces) {
+      p.out = temp < 0 ? out_k : 0;
       for (int k = 0; k < p.n(); ++k)
         if (p.ext[k] > INT32_MAX) return err(AMAP_EOVERFLOW, "a merged loop exceeds 2^31-1 iterations");
+    }
+    done->insert(done->end(), pieces.begin(), pieces.end());
+    return Status();
+  };
+  auto finish_stage = [&](int t, int temp) -> Status {
+    std::vector<Piece> pieces;
+    Status s = close_tensor(t, temp, 0, &pieces);
+    if (!s.ok()) return s;
     StageInfo st;
     st.first_piece = (int)out->pieces.size();
     st.n_pieces = (int)pieces.size();
@@ -695,9 +712,23 @@ static Status compose_chain(const amap_chain *ch, uint32_t flags, Map *out) {
     if (!s.ok()) return s;
   }
 
-  // the output's definitions are the last stage
-  out->out_numel = T[ch->output].numel;
-  return finish_stage(ch->output, -1);
+  // the outputs' definitions are the last stage: no output depends on another (a tensor that is an output and is
+  // read again was composed through), so their pieces may run side by side
+  std::vector<Piece> last;
+  for (size_t k = 0; k < outputs.size(); ++k) {
+    out->out_numels.push_back(T[outputs[k]].numel);
+    Status s = close_tensor(outputs[k], -1, (int)k, &last);
+    if (!s.ok()) return s;
+  }
+  out->out_numel = out->out_numels[0];
+  StageInfo st;
+  st.first_piece = (int)out->pieces.size();
+  st.n_pieces = (int)last.size();
+  st.dst_temp = -1;
+  st.numel = out->out_numel;
+  out->stages.push_back(st);
+  out->pieces.insert(out->pieces.end(), last.begin(), last.end());
+  return Status();
 }
 
 int64_t piece_unique_reads(const Piece &p, int64_t in_numel) { return unique_reads(p, in_numel); }
@@ -724,12 +755,18 @@ static void log_map(const Map &m) {
 extern "C" int amap_compose(const amap_chain *chain, amap_map **out_map) { return amap_compose_ex(chain, 0, out_map); }
 
 extern "C" int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map **out_map) {
-  if (!out_map || (flags & ~(uint32_t)AMAP_COMPOSE_NO_FUSE)) return AMAP_EINVAL;
+  if (!chain) return AMAP_EINVAL;
+  return amap_compose_multi(chain, 1, &chain->output, flags, out_map);
+}
+
+extern "C" int amap_compose_multi(const amap_chain *chain, int32_t n_outputs, const int32_t *outputs, uint32_t flags,
+                                  amap_map **out_map) {
+  if (!out_map || !outputs || n_outputs < 1 || (flags & ~(uint32_t)AMAP_COMPOSE_NO_FUSE)) return AMAP_EINVAL;
   amap_map *m = new (std::nothrow) amap_map();
   if (!m) return AMAP_ENOMEM;
   Status s;
   try {
-    s = compose_chain(chain, flags, &m->m);
+    s = compose_chain(chain, std::vector<int>(outputs, outputs + n_outputs), flags, &m->m);
   } catch (const std::bad_alloc &) {
     s.code = AMAP_ENOMEM;
   }
@@ -773,6 +810,19 @@ extern "C" int amap_map_get_piece(const amap_map *map, int32_t k, amap_piece *ou
   out->n_domain = (int32_t)p.domain.size();
   out->domain = map->m.domain_views[k].data();
   out->fill_bits = p.fill;
+  out->output = p.out;
+  return AMAP_OK;
+}
+
+extern "C" int amap_map_num_outputs(const amap_map *map, int32_t *n) {
+  if (!map || !n) return AMAP_EINVAL;
+  *n = (int32_t)map->m.out_numels.size();
+  return AMAP_OK;
+}
+
+extern "C" int amap_map_output_numel(const amap_map *map, int32_t k, int64_t *numel) {
+  if (!map || !numel || k < 0 || k >= (int32_t)map->m.out_numels.size()) return AMAP_EINVAL;
+  *numel = map->m.out_numels[k];
   return AMAP_OK;
 }
 

@@ -7,6 +7,7 @@ namespace amap {
 constexpr int kDevMaxLoops = 12;
 constexpr int kDevMaxCons = 6;
 constexpr int kMaxInputs = 24;
+constexpr int kMaxOutputs = 8;
 constexpr int kStrip = 8;  // units per thread in the affine and strip kernels
 
 // unsigned 32-bit division by an invariant divisor, multiply-and-shift form
@@ -57,7 +58,7 @@ struct DevPiece {
   int32_t n_domain;
   int32_t unit_bytes;
   int32_t prefetch;  // 1: ask L2 for the block's first source lines before waiting for the previous kernel
-  int32_t pad0_;
+  int32_t out;  // slot of the destination pointer (0 unless the map has several outputs)
   uint32_t first_block;  // first block of this piece inside its launch
   uint32_t n_blocks;
   uint64_t n_items;
@@ -89,7 +90,7 @@ struct DevPiece {
 
 struct PtrTable {
   const char *src[kMaxInputs];
-  char *dst;
+  char *dst[kMaxOutputs];
 };
 
 }  // namespace amap

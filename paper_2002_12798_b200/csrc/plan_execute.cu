@@ -50,7 +50,8 @@ struct amap_plan_t {
   int pointer_align = 0;
   bool pdl = true;  // launch with programmatic stream serialisation
   std::vector<int64_t> in_numel;
-  int64_t out_numel = 0;
+  int64_t out_numel = 0;            // output 0
+  std::vector<int64_t> out_numels;  // every output
   std::vector<int64_t> temp_numel;  // temporaries between stages
   std::vector<int> stage_dst;       // per stage: temporary written, -1 = the output
   std::vector<void *> temps;        // device memory of the temporaries (owned)
@@ -123,6 +124,7 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
   memset(d, 0, sizeof *d);
   d->kind = kDevAffine;
   d->input = p.src;
+  d->out = p.out;
   d->unit_bytes = V;
   d->fill[0] = replicate_fill(p.fill, es);
   d->fill[1] = (es == 16) ? 0 : d->fill[0];
@@ -394,6 +396,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     memset(d, 0, sizeof *d);
     d->kind = kDevTranspose;
     d->input = p.src;
+    d->out = p.out;
     d->unit_bytes = es;
     d->tr_unit = ub;
     d->soff = p.srcoff.c0 * es;
@@ -674,6 +677,13 @@ struct PlanCtx {
   amap_plan_t *pl;
 };
 
+// bytes of the tensor piece q writes: the stage's temporary, or the piece's own output in the final stage
+static int64_t piece_out_bytes(const PlanCtx &c, int stage, size_t q) {
+  const StageInfo &st = c.m.stages[stage];
+  if (st.dst_temp >= 0 || c.m.out_numels.empty()) return st.numel * c.es;
+  return c.m.out_numels[c.m.pieces[q].out] * c.es;
+}
+
 static int plan_fail(int rc, size_t piece) {
   if (log_enabled()) fprintf(stderr, "[amap] planning piece %zu failed (%d)\n", piece, rc);
   return rc;
@@ -694,7 +704,6 @@ static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
 static int plan_stage_transposes(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
-  const int64_t out_bytes = st.numel * c.es;
   for (int access : {16, 8, 4, 2, 0, -1})
     for (int wide = 0; wide < 2; ++wide) {
       Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
@@ -703,7 +712,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
       for (size_t q = q_lo; q < q_hi; ++q) {
         if (!c.is_tr[q] || c.tr[q].tr_unit != access) continue;
         const DevPiece &d = c.tr[q];
-        const int64_t in_bytes = c.slot_numel[d.input] * c.es;
+        const int64_t in_bytes = c.slot_numel[d.input] * c.es, out_bytes = piece_out_bytes(c, stage, q);
         const bool needs_wide = (in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) && access > 0;
         if ((int)needs_wide != wide) continue;
         if (!check_transpose_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
@@ -724,7 +733,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
         DevPiece d;
         if (build_affine_piece(p, c.es, 16, &d) != AMAP_OK || d.n_items == 0) continue;
         make_strip(&d);
-        if (!check_affine_piece(d, 0, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
+        if (!check_affine_piece(d, 0, piece_out_bytes(c, stage, q))) return plan_fail(AMAP_EOVERFLOW, q);
         fills.push_back(d);
         taken.push_back(q);
       }
@@ -742,7 +751,6 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
 static int plan_stage_strips(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
-  const int64_t out_bytes = st.numel * c.es;
   for (int V = 16; V >= 1; V >>= 1)
     for (int cons : {0, 2, kDevMaxCons})
       for (int wide = 0; wide < 2; ++wide)
@@ -753,7 +761,7 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
             const Piece &p = c.m.pieces[q];
             const int n_cons = (int)(p.guards.size() + p.domain.size());
             if ((n_cons == 0 ? 0 : n_cons <= 2 ? 2 : kDevMaxCons) != cons) continue;
-            const int64_t in_bytes = (p.src >= 0) ? c.slot_numel[p.src] * c.es : 0;
+            const int64_t in_bytes = (p.src >= 0) ? c.slot_numel[p.src] * c.es : 0, out_bytes = piece_out_bytes(c, stage, q);
             if ((int)(in_bytes >= (1ll << 32) || out_bytes >= (1ll << 32)) != wide) continue;
             DevPiece d;
             const int rc = build_affine_piece(p, c.es, V, &d);
@@ -783,7 +791,7 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
 static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts, bool allow_slabs, amap_plan_t **out_plan);
 
 static void plan_slabs(const Map &m, int device, const amap_plan_opts &o, amap_plan_t *pl) {
-  if (m.stages.size() != 1 || m.pieces.empty() || m.out_numel == 0) return;
+  if (m.stages.size() != 1 || m.pieces.empty() || m.out_numel == 0 || m.out_numels.size() > 1) return;
   const int64_t N = m.pieces[0].n() > 0 ? m.pieces[0].ext[0] : 0;
   if (N < 2 || m.out_numel % N) return;
   const int64_t DS = m.out_numel / N;
@@ -816,6 +824,7 @@ static void plan_slabs(const Map &m, int device, const amap_plan_opts &o, amap_p
   sub.m.domain_views.clear();
   for (Piece &p : sub.m.pieces) p.ext[0] = per;
   sub.m.out_numel = DS * per;
+  sub.m.out_numels = {sub.m.out_numel};
   sub.m.stages[0].numel = sub.m.out_numel;
   for (size_t q = 0; q < m.in_numel.size(); ++q) sub.m.in_numel[q] = m.in_numel[q] / N * per;
   if ((sub.m.out_numel * es) % pl->pointer_align) return;
@@ -861,6 +870,11 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
   pl->pdl = !(o.flags & AMAP_PLAN_NO_PDL);
   pl->in_numel = m.in_numel;
   pl->out_numel = m.out_numel;
+  pl->out_numels = m.out_numels.empty() ? std::vector<int64_t>{m.out_numel} : m.out_numels;
+  if ((int)pl->out_numels.size() > kMaxOutputs) {
+    delete pl;
+    return AMAP_EUNSUPPORTED;
+  }
   pl->temp_numel = m.temp_numel;
   for (const StageInfo &st : m.stages) pl->stage_dst.push_back(st.dst_temp);
   memset(&pl->stats, 0, sizeof pl->stats);
@@ -1121,33 +1135,50 @@ static cudaError_t enqueue(const DescSource &ds, const Launch &L, const PtrTable
   return cudaGetLastError();
 }
 
-// Argument checks shared by amap_execute and amap_execute_static: null pointers, alignment to the plan's
-// pointer_align, and no overlap between any source's byte range and the destination's.  Fills pt->src for the
-// external inputs.
-static int bind_buffers(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, PtrTable *pt) {
+// Argument checks shared by the execute entry points: null pointers, alignment to the plan's pointer_align, and no
+// overlap between the byte ranges of any two buffers of which one is written.  Fills pt->src for the external
+// inputs and pt->dst for the outputs.
+static int bind_buffers(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *const *dst_dev_ptrs, PtrTable *pt) {
   if (!src_dev_ptrs && !plan->in_numel.empty()) return AMAP_EINVAL;
-  if (!dst_dev_ptr) return AMAP_EINVAL;
+  if (!dst_dev_ptrs) return AMAP_EINVAL;
   memset(pt, 0, sizeof *pt);
   const uintptr_t mask = (uintptr_t)plan->pointer_align - 1;
-  const uintptr_t d0 = (uintptr_t)dst_dev_ptr, d1 = d0 + (uintptr_t)plan->out_numel * plan->elem_size;
+  const size_t n_out = plan->out_numels.size();
+  for (size_t k = 0; k < n_out; ++k) {
+    if (!dst_dev_ptrs[k] && plan->out_numels[k] > 0) return AMAP_EINVAL;
+    const uintptr_t d0 = (uintptr_t)dst_dev_ptrs[k], d1 = d0 + (uintptr_t)plan->out_numels[k] * plan->elem_size;
+    if (d0 & mask) return AMAP_EALIGN;
+    for (size_t j = 0; j < k; ++j) {  // two outputs must not overlap either
+      const uintptr_t e0 = (uintptr_t)dst_dev_ptrs[j], e1 = e0 + (uintptr_t)plan->out_numels[j] * plan->elem_size;
+      if (d0 < e1 && e0 < d1) return AMAP_EINVAL;
+    }
+    pt->dst[k] = (char *)dst_dev_ptrs[k];
+  }
   for (size_t q = 0; q < plan->in_numel.size(); ++q) {
     if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
     if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
     const uintptr_t s0 = (uintptr_t)src_dev_ptrs[q], s1 = s0 + (uintptr_t)plan->in_numel[q] * plan->elem_size;
-    if (s0 < d1 && d0 < s1) return AMAP_EINVAL;  // source and destination ranges must not overlap
+    for (size_t k = 0; k < n_out; ++k) {  // source and destination ranges must not overlap
+      const uintptr_t d0 = (uintptr_t)dst_dev_ptrs[k], d1 = d0 + (uintptr_t)plan->out_numels[k] * plan->elem_size;
+      if (s0 < d1 && d0 < s1) return AMAP_EINVAL;
+    }
     pt->src[q] = (const char *)src_dev_ptrs[q];
   }
-  if (d0 & mask) return AMAP_EALIGN;
-  pt->dst = (char *)dst_dev_ptr;
   return AMAP_OK;
 }
 
-extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
-                            void *cuda_stream) {
+static bool nothing_to_write(const amap_plan_t *plan) {
+  for (int64_t n : plan->out_numels)
+    if (n > 0) return false;
+  return true;
+}
+
+extern "C" int amap_execute_multi(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *const *dst_dev_ptrs,
+                                  void *cuda_stream) {
   if (!plan || plan->device < 0) return AMAP_EINVAL;
-  if (plan->out_numel == 0) return AMAP_OK;
+  if (nothing_to_write(plan)) return AMAP_OK;
   PtrTable pt;
-  const int brc = bind_buffers(plan, src_dev_ptrs, dst_dev_ptr, &pt);
+  const int brc = bind_buffers(plan, src_dev_ptrs, dst_dev_ptrs, &pt);
   if (brc != AMAP_OK) return brc;
   const size_t n_in = plan->in_numel.size();
   for (size_t k = 0; k < plan->temps.size(); ++k) pt.src[n_in + k] = (const char *)plan->temps[k];
@@ -1163,17 +1194,28 @@ extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_
     const Launch &L = plan->launches[li];
     const LaunchDesc &ld = plan->launch_desc[li];
     const int t = plan->stage_dst[L.stage];
-    pt.dst = (t < 0) ? (char *)dst_dev_ptr : (char *)plan->temps[t];  // stages run in stream order
+    PtrTable stage_pt = pt;  // stages run in stream order; a stage that writes a temporary has one destination
+    if (t >= 0) stage_pt.dst[0] = (char *)plan->temps[t];
     const DescSource ds{ld.n_pieces > 0 ? &ld : nullptr, plan->dev_table};
-    const cudaError_t e = enqueue(ds, L, pt, s, plan->pdl);
+    const cudaError_t e = enqueue(ds, L, stage_pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
   }
   return AMAP_OK;
 }
 
+extern "C" int amap_execute(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
+                            void *cuda_stream) {
+  if (!plan || plan->out_numels.size() != 1) return AMAP_EINVAL;
+  if (plan->out_numel == 0) return AMAP_OK;
+  if (!dst_dev_ptr) return AMAP_EINVAL;
+  void *dsts[1] = {dst_dev_ptr};
+  return amap_execute_multi(plan, src_dev_ptrs, dsts, cuda_stream);
+}
+
 extern "C" int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void *dst_host_ptr,
                                  void *cuda_stream) {
-  if (!plan || plan->device < 0 || (!src_host_ptrs && !plan->in_numel.empty()) || (!dst_host_ptr && plan->out_numel > 0))
+  if (!plan || plan->device < 0 || plan->out_numels.size() != 1 || (!src_host_ptrs && !plan->in_numel.empty()) ||
+      (!dst_host_ptr && plan->out_numel > 0))
     return AMAP_EINVAL;
   int prev = 0;
   CUDA_TRY(cudaGetDevice(&prev));
@@ -1294,12 +1336,13 @@ static int static_device_sms(int device) {
 
 extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr,
                                    void *cuda_stream) {
-  if (!plan) return AMAP_EINVAL;
+  if (!plan || plan->out_numels.size() != 1) return AMAP_EINVAL;
   if (plan->table.size() > (size_t)kStaticMaxPieces) return AMAP_ETOOLARGE;
   if (!plan->temp_numel.empty()) return AMAP_EUNSUPPORTED;  // temporaries would need device memory
   if (plan->out_numel == 0) return AMAP_OK;
   PtrTable pt;
-  const int brc = bind_buffers(plan, src_dev_ptrs, dst_dev_ptr, &pt);  // the same refusals as amap_execute
+  void *dsts[1] = {dst_dev_ptr};
+  const int brc = bind_buffers(plan, src_dev_ptrs, dsts, &pt);  // the same refusals as amap_execute
   if (brc != AMAP_OK) return brc;
   int device = 0;
   CUDA_TRY(cudaGetDevice(&device));

@@ -278,6 +278,21 @@ def qkv_split(B=16, S=2048, heads=32, D=128, part=0, dtype="bf16") -> Chain:
     )
 
 
+def qkv_split_all(B=16, S=2048, heads=32, D=128, dtype="bf16") -> Chain:
+    """The same cut with all three parts in ONE chain; `meta["outputs"]` names the three results (tensor numbers)."""
+    hd = heads * D
+    ops = []
+    outs = []
+    for part in range(3):
+        base = 1 + len(ops)
+        ops.append({"kind": "split", "src": 0, "axis": 2, "sizes": [hd, hd, hd], "part": part})
+        ops.append({"kind": "reshape", "src": base, "shape": [B, S, heads, D]})
+        ops.append({"kind": "transpose", "src": base + 1, "perm": [0, 2, 1, 3]})
+        outs.append(base + 2)
+    return Chain(name="qkv_split_all", dtype=dtype, inputs=[[B, S, 3 * hd]], ops=ops, values="normal", seed=BASE_SEED + 7,
+                 meta={"outputs": outs})
+
+
 def full_configs() -> dict:
     """The configurations at the sizes the benchmark quotes."""
     return {

@@ -21,9 +21,25 @@ def eval_map(m, inputs):
     pieces = m.pieces()
     result = None
     for first, n_pieces, dst_temp, numel in m.stages():
-        out = np.zeros(numel, dtype=inputs[0].dtype)
+        if dst_temp < 0 and len(m.out_numels) > 1:  # the last stage of a map with several outputs
+            result = [_eval_pieces([p for p in pieces[first : first + n_pieces] if p["output"] == k], n, flat, inputs[0].dtype)
+                      for k, n in enumerate(m.out_numels)]
+            continue
+        out = _eval_pieces(pieces[first : first + n_pieces], numel, flat, inputs[0].dtype)
+        if dst_temp >= 0:
+            assert dst_temp == len(flat) - len(inputs), "temporaries are numbered in the order they are written"
+            flat.append(out)
+        else:
+            result = out
+    assert result is not None and m.stages()[-1][2] == -1
+    return result
+
+
+def _eval_pieces(pieces, numel, flat, dtype):
+    if True:
+        out = np.zeros(numel, dtype=dtype)
         cnt = np.zeros(numel, dtype=np.int32)
-        for p in pieces[first : first + n_pieces]:
+        for p in pieces:
             nl = len(p["bounds"])
             idx = np.indices(p["bounds"], dtype=np.int64).reshape(nl, -1) if nl else np.zeros((0, 1), dtype=np.int64)
 
@@ -51,13 +67,7 @@ def eval_map(m, inputs):
             out[d] = vals
             np.add.at(cnt, d, 1)
         assert (cnt == 1).all(), "the pieces of a stage must write every element exactly once"
-        if dst_temp >= 0:
-            assert dst_temp == len(flat) - len(inputs), "temporaries are numbered in the order they are written"
-            flat.append(out)
-        else:
-            result = out
-    assert result is not None and m.stages()[-1][2] == -1
-    return result
+        return out
 
 
 @pytest.mark.parametrize("name", sorted(W.reduced_configs()))
@@ -375,3 +385,84 @@ def test_strerror_is_distinct_per_code():
     lib.amap_strerror.restype = ctypes.c_char_p
     msgs = {lib.amap_strerror(c) for c in range(0, -11, -1)}
     assert len(msgs) == 11
+
+
+# ---------------------------------------------------------------------------
+# several outputs from one compose, and operators that are not layout operators
+# ---------------------------------------------------------------------------
+def _qkv_chain(Bt=2, S=12, heads=3, D=8):
+    hd = heads * D
+    ops = []
+    for part in range(3):
+        base = 1 + len(ops)
+        ops.append({"kind": "split", "src": 0, "axis": 2, "sizes": [hd, hd, hd], "part": part})
+        ops.append({"kind": "reshape", "src": base, "shape": [Bt, S, heads, D]})
+        ops.append({"kind": "transpose", "src": base + 1, "perm": [0, 2, 1, 3]})
+    return W.Chain(name="qkv", dtype="bf16", inputs=[[Bt, S, 3 * hd]], ops=ops, values="normal"), [3, 6, 9]
+
+
+def test_split_parts_compose_into_one_map_with_three_outputs():
+    chain, outs = _qkv_chain()
+    xs = W.make_inputs(chain)
+    tensors = oracle.run_chain(chain, xs, keep_intermediates=True)
+    m = B.compose_chain(chain, outputs=outs)
+    assert len(m.out_numels) == 3 and len(m.stages()) == 1
+    got = eval_map(m, xs)
+    for k, t in enumerate(outs):
+        assert np.array_equal(got[k], tensors[t].reshape(-1)), k
+    st = m.plan(device=-1).stats()
+    assert st["n_launches"] == 1 and st["n_stages"] == 1  # one launch writes q, k and v
+    assert st["bytes_written"] == sum(m.out_numels) * 2 and st["bytes_read"] == xs[0].nbytes
+
+
+def test_a_tensor_can_be_an_output_and_be_read_again():
+    chain = W.Chain(
+        name="both", dtype="fp32", inputs=[[6, 10]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},                 # 1: [10, 6], an output
+            {"kind": "pad", "src": 1, "lo": [1, 0], "hi": [0, 2]},           # 2: [11, 8], an output too
+            {"kind": "slice", "src": 1, "start": [2, 1], "stop": [9, 6], "step": [3, 2]},  # 3: a third
+        ],
+        values="raw",
+    )
+    xs = W.make_index_tagged_inputs(chain)
+    tensors = oracle.run_chain(chain, xs, keep_intermediates=True)
+    m = B.compose_chain(chain, outputs=[2, 1, 3])  # in the order asked for
+    got = eval_map(m, xs)
+    for k, t in enumerate([2, 1, 3]):
+        assert np.array_equal(got[k], tensors[t].reshape(-1))
+    assert [p["input"] for p in m.pieces() if p["input"] >= 0] == [0] * sum(p["input"] >= 0 for p in m.pieces())
+
+
+def test_outputs_are_validated():
+    b = B.Builder(4)
+    x = b.input([4, 6])
+    y = b.transpose(x, [1, 0])
+    z = b.reshape(y, [3, 8])
+    for outs in ([y, y], [x, y], [], [99], [y] * 9):
+        with pytest.raises(B.AmapError) as e:
+            b.compose_multi(outs)
+        assert e.value.code == -1
+    assert len(b.compose_multi([z, y]).out_numels) == 2
+
+
+def test_composition_stops_at_an_operator_that_is_not_a_layout_operator():
+    """x -> transpose -> [compute operator] -> pad -> transpose.  The statements before the operator compose into its
+    input (asked for as an output), the statements behind it into reads of its result (bound like an input)."""
+    b = B.Builder(2)
+    x = b.input([8, 20])
+    t = b.transpose(b.reshape(x, [8, 4, 5]), [2, 0, 1])        # [5, 8, 4]: what the operator consumes
+    o = b.opaque([t], [5, 8, 4])                                # its result
+    z = b.transpose(b.pad(o, [0, 1, 0], [0, 0, 2]), [1, 0, 2])  # [9, 5, 6]
+    first = b.compose_multi([t])
+    second = b.compose(z)
+    xv = np.arange(160, dtype=np.uint16).reshape(8, 20)
+    tv = eval_map(first, [xv])
+    assert np.array_equal(tv, xv.reshape(8, 4, 5).transpose(2, 0, 1).reshape(-1))
+    ov = (tv.astype(np.uint32) * 3 + 7).astype(np.uint16)      # stands in for the compute operator
+    zv = eval_map(second, [xv, ov])
+    want = np.pad(ov.reshape(5, 8, 4), ((0, 0), (1, 0), (0, 2))).transpose(1, 0, 2)
+    assert np.array_equal(zv, want.reshape(-1))
+    assert all(p["input"] in (1, -1) for p in second.pieces())  # nothing behind the operator reads x
+    # one compose cannot reach through the operator: a map that wants z never reads the transposed tensor
+    assert second.in_numel == [160, 160]

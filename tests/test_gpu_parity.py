@@ -155,6 +155,104 @@ def test_split_parts_each_compose_to_one_copy(B):
         assert np.array_equal(want, x[:, :, part].transpose(0, 2, 1, 3))
 
 
+def test_split_into_three_outputs_is_one_launch(B):
+    """q, k and v cut out of one fused projection and moved to [B, heads, S, D]: ONE composed map with three
+    outputs, one plan, one kernel launch (amap_compose_multi / amap_execute_multi)."""
+    import torch
+
+    Bt, S, heads, D = 2, 40, 3, 16
+    hd = heads * D
+    ops = []
+    for part in range(3):
+        base = 1 + len(ops)
+        ops.append({"kind": "split", "src": 0, "axis": 2, "sizes": [hd, hd, hd], "part": part})
+        ops.append({"kind": "reshape", "src": base, "shape": [Bt, S, heads, D]})
+        ops.append({"kind": "transpose", "src": base + 1, "perm": [0, 2, 1, 3]})
+    chain = W.Chain(name="qkv", dtype="bf16", inputs=[[Bt, S, 3 * hd]], ops=ops, values="normal")
+    outs = [3, 6, 9]
+    xs = W.make_inputs(chain)
+    tensors = oracle.run_chain(chain, xs, keep_intermediates=True)
+    m = B.compose_chain(chain, outputs=outs)
+    plan = m.plan(0)
+    assert plan.stats()["n_launches"] == 1 and plan.stats()["n_stages"] == 1
+    src = torch.from_numpy(xs[0].view(np.int16)).cuda()
+    bands = [torch.full((n + 2 * CANARY,), 0x5A5A, dtype=torch.int16, device="cuda") for n in m.out_numels]
+    dsts = [b[CANARY : CANARY + n] for b, n in zip(bands, m.out_numels)]
+    plan.execute_multi_ptrs([src.data_ptr()], [d.data_ptr() for d in dsts], torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for k, t in enumerate(outs):
+        host = bands[k].cpu().numpy().view(np.uint16)
+        assert (host[:CANARY] == 0x5A5A).all() and (host[-CANARY:] == 0x5A5A).all()
+        assert np.array_equal(host[CANARY:-CANARY], tensors[t].reshape(-1)), k
+    # the single-output entry point refuses this plan; overlapping outputs are refused as well
+    with pytest.raises(B.AmapError) as e:
+        plan.execute_ptrs([src.data_ptr()], dsts[0].data_ptr(), 0)
+    assert e.value.code == -1
+    with pytest.raises(B.AmapError) as e:
+        plan.execute_multi_ptrs([src.data_ptr()], [dsts[0].data_ptr(), dsts[0].data_ptr() + 32, dsts[2].data_ptr()], 0)
+    assert e.value.code == -1
+
+
+def test_outputs_of_different_kernel_families_and_a_tensor_read_again(B):
+    """Three results of one chain: a transposed tensor (tiled transpose kernel), its padded copy (transpose plus
+    fills) and a strided slice of it (gather): each output written by its own pieces, every family indexing its
+    own destination."""
+    import torch
+
+    chain = W.Chain(
+        name="three", dtype="bf16", inputs=[[2, 72, 16, 24]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [0, 2, 3, 1]},                                   # 1: NHWC
+            {"kind": "pad", "src": 1, "lo": [0, 1, 1, 0], "hi": [0, 1, 1, 0]},                        # 2
+            {"kind": "slice", "src": 1, "start": [0, 0, 1, 0], "stop": [2, 16, 24, 72], "step": [1, 2, 3, 1]},  # 3
+        ],
+        values="normal",
+    )
+    xs = W.make_inputs(chain)
+    tensors = oracle.run_chain(chain, xs, keep_intermediates=True)
+    outs = [1, 2, 3]
+    m = B.compose_chain(chain, outputs=outs)
+    plan = m.plan(0)
+    src = torch.from_numpy(xs[0].view(np.int16)).cuda()
+    dsts = [torch.full((n,), 0x1111, dtype=torch.int16, device="cuda") for n in m.out_numels]
+    plan.execute_multi_ptrs([src.data_ptr()], [d.data_ptr() for d in dsts], torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    for k, t in enumerate(outs):
+        assert np.array_equal(dsts[k].cpu().numpy().view(np.uint16), tensors[t].reshape(-1)), k
+
+
+def test_chain_cut_at_an_operator_that_is_not_a_layout_operator(B):
+    """Layout operators on both sides of a compute operator (here: torch adds 1 to every element): the part before
+    it is one composed copy into the operator's input, the part behind it one composed copy of its result."""
+    import torch
+
+    b = B.Builder(2)
+    x = b.input([6, 64, 10])
+    t = b.transpose(x, [2, 0, 1])                                # [10, 6, 64]
+    o = b.opaque([t], [10, 6, 64])
+    z = b.transpose(b.pad(b.reshape(o, [10, 6, 8, 8]), [0, 0, 1, 0], [0, 0, 0, 0]), [1, 0, 3, 2])  # [6, 10, 8, 9]
+    first, second = b.compose_multi([t]), b.compose(z)
+    xv = W.make_values(6 * 64 * 10, "bf16", "normal", np.random.default_rng(7)).reshape(6, 64, 10)
+    xd = torch.from_numpy(xv.view(np.int16)).cuda()
+    td = torch.zeros(first.out_numel, dtype=torch.int16, device="cuda")
+    first.plan(0).execute([xd], td)
+    od = td + 1                                                    # the compute operator, on the same stream
+    zd = torch.zeros(second.out_numel, dtype=torch.int16, device="cuda")
+    second.plan(0).execute([xd, od], zd)
+    torch.cuda.synchronize()
+    # the oracle: chain, operator (numpy), chain
+    c1 = W.Chain(name="a", dtype="bf16", inputs=[[6, 64, 10]], ops=[{"kind": "transpose", "src": 0, "perm": [2, 0, 1]}])
+    tv = oracle.run_chain(c1, [xv])
+    ov = (tv.view(np.int16) + np.int16(1)).view(np.uint16)
+    c2 = W.Chain(name="b", dtype="bf16", inputs=[[10, 6, 64]], ops=[
+        {"kind": "reshape", "src": 0, "shape": [10, 6, 8, 8]},
+        {"kind": "pad", "src": 1, "lo": [0, 0, 1, 0], "hi": [0, 0, 0, 0]},
+        {"kind": "transpose", "src": 2, "perm": [1, 0, 3, 2]},
+    ])
+    want = oracle.run_chain(c2, [ov])
+    assert np.array_equal(zd.cpu().numpy().view(np.uint16), want.reshape(-1))
+
+
 def test_dag_with_a_shared_intermediate(B):
     """One transposed tensor feeds a slice and a pad that are joined again: two readers of one intermediate."""
     chain = W.Chain(
