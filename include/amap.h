@@ -294,7 +294,8 @@ int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
 /* ---------------------------------------------------------------------------
  * amap_execute: the surviving copy (the data movement Section 2.1 cannot
  * remove and Section 2.2 wants run at full memory bandwidth).
- *   src_dev_ptrs  host array of n_inputs DEVICE pointers, in amap_chain.inputs order
+ *   src_dev_ptrs  host array of n_inputs DEVICE pointers, in amap_chain.inputs order (the entry of an input
+ *                 that no piece of the map reads may be NULL)
  *   dst_dev_ptr   DEVICE pointer to the output (out_numel * elem_size bytes)
  *   cuda_stream   a cudaStream_t (NULL = the legacy default stream)
  * Enqueues the plan's kernel(s) -- one per kernel family present in the map,

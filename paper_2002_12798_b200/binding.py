@@ -344,19 +344,25 @@ class Plan:
             out.append(KERNEL_NAMES[kind.value])
         return out
 
+    def _src_array(self, src_ptrs):
+        """n_inputs pointers; inputs left out at the end (not read by this map) are passed as NULL."""
+        n = max(len(self.map.in_numel), len(src_ptrs), 1)
+        ptrs = list(src_ptrs) + [None] * (n - len(src_ptrs))
+        return (c_void_p * n)(*[c_void_p(p) for p in ptrs])
+
     def execute_ptrs(self, src_ptrs, dst_ptr, stream=0):
-        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        arr = self._src_array(src_ptrs)
         _check(_lib.amap_execute(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute")
 
     def execute_multi_ptrs(self, src_ptrs, dst_ptrs, stream=0):
         """amap_execute_multi: one destination pointer per output of the map."""
-        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        arr = self._src_array(src_ptrs)
         darr = (c_void_p * max(len(dst_ptrs), 1))(*[c_void_p(p) for p in dst_ptrs])
         _check(_lib.amap_execute_multi(self._h, arr, darr, c_void_p(stream)), "amap_execute_multi")
 
     def execute_static_ptrs(self, src_ptrs, dst_ptr, stream=0):
         """amap_execute_static: no device allocation; the descriptors go through the library's fixed table."""
-        arr = (c_void_p * max(len(src_ptrs), 1))(*[c_void_p(p) for p in src_ptrs])
+        arr = self._src_array(src_ptrs)
         _check(_lib.amap_execute_static(self._h, arr, c_void_p(dst_ptr), c_void_p(stream)), "amap_execute_static")
 
     def bind(self, srcs, dst, stream=None):
@@ -364,7 +370,7 @@ class Plan:
         Keeps `srcs` and `dst` alive.  For loops that launch the same plan on the same buffers many times."""
         import torch
 
-        arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(t.data_ptr()) for t in srcs])
+        arr = self._src_array([t.data_ptr() for t in srcs])
         if isinstance(dst, (list, tuple)):  # a map with several outputs
             s = (stream or torch.cuda.current_stream(dst[0].device)).cuda_stream
             d = (c_void_p * len(dst))(*[c_void_p(t.data_ptr()) for t in dst])

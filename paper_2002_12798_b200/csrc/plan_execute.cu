@@ -50,6 +50,7 @@ struct amap_plan_t {
   int pointer_align = 0;
   bool pdl = true;  // launch with programmatic stream serialisation
   std::vector<int64_t> in_numel;
+  std::vector<char> in_used;        // per input: some piece reads it (the pointer of an unused input may be null)
   int64_t out_numel = 0;            // output 0
   std::vector<int64_t> out_numels;  // every output
   std::vector<int64_t> temp_numel;  // temporaries between stages
@@ -869,6 +870,9 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
   pl->pointer_align = align;
   pl->pdl = !(o.flags & AMAP_PLAN_NO_PDL);
   pl->in_numel = m.in_numel;
+  pl->in_used.assign(m.in_numel.size(), 0);
+  for (const Piece &p : m.pieces)
+    if (p.src >= 0 && p.src < (int)m.in_numel.size()) pl->in_used[p.src] = 1;
   pl->out_numel = m.out_numel;
   pl->out_numels = m.out_numels.empty() ? std::vector<int64_t>{m.out_numel} : m.out_numels;
   if ((int)pl->out_numels.size() > kMaxOutputs) {
@@ -1155,7 +1159,10 @@ static int bind_buffers(const amap_plan_t *plan, const void *const *src_dev_ptrs
     pt->dst[k] = (char *)dst_dev_ptrs[k];
   }
   for (size_t q = 0; q < plan->in_numel.size(); ++q) {
-    if (!src_dev_ptrs[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
+    if (!src_dev_ptrs[q]) {  // allowed for an input that no piece of this map reads
+      if (plan->in_used[q] && plan->in_numel[q] > 0) return AMAP_EINVAL;
+      continue;
+    }
     if ((uintptr_t)src_dev_ptrs[q] & mask) return AMAP_EALIGN;
     const uintptr_t s0 = (uintptr_t)src_dev_ptrs[q], s1 = s0 + (uintptr_t)plan->in_numel[q] * plan->elem_size;
     for (size_t k = 0; k < n_out; ++k) {  // source and destination ranges must not overlap
