@@ -389,6 +389,39 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
     return out
 
 
+def consumer_rows(torch, B, device, stream, l2, names=("c5", "c3"), flags=0, reps=10):
+    """The composed map handed to the CONSUMER instead of being run as a copy: a row-sum kernel that reads the
+    inputs through the map, against the same kernel reading a materialised result (copy first, then reduce)."""
+    out = {}
+    configs = bench_configs()
+    for name in names:
+        case = Case(torch, B, configs[name], device, stream, l2, flags)
+        m, es, n_sets = case.maps[0], case.es, case.n_sets
+        rows = {"c5": m.out_numel // (9 * 128), "c3": m.out_numel // 128}.get(name, m.out_numel // 128)
+        cols = m.out_numel // rows
+        sums = [torch.empty(rows, dtype=torch.int32, device=device) for _ in range(n_sets)]
+        fused = [m.bind_consume_row_sums(case.ins[i], rows, cols, sums[i], stream) for i in range(n_sets)]
+        ident = B.compose_chain(plain_copy_chain(m.out_numel, case.chain.dtype))
+        reduce_ = [ident.bind_consume_row_sums([case.outs[i][0]], rows, cols, sums[i], stream) for i in range(n_sets)]
+        copy_then = [lambda i=i: (case.calls[i](), reduce_[i]()) for i in range(n_sets)]
+        st = case.stats[0]
+        fused_bytes = st["bytes_read"] + 4 * rows
+        unfused_bytes = st["bytes_read"] + 2 * st["bytes_written"] + 4 * rows
+        f = measure_calls(torch, fused, stream, fused_bytes, device.index, reps=reps, max_launches=1000)
+        ref = sums[0].clone()
+        u = measure_calls(torch, copy_then, stream, unfused_bytes, device.index, reps=reps, max_launches=1000)
+        out[name] = {
+            "what": "uint32 row sums of the chain's result [%d, %d]" % (rows, cols),
+            "through_the_map": {"us": f["us"], "bytes_moved": fused_bytes},
+            "copy_then_reduce": {"us": u["us"], "bytes_moved": unfused_bytes},
+            "speedup": round(u["us"] / f["us"], 2),
+            "same_sums": bool(torch.equal(ref, sums[0])),
+        }
+        del case, sums, fused, reduce_, copy_then
+        torch.cuda.empty_cache()
+    return out
+
+
 def oracle_row(oracle, chain, xs, total_bytes, gpu_out):
     """The oracle on one configuration: single thread and all cores, its output compared with the GPU's."""
     cores = os.cpu_count() or 1
@@ -629,6 +662,7 @@ def run_ours(args):
         if not args.no_table:
             line["configs"] = config_rows(torch, B, device, stream, l2, peak, names, flags=args.plan_flags,
                                           extras=args.all_configs, oracle=oracle, reps=max(10, args.reps))
+            line["consumer"] = consumer_rows(torch, B, device, stream, l2, flags=args.plan_flags, reps=max(10, args.reps))
     if rank == 0:
         print(json.dumps(line))
     if world > 1:

@@ -370,6 +370,31 @@ int amap_execute_host(amap_plan_t *plan, const void *const *src_host_ptrs, void 
  * ------------------------------------------------------------------------- */
 int amap_execute_static(const amap_plan_t *plan, const void *const *src_dev_ptrs, void *dst_dev_ptr, void *cuda_stream);
 
+/* ---------------------------------------------------------------------------
+ * Handing the composed map to the consumer (Section 2.2: make an operator's
+ * data lie where the next operator needs it, so that no copy runs between
+ * them).  amap_map_device_view flattens a map into the plain struct of
+ * amap_device.h, which a CUDA kernel takes by value and reads through with
+ * amap_view_locate(): the result tensor of the chain is never materialised.
+ * Only maps with one stage and one output, at most AMAP_VIEW_MAX_PIECES
+ * pieces of at most AMAP_VIEW_MAX_LOOPS loops and AMAP_VIEW_MAX_CONS
+ * constraints each, qualify (AMAP_ETOOLARGE / AMAP_EUNSUPPORTED otherwise).
+ * `out` is a host pointer to a caller-owned struct; no CUDA call is made.
+ * ------------------------------------------------------------------------- */
+struct amap_device_view;
+int amap_map_device_view(const amap_map *map, struct amap_device_view *out);
+
+/* A demonstration consumer: the sums of the rows of the chain's RESULT, seen as a rows x cols matrix of unsigned
+ * integers of elem_size (1, 2 or 4) bytes, added modulo 2^32 -- computed by a kernel that reads the external inputs
+ * through the view, without the result ever being written (for an im2col map this is a box filter that touches
+ * only the image).  rows * cols must equal the view's out_numel.
+ *   view          host pointer (copied into the kernel's parameters)
+ *   src_dev_ptrs  host array of the view's n_inputs DEVICE pointers (16-byte aligned)
+ *   sums_dev      DEVICE pointer to rows uint32 values
+ * Enqueues one kernel on cuda_stream of the current device and returns without synchronising or allocating. */
+int amap_consume_row_sums(const struct amap_device_view *view, const void *const *src_dev_ptrs, int64_t rows,
+                          int64_t cols, uint32_t *sums_dev, void *cuda_stream);
+
 const char *amap_strerror(int code);
 /* text of the last CUDA error seen by this thread in this library ("" if none) */
 const char *amap_last_cuda_error(void);

@@ -1,0 +1,121 @@
+/*
+ * amap_device.h -- reading THROUGH a composed map instead of running the copy.
+ *
+ * Section 2.2 of the paper wants the output of an operator to land where the
+ * next operator needs it, so that no copy runs in between.  On a GPU the same
+ * end is reached from the consumer's side: the kernel that would read the
+ * result of a layout chain is handed the composed access map g' (Section 2.1,
+ * equation (2)) and loads every element it wants straight from the external
+ * input -- the "result" tensor never exists.
+ *
+ * amap_map_device_view() (amap.h) flattens a composed, single-stage,
+ * single-output map into the plain struct below, small enough to be passed to
+ * a kernel by value.  amap_view_locate() is the functor: output element index
+ * -> (input, source element index) or the fill value.
+ *
+ * The header is plain C for the struct and CUDA C++ (under __CUDACC__) for the
+ * device function; it has no dependency on the library's internals.
+ */
+#ifndef AMAP_DEVICE_H_
+#define AMAP_DEVICE_H_
+
+#include <stdint.h>
+
+#define AMAP_VIEW_MAX_PIECES 8
+#define AMAP_VIEW_MAX_LOOPS 8
+#define AMAP_VIEW_MAX_CONS 4
+
+/* 0 <= offset + sum_k coef[k] * i_k < extent */
+typedef struct amap_view_con {
+  int64_t coef[AMAP_VIEW_MAX_LOOPS];
+  int64_t offset, extent;
+} amap_view_con;
+
+/* One piece: out.flat[b_s + sum dst_stride[k] i_k] = in[input].flat[b_l + sum src_stride[k] i_k] over the box
+ * 0 <= i_k < ext[k].  Loops are ordered by destination stride, largest first; destination strides are positive
+ * and nested (each exceeds everything the loops after it can add up to), so an output index decodes into loop
+ * indices digit by digit. */
+typedef struct amap_view_piece {
+  int32_t n_loops;
+  int32_t input;    /* slot of the external input read, -1: the piece stores fill_bits */
+  int32_t n_guards; /* cons[0 .. n_guards): where one fails the element is fill_bits   */
+  int32_t n_domain; /* cons[n_guards .. n_guards + n_domain): where one fails the point is not this piece's */
+  int64_t ext[AMAP_VIEW_MAX_LOOPS];
+  int64_t dst_stride[AMAP_VIEW_MAX_LOOPS];
+  int64_t src_stride[AMAP_VIEW_MAX_LOOPS];
+  int64_t b_s, b_l;
+  uint64_t fill_bits;
+  amap_view_con cons[AMAP_VIEW_MAX_CONS];
+} amap_view_piece;
+
+typedef struct amap_device_view {
+  int32_t n_pieces;
+  int32_t elem_size;
+  int32_t n_inputs;
+  int32_t reserved;
+  int64_t out_numel;
+  amap_view_piece piece[AMAP_VIEW_MAX_PIECES];
+} amap_device_view;
+
+/* where an output element comes from */
+typedef struct amap_view_source {
+  int32_t input;     /* slot of the external input, or -1: the element is `fill_bits` */
+  int64_t index;     /* element index within that input (flat, row-major)             */
+  int64_t run;       /* this and the next run-1 output elements come from consecutive source elements of the same
+                        input (or are all fill): a consumer may fetch them with one vector load */
+  uint64_t fill_bits;
+} amap_view_source;
+
+#ifdef __CUDACC__
+/* Output element `o` (0 <= o < out_numel) -> its source.  Returns false if no piece covers o (cannot happen for a
+ * view made by amap_map_device_view: the pieces of a composed map cover the output exactly once). */
+__host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int64_t o, amap_view_source *out) {
+  for (int p = 0; p < v.n_pieces; ++p) {
+    const amap_view_piece &pc = v.piece[p];
+    int64_t rem = o - pc.b_s;
+    if (rem < 0) continue;
+    int64_t idx[AMAP_VIEW_MAX_LOOPS];
+    bool inside = true;
+    for (int k = 0; k < pc.n_loops; ++k) {
+      /* 32-bit division where the values allow it: far cheaper on the device */
+      const int64_t d = pc.dst_stride[k];
+      const int64_t i = (rem < 0x7fffffffLL) ? (int64_t)((uint32_t)rem / (uint32_t)d) : rem / d;
+      if (i >= pc.ext[k]) {
+        inside = false;
+        break;
+      }
+      idx[k] = i;
+      rem -= i * d;
+    }
+    if (!inside || rem != 0) continue;
+    bool load = pc.input >= 0;
+    const int nc = pc.n_guards + pc.n_domain;
+    for (int c = 0; c < nc; ++c) {
+      int64_t e = pc.cons[c].offset;
+      for (int k = 0; k < pc.n_loops; ++k) e += pc.cons[c].coef[k] * idx[k];
+      const bool ok = e >= 0 && e < pc.cons[c].extent;
+      if (c < pc.n_guards) load = load && ok;
+      else inside = inside && ok;
+    }
+    if (!inside) continue;
+    int64_t s = pc.b_l;
+    for (int k = 0; k < pc.n_loops; ++k) s += pc.src_stride[k] * idx[k];
+    out->input = load ? pc.input : -1;
+    out->index = load ? s : 0;
+    out->fill_bits = pc.fill_bits;
+    /* the innermost loop is a run when it is contiguous on both sides and no constraint looks at it */
+    int64_t run = 1;
+    if (pc.n_loops > 0) {
+      const int in = pc.n_loops - 1;
+      bool plain = pc.dst_stride[in] == 1 && (pc.input < 0 || pc.src_stride[in] == 1);
+      for (int c = 0; c < nc && plain; ++c) plain = pc.cons[c].coef[in] == 0;
+      if (plain) run = pc.ext[in] - idx[in];
+    }
+    out->run = run;
+    return true;
+  }
+  return false;
+}
+#endif /* __CUDACC__ */
+
+#endif /* AMAP_DEVICE_H_ */

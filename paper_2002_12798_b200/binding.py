@@ -27,7 +27,7 @@ EXPORTS = [
     "amap_builder_window", "amap_builder_window_ex", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
     "amap_builder_stmt",
     "amap_builder_opaque", "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_compose_multi",
-    "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
+    "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_device_view", "amap_consume_row_sums", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
@@ -63,6 +63,29 @@ class _Piece(Structure):
         ("b_l", c_int64), ("C_s", POINTER(c_int64)), ("b_s", c_int64), ("n_guards", c_int32),
         ("guards", POINTER(_Constraint)), ("n_domain", c_int32), ("domain", POINTER(_Constraint)),
         ("fill_bits", c_uint64), ("output", c_int32),
+    ]
+
+
+VIEW_MAX_PIECES, VIEW_MAX_LOOPS, VIEW_MAX_CONS = 8, 8, 4
+
+
+class _ViewCon(Structure):
+    _fields_ = [("coef", c_int64 * VIEW_MAX_LOOPS), ("offset", c_int64), ("extent", c_int64)]
+
+
+class _ViewPiece(Structure):
+    _fields_ = [
+        ("n_loops", c_int32), ("input", c_int32), ("n_guards", c_int32), ("n_domain", c_int32),
+        ("ext", c_int64 * VIEW_MAX_LOOPS), ("dst_stride", c_int64 * VIEW_MAX_LOOPS), ("src_stride", c_int64 * VIEW_MAX_LOOPS),
+        ("b_s", c_int64), ("b_l", c_int64), ("fill_bits", c_uint64), ("cons", _ViewCon * VIEW_MAX_CONS),
+    ]
+
+
+class DeviceView(Structure):
+    """amap_device_view (include/amap_device.h): the composed map as a plain struct a kernel takes by value."""
+    _fields_ = [
+        ("n_pieces", c_int32), ("elem_size", c_int32), ("n_inputs", c_int32), ("reserved", c_int32),
+        ("out_numel", c_int64), ("piece", _ViewPiece * VIEW_MAX_PIECES),
     ]
 
 
@@ -304,6 +327,42 @@ class Map:
             _check(_lib.amap_map_get_stage(self._h, s, byref(fp), byref(np_), byref(dt), byref(ne)), "amap_map_get_stage")
             out.append((fp.value, np_.value, dt.value, ne.value))
         return out
+
+    def device_view(self) -> DeviceView:
+        """amap_map_device_view: the map flattened for a consumer kernel that reads through it."""
+        v = DeviceView()
+        _check(_lib.amap_map_device_view(self._h, byref(v)), "amap_map_device_view")
+        return v
+
+    def consume_row_sums(self, srcs, rows, cols, sums, stream=None):
+        """amap_consume_row_sums: uint32 sums of the rows of the chain's result, read through the map from the
+        inputs (CUDA tensors `srcs`); `sums`: a CUDA int32/uint32 tensor of `rows` elements."""
+        import torch
+
+        v = self.device_view()
+        arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(t.data_ptr()) for t in srcs])
+        s = (stream or torch.cuda.current_stream(sums.device)).cuda_stream
+        _check(
+            _lib.amap_consume_row_sums(byref(v), arr, c_int64(rows), c_int64(cols), c_void_p(sums.data_ptr()), c_void_p(s)),
+            "amap_consume_row_sums",
+        )
+
+    def bind_consume_row_sums(self, srcs, rows, cols, sums, stream=None):
+        """consume_row_sums with the arguments marshalled once; the returned callable only makes the C call."""
+        import torch
+
+        v = self.device_view()
+        arr = (c_void_p * max(len(srcs), 1))(*[c_void_p(t.data_ptr()) for t in srcs])
+        s = c_void_p((stream or torch.cuda.current_stream(sums.device)).cuda_stream)
+        vp, r, c, d, fn = byref(v), c_int64(rows), c_int64(cols), c_void_p(sums.data_ptr()), _lib.amap_consume_row_sums
+
+        def call():
+            rc = fn(vp, arr, r, c, d, s)
+            if rc != 0:
+                raise AmapError(rc, "amap_consume_row_sums")
+
+        call.keep = (v, list(srcs), sums, self)
+        return call
 
     def plan(self, device=0, force_kernel=KERNEL_AUTO, pointer_align=16, flags=0) -> "Plan":
         opts = _PlanOpts()

@@ -28,6 +28,7 @@
 #include <numeric>
 
 #include "amap_internal.hpp"
+#include "amap_device.h"
 
 namespace amap {
 
@@ -851,6 +852,50 @@ extern "C" int amap_map_sizes(const amap_map *map, int32_t *n_inputs, int64_t *i
     for (size_t q = 0; q < map->m.in_numel.size(); ++q) in_numel[q] = map->m.in_numel[q];
   if (out_numel) *out_numel = map->m.out_numel;
   if (elem_size) *elem_size = map->m.elem_size;
+  return AMAP_OK;
+}
+
+extern "C" int amap_map_device_view(const amap_map *map, amap_device_view *out) {
+  if (!map || !out) return AMAP_EINVAL;
+  const Map &m = map->m;
+  if (m.stages.size() != 1 || m.out_numels.size() > 1) return AMAP_EUNSUPPORTED;
+  if (m.pieces.size() > (size_t)AMAP_VIEW_MAX_PIECES) return AMAP_ETOOLARGE;
+  memset(out, 0, sizeof *out);
+  out->n_pieces = (int32_t)m.pieces.size();
+  out->elem_size = m.elem_size;
+  out->n_inputs = (int32_t)m.in_numel.size();
+  out->out_numel = m.out_numel;
+  for (size_t q = 0; q < m.pieces.size(); ++q) {
+    const Piece &p = m.pieces[q];
+    amap_view_piece &v = out->piece[q];
+    if (p.n() > AMAP_VIEW_MAX_LOOPS || p.guards.size() + p.domain.size() > (size_t)AMAP_VIEW_MAX_CONS) return AMAP_ETOOLARGE;
+    // canonical pieces have positive destination strides in descending order; decoding an output index digit by
+    // digit also needs them nested
+    for (int k = 0; k < p.n(); ++k)
+      if (p.dst.c[k] <= 0 || (k > 0 && p.dst.c[k] > p.dst.c[k - 1])) return AMAP_EUNSUPPORTED;
+    if (!nested_strides(p.dst.c, p.ext)) return AMAP_EUNSUPPORTED;
+    v.n_loops = p.n();
+    v.input = p.src;
+    v.n_guards = (int32_t)p.guards.size();
+    v.n_domain = (int32_t)p.domain.size();
+    v.b_s = p.dst.c0;
+    v.b_l = p.src == AMAP_CONST ? 0 : p.srcoff.c0;
+    v.fill_bits = p.fill;
+    for (int k = 0; k < p.n(); ++k) {
+      v.ext[k] = p.ext[k];
+      v.dst_stride[k] = p.dst.c[k];
+      v.src_stride[k] = p.src == AMAP_CONST ? 0 : p.srcoff.c[k];
+    }
+    int c = 0;
+    auto put = [&](const Con &g) {
+      for (int k = 0; k < p.n(); ++k) v.cons[c].coef[k] = g.e.c[k];
+      v.cons[c].offset = g.e.c0;
+      v.cons[c].extent = g.extent;
+      ++c;
+    };
+    for (auto &g : p.guards) put(g);
+    for (auto &g : p.domain) put(g);
+  }
   return AMAP_OK;
 }
 

@@ -466,3 +466,70 @@ def test_composition_stops_at_an_operator_that_is_not_a_layout_operator():
     assert all(p["input"] in (1, -1) for p in second.pieces())  # nothing behind the operator reads x
     # one compose cannot reach through the operator: a map that wants z never reads the transposed tensor
     assert second.in_numel == [160, 160]
+
+
+# ---------------------------------------------------------------------------
+# the map flattened for a consumer kernel (include/amap_device.h)
+# ---------------------------------------------------------------------------
+def eval_view(v, inputs):
+    """What amap_view_locate computes, for every output index at once: decode the index into a piece's loop indices
+    digit by digit, check the constraints, follow the source strides."""
+    flat = [x.reshape(-1) for x in inputs]
+    o = np.arange(v.out_numel, dtype=np.int64)
+    out = np.zeros(v.out_numel, dtype=inputs[0].dtype)
+    hit = np.zeros(v.out_numel, dtype=np.int32)
+    for q in range(v.n_pieces):
+        pc = v.piece[q]
+        rem = o - pc.b_s
+        ok = rem >= 0
+        idx = []
+        for k in range(pc.n_loops):
+            i = np.where(ok, rem // pc.dst_stride[k], 0)
+            ok &= i < pc.ext[k]
+            idx.append(i)
+            rem = rem - i * pc.dst_stride[k]
+        ok &= rem == 0
+        load = np.full(v.out_numel, pc.input >= 0)
+        for c in range(pc.n_guards + pc.n_domain):
+            e = np.full(v.out_numel, pc.cons[c].offset, dtype=np.int64)
+            for k in range(pc.n_loops):
+                e += pc.cons[c].coef[k] * idx[k]
+            good = (e >= 0) & (e < pc.cons[c].extent)
+            if c < pc.n_guards:
+                load &= good
+            else:
+                ok &= good
+        s = np.full(v.out_numel, pc.b_l, dtype=np.int64)
+        for k in range(pc.n_loops):
+            s += pc.src_stride[k] * idx[k]
+        take = ok & load
+        if pc.input >= 0:
+            out[take] = flat[pc.input][s[take]]
+        out[ok & ~load] = pc.fill_bits
+        hit += ok
+    assert (hit == 1).all(), "every output index must decode into exactly one piece"
+    return out
+
+
+@pytest.mark.parametrize("name", ["c1", "c2_fwd", "c2_inv_odd_f32", "c3", "c3_odd", "c4", "c4_odd", "c5", "c5_odd", "c5_dil2", "c5_crs"])
+def test_device_view_reproduces_the_chain(name):
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    m = B.compose_chain(chain)
+    v = m.device_view()
+    assert v.out_numel == m.out_numel and v.elem_size == chain.elem_size and v.n_inputs == len(xs)
+    assert np.array_equal(eval_view(v, xs), want.reshape(-1))
+
+
+def test_device_view_refuses_what_it_cannot_hold():
+    b = B.Builder(2)
+    ids = [b.input([4, 8]) for _ in range(5)]
+    m = b.compose(b.concat([b.pad(t, [1, 1], [1, 1]) for t in ids], 0))  # far more than 8 pieces
+    with pytest.raises(B.AmapError) as e:
+        m.device_view()
+    assert e.value.code == -11
+    chain, outs = _qkv_chain()
+    with pytest.raises(B.AmapError) as e:
+        B.compose_chain(chain, outputs=outs).device_view()  # several outputs
+    assert e.value.code == -9

@@ -253,6 +253,28 @@ def test_chain_cut_at_an_operator_that_is_not_a_layout_operator(B):
     assert np.array_equal(zd.cpu().numpy().view(np.uint16), want.reshape(-1))
 
 
+@pytest.mark.parametrize("name,rows", [("c5", None), ("c5_odd", None), ("c3", 2 * 3 * 100), ("c4_odd", 3 * 9 * 11), ("c1", 64),
+                                       ("c2_inv_odd_u8", 2 * 64), ("c2_fwd_f32", 2 * 13 * 12)])
+def test_consumer_reads_through_the_map(B, name, rows):
+    """amap_consume_row_sums: the row sums of the chain's result, computed from the inputs through the composed map
+    (the result is never written), against the sums of the oracle's result."""
+    import torch
+
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    rows = rows or want.shape[0]
+    cols = want.size // rows
+    m = B.compose_chain(chain)
+    es = chain.elem_size
+    dev = [torch.from_numpy(np.ascontiguousarray(x).view(SIGNED[es])).cuda() for x in xs]
+    sums = torch.full((rows,), -1, dtype=torch.int32, device="cuda")
+    m.consume_row_sums(dev, rows, cols, sums)
+    torch.cuda.synchronize()
+    want_sums = want.reshape(rows, cols).astype(np.uint64).sum(axis=1).astype(np.uint32)
+    assert np.array_equal(sums.cpu().numpy().view(np.uint32), want_sums)
+
+
 def test_dag_with_a_shared_intermediate(B):
     """One transposed tensor feeds a slice and a pad that are joined again: two readers of one intermediate."""
     chain = W.Chain(
