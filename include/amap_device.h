@@ -46,13 +46,18 @@ typedef struct amap_view_piece {
   int64_t b_s, b_l;
   uint64_t fill_bits;
   amap_view_con cons[AMAP_VIEW_MAX_CONS];
+  /* 32-bit fast path (amap_device_view.small): division by dst_stride[k] as multiply-and-shift,
+   * q = (t + ((n - t) >> sh1)) >> sh2 with t = mulhi(mul, n)  (Granlund & Montgomery 1994, round-up form) */
+  uint32_t fd_mul[AMAP_VIEW_MAX_LOOPS];
+  uint8_t fd_sh1[AMAP_VIEW_MAX_LOOPS], fd_sh2[AMAP_VIEW_MAX_LOOPS];
 } amap_view_piece;
 
 typedef struct amap_device_view {
   int32_t n_pieces;
   int32_t elem_size;
   int32_t n_inputs;
-  int32_t reserved;
+  int32_t small;    /* 1: every index, offset and partial sum of the map fits 31 bits: amap_view_locate computes in
+                       32-bit arithmetic with the precomputed divisions */
   int64_t out_numel;
   amap_view_piece piece[AMAP_VIEW_MAX_PIECES];
 } amap_device_view;
@@ -68,48 +73,88 @@ typedef struct amap_view_source {
 
 #ifdef __CUDACC__
 /* Output element `o` (0 <= o < out_numel) -> its source.  Returns false if no piece covers o (cannot happen for a
- * view made by amap_map_device_view: the pieces of a composed map cover the output exactly once). */
+ * view made by amap_map_device_view: the pieces of a composed map cover the output exactly once).  One pass over the
+ * piece's loops decodes the index digit by digit and accumulates the source offset and every constraint on the way,
+ * so no per-loop value has to be kept. */
 __host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int64_t o, amap_view_source *out) {
   for (int p = 0; p < v.n_pieces; ++p) {
     const amap_view_piece &pc = v.piece[p];
-    int64_t rem = o - pc.b_s;
-    if (rem < 0) continue;
-    int64_t idx[AMAP_VIEW_MAX_LOOPS];
-    bool inside = true;
-    for (int k = 0; k < pc.n_loops; ++k) {
-      /* 32-bit division where the values allow it: far cheaper on the device */
-      const int64_t d = pc.dst_stride[k];
-      const int64_t i = (rem < 0x7fffffffLL) ? (int64_t)((uint32_t)rem / (uint32_t)d) : rem / d;
-      if (i >= pc.ext[k]) {
-        inside = false;
-        break;
+    const int n = pc.n_loops, nc = pc.n_guards + pc.n_domain;
+    bool inside = true, load = pc.input >= 0;
+    int64_t s, left = 1;  /* left: elements of the innermost loop from this one on */
+    if (o < pc.b_s) continue;
+    if (v.small) {
+      uint32_t rem = (uint32_t)(o - pc.b_s), s32 = (uint32_t)pc.b_l;
+      int32_t e[AMAP_VIEW_MAX_CONS];
+#pragma unroll
+      for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] = c < nc ? (int32_t)pc.cons[c].offset : 0;
+#pragma unroll 1
+      for (int k = 0; k < n; ++k) {
+#ifdef __CUDA_ARCH__
+        const uint32_t t = __umulhi(pc.fd_mul[k], rem);
+#else
+        const uint32_t t = (uint32_t)(((uint64_t)pc.fd_mul[k] * rem) >> 32);
+#endif
+        const uint32_t i = (t + ((rem - t) >> pc.fd_sh1[k])) >> pc.fd_sh2[k];
+        inside = inside && i < (uint32_t)pc.ext[k];
+        rem -= i * (uint32_t)pc.dst_stride[k];
+        s32 += i * (uint32_t)pc.src_stride[k];  /* wrap-around arithmetic: the true value fits 31 bits */
+        if (nc > 0) {
+#pragma unroll
+          for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] += (int32_t)pc.cons[c].coef[k] * (int32_t)i;
+        }
+        if (k == n - 1) left = pc.ext[k] - (int64_t)i;
       }
-      idx[k] = i;
-      rem -= i * d;
+      if (!inside || rem != 0) continue;
+#pragma unroll
+      for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) {
+        if (c < nc) {
+          const bool ok = (uint32_t)e[c] < (uint32_t)pc.cons[c].extent;
+          if (c < pc.n_guards) load = load && ok;
+          else inside = inside && ok;
+        }
+      }
+      if (!inside) continue;
+      s = (int64_t)s32;
+    } else {
+      int64_t rem = o - pc.b_s;
+      int64_t e[AMAP_VIEW_MAX_CONS];
+#pragma unroll
+      for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] = c < nc ? pc.cons[c].offset : 0;
+      s = pc.b_l;
+#pragma unroll 1
+      for (int k = 0; k < n; ++k) {
+        const int64_t i = rem / pc.dst_stride[k];
+        inside = inside && i < pc.ext[k];
+        rem -= i * pc.dst_stride[k];
+        s += i * pc.src_stride[k];
+        if (nc > 0) {
+#pragma unroll
+          for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] += pc.cons[c].coef[k] * i;
+        }
+        if (k == n - 1) left = pc.ext[k] - i;
+      }
+      if (!inside || rem != 0) continue;
+#pragma unroll
+      for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) {
+        if (c < nc) {
+          const bool ok = e[c] >= 0 && e[c] < pc.cons[c].extent;
+          if (c < pc.n_guards) load = load && ok;
+          else inside = inside && ok;
+        }
+      }
+      if (!inside) continue;
     }
-    if (!inside || rem != 0) continue;
-    bool load = pc.input >= 0;
-    const int nc = pc.n_guards + pc.n_domain;
-    for (int c = 0; c < nc; ++c) {
-      int64_t e = pc.cons[c].offset;
-      for (int k = 0; k < pc.n_loops; ++k) e += pc.cons[c].coef[k] * idx[k];
-      const bool ok = e >= 0 && e < pc.cons[c].extent;
-      if (c < pc.n_guards) load = load && ok;
-      else inside = inside && ok;
-    }
-    if (!inside) continue;
-    int64_t s = pc.b_l;
-    for (int k = 0; k < pc.n_loops; ++k) s += pc.src_stride[k] * idx[k];
     out->input = load ? pc.input : -1;
     out->index = load ? s : 0;
     out->fill_bits = pc.fill_bits;
     /* the innermost loop is a run when it is contiguous on both sides and no constraint looks at it */
     int64_t run = 1;
-    if (pc.n_loops > 0) {
-      const int in = pc.n_loops - 1;
+    if (n > 0) {
+      const int in = n - 1;
       bool plain = pc.dst_stride[in] == 1 && (pc.input < 0 || pc.src_stride[in] == 1);
       for (int c = 0; c < nc && plain; ++c) plain = pc.cons[c].coef[in] == 0;
-      if (plain) run = pc.ext[in] - idx[in];
+      if (plain) run = left;
     }
     out->run = run;
     return true;

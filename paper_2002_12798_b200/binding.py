@@ -78,13 +78,15 @@ class _ViewPiece(Structure):
         ("n_loops", c_int32), ("input", c_int32), ("n_guards", c_int32), ("n_domain", c_int32),
         ("ext", c_int64 * VIEW_MAX_LOOPS), ("dst_stride", c_int64 * VIEW_MAX_LOOPS), ("src_stride", c_int64 * VIEW_MAX_LOOPS),
         ("b_s", c_int64), ("b_l", c_int64), ("fill_bits", c_uint64), ("cons", _ViewCon * VIEW_MAX_CONS),
+        ("fd_mul", ctypes.c_uint32 * VIEW_MAX_LOOPS), ("fd_sh1", ctypes.c_uint8 * VIEW_MAX_LOOPS),
+        ("fd_sh2", ctypes.c_uint8 * VIEW_MAX_LOOPS),
     ]
 
 
 class DeviceView(Structure):
     """amap_device_view (include/amap_device.h): the composed map as a plain struct a kernel takes by value."""
     _fields_ = [
-        ("n_pieces", c_int32), ("elem_size", c_int32), ("n_inputs", c_int32), ("reserved", c_int32),
+        ("n_pieces", c_int32), ("elem_size", c_int32), ("n_inputs", c_int32), ("small", c_int32),
         ("out_numel", c_int64), ("piece", _ViewPiece * VIEW_MAX_PIECES),
     ]
 

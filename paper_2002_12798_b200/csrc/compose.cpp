@@ -895,7 +895,32 @@ extern "C" int amap_map_device_view(const amap_map *map, amap_device_view *out) 
     };
     for (auto &g : p.guards) put(g);
     for (auto &g : p.domain) put(g);
+    for (int k = 0; k < p.n(); ++k) {  // division by the destination strides as multiply-and-shift (32-bit path)
+      const uint64_t d = (uint64_t)std::min<int64_t>(p.dst.c[k], 0xFFFFFFFFll);
+      uint32_t l = 0;
+      while (l < 32 && (1ull << l) < d) ++l;
+      v.fd_mul[k] = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+      v.fd_sh1[k] = (uint8_t)(l < 1 ? l : 1);
+      v.fd_sh2[k] = (uint8_t)(l < 1 ? 0 : l - 1);
+    }
   }
+  // The 32-bit path is valid when nothing the functor computes can leave 31 bits: output and input sizes, and the
+  // range of every constraint expression over its piece's box.
+  bool small = m.out_numel < (1ll << 31);
+  for (int64_t n : m.in_numel) small = small && n < (1ll << 31);
+  for (const Piece &p : m.pieces) {
+    auto fits = [&](const Aff &a) {
+      int64_t lo, hi;
+      aff_range(a, p.ext, &lo, &hi);
+      __int128 span = std::llabs(a.c0);
+      for (int k = 0; k < p.n(); ++k) span += (__int128)std::llabs(a.c[k]) * (p.ext[k] - 1);
+      return span < (1ll << 31) && lo > -(1ll << 31) && hi < (1ll << 31);
+    };
+    for (auto &g : p.guards) small = small && fits(g.e) && g.extent < (1ll << 31);
+    for (auto &g : p.domain) small = small && fits(g.e);
+    for (int k = 0; k < p.n(); ++k) small = small && p.ext[k] < (1ll << 31) && p.dst.c[k] < (1ll << 31);
+  }
+  out->small = small ? 1 : 0;
   return AMAP_OK;
 }
 
