@@ -168,6 +168,17 @@ int amap_compose(const amap_chain *chain, amap_map **out_map);
 /* amap_compose with options.  AMAP_COMPOSE_NO_FUSE keeps EVERY intermediate tensor as a temporary, i.e. runs the
  * chain operator by operator as the paper's Section 2.1 finds it before the optimisation (the comparison baseline). */
 #define AMAP_COMPOSE_NO_FUSE 1u
+/* Quasi-affine pieces.  Where a pair has no affine composition (a reshape whose factors do not line up with the loops
+ * around it: the reverse of the store needs floor-division and remainder, which the paper leaves to ISL, Section
+ * 2.1), amap_compose can still eliminate the intermediate with a piece whose source offset is
+ *     b_l + sum_k digit_stride[k] * digit_k(f0 + F i),
+ * digit_k being the digits of the affine form f0 + F i in the mixed radix digit_radix[] (innermost last).  By default
+ * it does so only where a contiguous run of at least 16 bytes survives on both sides (one division chain per run);
+ * otherwise the intermediate stays a temporary (two passes of vector kernels beat one pass of scattered element
+ * accesses).  AMAP_COMPOSE_QUASI_AFFINE: wherever a pair allows one, also in place of an affine composition (for
+ * measurements and tests); AMAP_COMPOSE_NO_QUASI_AFFINE: never. */
+#define AMAP_COMPOSE_QUASI_AFFINE 2u
+#define AMAP_COMPOSE_NO_QUASI_AFFINE 4u
 int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map **out_map);
 /* Several results from one chain (Section 2.1 names split; its last paragraph repeats the elimination until no pair
  * is left, over the whole graph): `outputs` (host array of n_outputs distinct tensor ids, 1..8; chain->output is
@@ -218,6 +229,12 @@ typedef struct amap_piece {
   const amap_constraint *domain;
   uint64_t fill_bits;
   int32_t output; /* which output of the map the piece writes (0 unless amap_compose_multi named several) */
+  /* quasi-affine pieces only (n_digits > 0; C_l is all zero then): see AMAP_COMPOSE_QUASI_AFFINE */
+  int32_t n_digits;
+  const int64_t *digit_radix;  /* n_digits (host, owned by the map) */
+  const int64_t *digit_stride; /* n_digits source strides in elements */
+  const int64_t *F;            /* n_loops coefficients of the inner affine form */
+  int64_t f0;
 } amap_piece;
 
 /* number of pieces of the composed map (all stages): the load/store pairs that are left once Section 2.1's

@@ -13,8 +13,9 @@
  * a kernel by value.  amap_view_locate() is the functor: output element index
  * -> (input, source element index) or the fill value.
  *
- * The header is plain C for the struct and CUDA C++ (under __CUDACC__) for the
- * device function; it has no dependency on the library's internals.
+ * The header is plain C for the struct and CUDA C++ (under __CUDACC__, unless
+ * AMAP_DEVICE_STRUCTS_ONLY is defined) for the device function; it has no
+ * dependency on the library's internals.
  */
 #ifndef AMAP_DEVICE_H_
 #define AMAP_DEVICE_H_
@@ -71,7 +72,14 @@ typedef struct amap_view_source {
   uint64_t fill_bits;
 } amap_view_source;
 
-#ifdef __CUDACC__
+#if defined(__CUDACC__) && !defined(AMAP_DEVICE_STRUCTS_ONLY)
+#ifdef __CUDA_ARCH__ /* unroll hints mean something to the device compiler only */
+#define AMAP_PRAGMA_UNROLL _Pragma("unroll")
+#define AMAP_PRAGMA_UNROLL_1 _Pragma("unroll 1")
+#else
+#define AMAP_PRAGMA_UNROLL
+#define AMAP_PRAGMA_UNROLL_1
+#endif
 /* Output element `o` (0 <= o < out_numel) -> its source.  Returns false if no piece covers o (cannot happen for a
  * view made by amap_map_device_view: the pieces of a composed map cover the output exactly once).  One pass over the
  * piece's loops decodes the index digit by digit and accumulates the source offset and every constraint on the way,
@@ -86,9 +94,9 @@ __host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int6
     if (v.small) {
       uint32_t rem = (uint32_t)(o - pc.b_s), s32 = (uint32_t)pc.b_l;
       int32_t e[AMAP_VIEW_MAX_CONS];
-#pragma unroll
+AMAP_PRAGMA_UNROLL
       for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] = c < nc ? (int32_t)pc.cons[c].offset : 0;
-#pragma unroll 1
+AMAP_PRAGMA_UNROLL_1
       for (int k = 0; k < n; ++k) {
 #ifdef __CUDA_ARCH__
         const uint32_t t = __umulhi(pc.fd_mul[k], rem);
@@ -100,13 +108,13 @@ __host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int6
         rem -= i * (uint32_t)pc.dst_stride[k];
         s32 += i * (uint32_t)pc.src_stride[k];  /* wrap-around arithmetic: the true value fits 31 bits */
         if (nc > 0) {
-#pragma unroll
+AMAP_PRAGMA_UNROLL
           for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] += (int32_t)pc.cons[c].coef[k] * (int32_t)i;
         }
         if (k == n - 1) left = pc.ext[k] - (int64_t)i;
       }
       if (!inside || rem != 0) continue;
-#pragma unroll
+AMAP_PRAGMA_UNROLL
       for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) {
         if (c < nc) {
           const bool ok = (uint32_t)e[c] < (uint32_t)pc.cons[c].extent;
@@ -119,23 +127,23 @@ __host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int6
     } else {
       int64_t rem = o - pc.b_s;
       int64_t e[AMAP_VIEW_MAX_CONS];
-#pragma unroll
+AMAP_PRAGMA_UNROLL
       for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] = c < nc ? pc.cons[c].offset : 0;
       s = pc.b_l;
-#pragma unroll 1
+AMAP_PRAGMA_UNROLL_1
       for (int k = 0; k < n; ++k) {
         const int64_t i = rem / pc.dst_stride[k];
         inside = inside && i < pc.ext[k];
         rem -= i * pc.dst_stride[k];
         s += i * pc.src_stride[k];
         if (nc > 0) {
-#pragma unroll
+AMAP_PRAGMA_UNROLL
           for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) e[c] += pc.cons[c].coef[k] * i;
         }
         if (k == n - 1) left = pc.ext[k] - i;
       }
       if (!inside || rem != 0) continue;
-#pragma unroll
+AMAP_PRAGMA_UNROLL
       for (int c = 0; c < AMAP_VIEW_MAX_CONS; ++c) {
         if (c < nc) {
           const bool ok = e[c] >= 0 && e[c] < pc.cons[c].extent;
@@ -161,6 +169,6 @@ __host__ __device__ inline bool amap_view_locate(const amap_device_view &v, int6
   }
   return false;
 }
-#endif /* __CUDACC__ */
+#endif /* __CUDACC__ && !AMAP_DEVICE_STRUCTS_ONLY */
 
 #endif /* AMAP_DEVICE_H_ */

@@ -17,6 +17,8 @@ from . import build as _build
 AMAP_CONST = -1
 KERNEL_AUTO, KERNEL_GATHER, KERNEL_COPY, KERNEL_TRANSPOSE, KERNEL_FILL = 0, 1, 2, 3, 4
 COMPOSE_NO_FUSE = 1
+COMPOSE_QUASI_AFFINE = 2
+COMPOSE_NO_QUASI_AFFINE = 4
 PLAN_NO_PDL = 1
 PLAN_NO_PREFETCH = 2
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
@@ -62,7 +64,8 @@ class _Piece(Structure):
         ("n_loops", c_int32), ("bounds", POINTER(c_int64)), ("input", c_int32), ("C_l", POINTER(c_int64)),
         ("b_l", c_int64), ("C_s", POINTER(c_int64)), ("b_s", c_int64), ("n_guards", c_int32),
         ("guards", POINTER(_Constraint)), ("n_domain", c_int32), ("domain", POINTER(_Constraint)),
-        ("fill_bits", c_uint64), ("output", c_int32),
+        ("fill_bits", c_uint64), ("output", c_int32), ("n_digits", c_int32), ("digit_radix", POINTER(c_int64)),
+        ("digit_stride", POINTER(c_int64)), ("F", POINTER(c_int64)), ("f0", c_int64),
     ]
 
 
@@ -315,6 +318,11 @@ class Map:
                     "domain": cons(p.domain, p.n_domain),
                     "fill_bits": p.fill_bits,
                     "output": p.output,
+                    "quasi": None if p.n_digits == 0 else {
+                        "radix": [p.digit_radix[d] for d in range(p.n_digits)],
+                        "stride": [p.digit_stride[d] for d in range(p.n_digits)],
+                        "F": [p.F[j] for j in range(nl)], "f0": p.f0,
+                    },
                 }
             )
         return out

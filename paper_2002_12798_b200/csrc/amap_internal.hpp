@@ -28,6 +28,18 @@ struct Con {
   int64_t extent = 0;
 };
 
+// A source offset that is only QUASI-affine in the loops (the reverse of a store composed with a reshape whose
+// factors do not line up needs floor-division and remainder; the paper leaves these to ISL, Section 2.1): the
+// affine form f(i) is an offset into a tensor that was composed away, and the source offset is
+//     srcoff.c0 + sum_k stride[k] * digit_k(f),
+// digit_k being f's digits in the mixed radix (radix[0], ..., radix[K-1]), innermost last -- the loop indices of the
+// statement that wrote that tensor.
+struct QuasiSrc {
+  bool on = false;
+  Aff f;
+  std::vector<int64_t> radix, stride;
+};
+
 // One loop nest of the composed form: for i in the box (and where `domain`
 // holds) dst.flat[dst(i)] = guards hold ? src.flat[srcoff(i)] : fill.
 struct Piece {
@@ -35,6 +47,7 @@ struct Piece {
   Aff dst;
   int src = AMAP_CONST;  // tensor id while composing; input slot in a finished map
   Aff srcoff;
+  QuasiSrc qa;  // when on, srcoff holds the constant only
   std::vector<Con> guards;
   std::vector<Con> domain;
   uint64_t fill = 0;
@@ -69,6 +82,10 @@ void drop_unit_loops(Piece &p);
 // final canonical form of a composed map's pieces (splits single-loop guards
 // into copy + fill pieces, sorts by destination stride, merges loops)
 Status canonicalise(std::vector<Piece> &pieces);
+
+// elements of the contiguous run (on both sides) that loop `in` of the piece walks, as a power of two that divides
+// everything a vector access needs divided: 1 when the loop is no run
+int64_t piece_run_elems(const Piece &p, int in, int64_t cap);
 
 // ---- compose.cpp ---------------------------------------------------------
 // A composed map runs as one or more STAGES.  Normally there is one: every intermediate tensor was composed

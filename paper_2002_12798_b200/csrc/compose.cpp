@@ -28,6 +28,7 @@
 #include <numeric>
 
 #include "amap_internal.hpp"
+#define AMAP_DEVICE_STRUCTS_ONLY
 #include "amap_device.h"
 
 namespace amap {
@@ -228,6 +229,7 @@ static void split_loop(Piece &p, int j, int64_t f) {
   };
   sp(p.dst);
   if (p.src != AMAP_CONST) sp(p.srcoff);
+  if (p.src != AMAP_CONST && p.qa.on) sp(p.qa.f);
   for (auto &g : p.guards) sp(g.e);
   for (auto &g : p.domain) sp(g.e);
   const int64_t e = p.ext[j];
@@ -371,6 +373,10 @@ static Status compose_pair(const Piece &R, const Piece &W, std::vector<PairResul
       pr.q.srcoff = substitute(Wc.srcoff, delta, digit_of_loop, nR);
     else
       pr.q.srcoff.c.assign(nR, 0);
+    if (Wc.src != AMAP_CONST && Wc.qa.on) {  // a quasi-affine writer stays one: its inner form follows the reader's loops
+      pr.q.qa = Wc.qa;
+      pr.q.qa.f = substitute(Wc.qa.f, delta, digit_of_loop, nR);
+    }
     pr.dR = Rc.domain;
     pr.gR = Rc.guards;
     for (int k = 0; k < K; ++k) {
@@ -400,7 +406,7 @@ static void append(std::vector<Con> &a, const std::vector<Con> &b) { a.insert(a.
 
 // Rewrites reader R (whose load names intermediate tensor t) to load external
 // tensors directly: equation (2) applied with every statement that defines t.
-static Status compose_reader(const Piece &R, const TensorState &ts, const TensorInfo &ti, std::vector<Piece> *out) {
+static Status compose_reader_affine(const Piece &R, const TensorState &ts, const TensorInfo &ti, std::vector<Piece> *out) {
   Piece Rin = R;  // the part of the reader that really loads
   append(Rin.domain, Rin.guards);
   Rin.guards.clear();
@@ -493,11 +499,86 @@ static Status compose_reader(const Piece &R, const TensorState &ts, const Tensor
   return Status();
 }
 
+// Where equation (2) has no affine form (a reshape whose factors do not line up with the loops around it), the
+// composition still exists as a QUASI-affine map: the reader's offset f(i') into t_s is split into the digits of the
+// writer's loop nest (floor-division and remainder by compile-time constants), and those digits go through the
+// writer's load.  Supported when one statement wrote t_s, unguarded, as a dense renumbering of all of it.  Such a
+// piece pays divisions per access, so it is only worth having where whole runs share them (a contiguous run of at
+// least 16 bytes on both sides); otherwise the caller keeps t_s as a temporary -- unless `force`.
+static const int kMaxQuasiDigits = 6;
+
+static Status compose_reader_quasi(const Piece &R, const TensorState &ts, const TensorInfo &ti, int es, bool force,
+                                   std::vector<Piece> *out) {
+  if (ts.defs.size() != 1) return err(AMAP_EUNSUPPORTED, "quasi-affine composition needs a single writer");
+  const Piece &W = ts.defs[0];
+  if (W.src == AMAP_CONST || W.qa.on || !W.guards.empty() || !W.domain.empty())
+    return err(AMAP_EUNSUPPORTED, "quasi-affine composition needs a plain writer");
+  if (ti.numel >= (1ll << 31)) return err(AMAP_EUNSUPPORTED, "tensor too large for a quasi-affine piece");
+  Piece Wc = W;
+  drop_unit_loops(Wc);
+  for (int k = 0; k < Wc.n(); ++k) {
+    if (Wc.dst.c[k] == 0) return err(AMAP_ESTORE_NOT_INJECTIVE, "a loop does not move the store");
+    if (Wc.dst.c[k] < 0) reverse_loop(Wc, k);
+  }
+  std::vector<int> order(Wc.n());
+  std::iota(order.begin(), order.end(), 0);
+  std::sort(order.begin(), order.end(), [&](int a, int b) { return Wc.dst.c[a] > Wc.dst.c[b]; });
+  permute_loops(Wc, order);
+  // dense: the writer's loops are exactly the digits of t_s's flat offsets
+  int64_t place = 1;
+  for (int k = Wc.n() - 1; k >= 0; --k) {
+    if (Wc.dst.c[k] != place) return err(AMAP_EUNSUPPORTED, "the writer does not number the tensor densely");
+    place *= Wc.ext[k];
+  }
+  if (Wc.dst.c0 != 0 || place != ti.numel || Wc.n() < 1 || Wc.n() > kMaxQuasiDigits)
+    return err(AMAP_EUNSUPPORTED, "the writer does not number the tensor densely");
+  if (R.guards.size() + R.domain.size() > (size_t)kMaxPieceConstraints)
+    return err(AMAP_EUNSUPPORTED, "the composed piece needs too many constraints");
+  Piece Q;
+  Q.ext = R.ext;
+  Q.dst = R.dst;
+  Q.src = Wc.src;
+  Q.fill = R.fill;
+  Q.guards = R.guards;
+  Q.domain = R.domain;
+  Q.srcoff.c0 = Wc.srcoff.c0;
+  Q.srcoff.c.assign(R.ext.size(), 0);
+  Q.qa.on = true;
+  Q.qa.f = R.srcoff;
+  Q.qa.radix = Wc.ext;
+  Q.qa.stride = Wc.srcoff.c;
+  if (!force) {
+    bool worth = false;
+    for (int k = 0; k < Q.n() && !worth; ++k) worth = piece_run_elems(Q, k, 64) * es >= 16;
+    if (!worth) return err(AMAP_EUNSUPPORTED, "a quasi-affine piece without runs is slower than a temporary");
+  }
+  if (tighten(Q)) out->push_back(std::move(Q));
+  return Status();
+}
+
+// quasi: 0 = where no affine composition exists and runs survive, 1 = wherever the pair allows one (also in place
+// of an affine composition), -1 = never
+static Status compose_reader(const Piece &R, const TensorState &ts, const TensorInfo &ti, int es, int quasi,
+                             std::vector<Piece> *out) {
+  const size_t before = out->size();
+  if (quasi > 0) {
+    if (compose_reader_quasi(R, ts, ti, es, true, out).ok()) return Status();
+    out->resize(before);
+  }
+  Status s = compose_reader_affine(R, ts, ti, out);
+  if (s.code != AMAP_EUNSUPPORTED || quasi != 0) return s;
+  out->resize(before);
+  if (compose_reader_quasi(R, ts, ti, es, false, out).ok()) return Status();
+  out->resize(before);
+  return s;
+}
+
 // ---------------------------------------------------------------------------
 static int64_t unique_reads(const Piece &p0, int64_t in_numel) {
   Piece p = p0;
   const int64_t pts = count_points(p);
   if (p.src == AMAP_CONST) return 0;
+  if (p.qa.on) return std::min(pts >= 0 ? pts : in_numel, in_numel);
   drop_unit_loops(p);
   std::vector<std::pair<int64_t, int64_t>> se;
   for (int k = 0; k < p.n(); ++k)
@@ -701,7 +782,8 @@ static Status compose_chain(const amap_chain *ch, const std::vector<int> &output
     }
     if (S[tl].defs.empty() && T[tl].numel > 0)
       return err(AMAP_EUNDEFINED, "a statement reads a tensor that no earlier statement writes");
-    s = compose_reader(R, S[tl], T[tl], &S[tsid].defs);
+    s = compose_reader(R, S[tl], T[tl], es, (flags & AMAP_COMPOSE_QUASI_AFFINE) ? 1 : (flags & AMAP_COMPOSE_NO_QUASI_AFFINE) ? -1 : 0,
+                       &S[tsid].defs);
     if (s.code == AMAP_EUNSUPPORTED) {
       // This pair cannot be eliminated (the paper's Section 3 also reports a pair that stays): keep t_l as a
       // temporary written by a stage of its own and read it like an input from here on.
@@ -748,8 +830,8 @@ static void log_map(const Map &m) {
     for (int k = 0; k < p.n(); ++k)
       fprintf(stderr, " (%lld: src %lld dst %lld)", (long long)p.ext[k], (long long)(p.src == AMAP_CONST ? 0 : p.srcoff.c[k]),
               (long long)p.dst.c[k]);
-    fprintf(stderr, " b_l %lld b_s %lld guards %zu domain %zu\n", (long long)p.srcoff.c0, (long long)p.dst.c0, p.guards.size(),
-            p.domain.size());
+    fprintf(stderr, " b_l %lld b_s %lld guards %zu domain %zu%s\n", (long long)p.srcoff.c0, (long long)p.dst.c0, p.guards.size(),
+            p.domain.size(), p.qa.on ? " quasi-affine" : "");
   }
 }
 
@@ -762,7 +844,9 @@ extern "C" int amap_compose_ex(const amap_chain *chain, uint32_t flags, amap_map
 
 extern "C" int amap_compose_multi(const amap_chain *chain, int32_t n_outputs, const int32_t *outputs, uint32_t flags,
                                   amap_map **out_map) {
-  if (!out_map || !outputs || n_outputs < 1 || (flags & ~(uint32_t)AMAP_COMPOSE_NO_FUSE)) return AMAP_EINVAL;
+  if (!out_map || !outputs || n_outputs < 1 ||
+      (flags & ~(uint32_t)(AMAP_COMPOSE_NO_FUSE | AMAP_COMPOSE_QUASI_AFFINE | AMAP_COMPOSE_NO_QUASI_AFFINE)))
+    return AMAP_EINVAL;
   amap_map *m = new (std::nothrow) amap_map();
   if (!m) return AMAP_ENOMEM;
   Status s;
@@ -812,6 +896,12 @@ extern "C" int amap_map_get_piece(const amap_map *map, int32_t k, amap_piece *ou
   out->domain = map->m.domain_views[k].data();
   out->fill_bits = p.fill;
   out->output = p.out;
+  const bool qa = p.src != AMAP_CONST && p.qa.on;
+  out->n_digits = qa ? (int32_t)p.qa.radix.size() : 0;
+  out->digit_radix = qa ? p.qa.radix.data() : nullptr;
+  out->digit_stride = qa ? p.qa.stride.data() : nullptr;
+  out->F = qa ? p.qa.f.c.data() : nullptr;
+  out->f0 = qa ? p.qa.f.c0 : 0;
   return AMAP_OK;
 }
 
@@ -869,6 +959,7 @@ extern "C" int amap_map_device_view(const amap_map *map, amap_device_view *out) 
     const Piece &p = m.pieces[q];
     amap_view_piece &v = out->piece[q];
     if (p.n() > AMAP_VIEW_MAX_LOOPS || p.guards.size() + p.domain.size() > (size_t)AMAP_VIEW_MAX_CONS) return AMAP_ETOOLARGE;
+    if (p.src != AMAP_CONST && p.qa.on) return AMAP_EUNSUPPORTED;  // the view holds affine pieces only
     // canonical pieces have positive destination strides in descending order; decoding an output index digit by
     // digit also needs them nested
     for (int k = 0; k < p.n(); ++k)

@@ -8,6 +8,7 @@ constexpr int kDevMaxLoops = 12;
 constexpr int kDevMaxCons = 6;
 constexpr int kMaxInputs = 24;
 constexpr int kMaxOutputs = 8;
+constexpr int kQuasiMaxDigits = 6;
 constexpr int kStrip = 8;  // units per thread in the affine and strip kernels
 
 // unsigned 32-bit division by an invariant divisor, multiply-and-shift form
@@ -37,6 +38,10 @@ constexpr int kTransposeThreads = 256;
 //
 // Affine kernel: one item = one unit of `unit_bytes` bytes; the innermost loop
 // counts units; ext/fd/sstride/dstride describe all loops.
+//
+// A quasi-affine piece (the composition of a reshape whose factors do not line
+// up) runs on the affine kernel: beside the affine offsets it accumulates the
+// inner form f and splits it into digits with multiply-and-shift divisions.
 //
 // Strip kernel: as the affine kernel, but loop `ku` (not the innermost) is cut
 // into strips of kStrip iterations: ext[ku] counts strips, its strides and
@@ -69,6 +74,15 @@ struct DevPiece {
   int64_t sstride[kDevMaxLoops];
   int64_t dstride[kDevMaxLoops];
   DevCon cons[kDevMaxCons];  // guards first, then domain constraints
+  // --- quasi-affine source (affine kernel only) -------------------------
+  // qa_n > 0: the source offset is soff + sum_d qa_stride[d] * digit_d(f), f = qa_f0 + sum_k qa_fstride[k] * i_k
+  // (in units, 32-bit wrap-around arithmetic), digits in the mixed radix qa_radix[] (innermost last).
+  int32_t qa_n;
+  uint32_t qa_f0;
+  uint32_t qa_fstride[kDevMaxLoops];
+  uint32_t qa_radix[kQuasiMaxDigits];
+  FastDiv qa_fd[kQuasiMaxDigits];
+  int64_t qa_stride[kQuasiMaxDigits];  // bytes
   // --- strip kernel only -----------------------------------------------
   int32_t ku;
   uint32_t ku_ext;

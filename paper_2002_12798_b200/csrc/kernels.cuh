@@ -117,7 +117,7 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
   const char *src = (sp.input >= 0) ? ptrs.src[sp.input] : nullptr;
   char *dst = ptrs.dst[sp.out];
 
-  uint32_t rem[U];
+  uint32_t rem[U], fu[U];
   OffT so[U], doff[U];
   bool live[U];
   int32_t acc[U][NC > 0 ? NC : 1];
@@ -126,6 +126,7 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
     const uint64_t L = item0 + (uint64_t)u * kAffineThreads;
     live[u] = L < sp.n_items;
     rem[u] = live[u] ? (uint32_t)L : 0u;
+    fu[u] = sp.qa_f0;
     so[u] = (OffT)sp.soff;
     doff[u] = (OffT)sp.doff;
     if constexpr (NC > 0) {
@@ -137,6 +138,7 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
     const FastDiv fd = sp.fd[k];
     const uint32_t ext = sp.ext[k];
     const OffT ss = (OffT)sp.sstride[k], ds = (OffT)sp.dstride[k];
+    const uint32_t fs = sp.qa_fstride[k];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const uint32_t q = fast_div(rem[u], fd);
@@ -144,9 +146,23 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
       rem[u] = q;
       so[u] += (OffT)i * ss;
       doff[u] += (OffT)i * ds;
+      fu[u] += i * fs;  // the inner form of a quasi-affine source (all zero otherwise)
       if constexpr (NC > 0) {
 #pragma unroll
         for (int c = 0; c < NC; ++c) acc[u][c] += sp.cons[c].coef[k] * (int32_t)i;
+      }
+    }
+  }
+  if (sp.qa_n > 0) {  // block-uniform: split f into the digits of the statement that wrote the eliminated tensor
+    for (int d = sp.qa_n - 1; d >= 0; --d) {
+      const FastDiv fd = sp.qa_fd[d];
+      const uint32_t radix = sp.qa_radix[d];
+      const OffT st = (OffT)sp.qa_stride[d];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint32_t q = fast_div(fu[u], fd);
+        so[u] += (OffT)(fu[u] - q * radix) * st;
+        fu[u] = q;
       }
     }
   }

@@ -95,6 +95,12 @@ static int pick_unit(const Piece &p, int es, int ptr_align, int force_kind) {
   const int n = p.n();
   if (n == 0) return es;
   const int in = n - 1;  // canonical order: innermost destination loop last
+  if (p.src != AMAP_CONST && p.qa.on) {  // quasi-affine: as wide as the run that shares one digit decomposition
+    const int64_t q = piece_run_elems(p, in, 16 / es);
+    int V = (int)(q * es);
+    while (V > es && V > ptr_align) V >>= 1;
+    return V;
+  }
   if (p.dst.c[in] != 1) return es;
   if (p.src != AMAP_CONST && p.srcoff.c[in] != 1) return es;
   for (auto &g : p.guards)
@@ -156,6 +162,26 @@ static int build_affine_piece(const Piece &p, int es, int V, DevPiece *d) {
   }
   if (items >= (1ull << 32) - (uint64_t)kAffineThreads * kUnroll) return AMAP_EUNSUPPORTED;
   d->n_items = (uint64_t)items;
+  if (p.src != AMAP_CONST && p.qa.on) {
+    const int K = (int)p.qa.radix.size();
+    if (K < 1 || K > kQuasiMaxDigits || p.qa.radix[K - 1] % q) return AMAP_EUNSUPPORTED;
+    int64_t lo, hi;
+    aff_range(p.qa.f, p.ext, &lo, &hi);
+    if (hi >= (1ll << 32) || lo <= -(1ll << 31)) return AMAP_EUNSUPPORTED;  // 32-bit arithmetic in the kernel
+    d->qa_n = K;
+    d->qa_f0 = (uint32_t)(p.qa.f.c0 / q);
+    for (size_t j = 0; j < loops.size(); ++j) {
+      const int k = loops[j];
+      d->qa_fstride[j] = (k == p.n() - 1 && q > 1) ? 1u : (uint32_t)(p.qa.f.c[k] / q);
+    }
+    for (int t = 0; t < K; ++t) {
+      const int64_t radix = (t == K - 1) ? p.qa.radix[t] / q : p.qa.radix[t];
+      if (radix < 1 || radix >= (1ll << 32)) return AMAP_EUNSUPPORTED;
+      d->qa_radix[t] = (uint32_t)radix;
+      d->qa_fd[t] = make_fastdiv((uint32_t)radix);
+      d->qa_stride[t] = p.qa.stride[t] * ((t == K - 1) ? (int64_t)V : (int64_t)es);
+    }
+  }
   d->n_guards = (int)p.guards.size();
   d->n_domain = (int)p.domain.size();
   int c = 0;
@@ -258,6 +284,20 @@ static bool check_affine_item(const DevPiece &d, uint64_t L, int64_t in_bytes, i
     for (int c = 0; c < nc; ++c) acc[c] += (int64_t)d.cons[c].coef[k] * i;
   }
   if (rem != 0) return false;
+  if (d.qa_n > 0) {  // the quasi-affine source offset, with the kernel's 32-bit arithmetic
+    uint32_t r2 = (uint32_t)L, f = d.qa_f0;
+    for (int k = d.n_loops - 1; k >= 0; --k) {
+      const uint32_t q = r2 / d.ext[k];
+      f += (r2 - q * d.ext[k]) * d.qa_fstride[k];
+      r2 = q;
+    }
+    for (int t = d.qa_n - 1; t >= 0; --t) {
+      const uint32_t q = host_fast_div(f, d.qa_fd[t]);
+      if (q != f / d.qa_radix[t]) return false;
+      s += (int64_t)(f - q * d.qa_radix[t]) * d.qa_stride[t];
+      f = q;
+    }
+  }
   if (d.kind == kDevStrip) {  // walk the strip as the kernel does
     uint32_t r2 = (uint32_t)L, strip = 0;
     for (int k = d.n_loops - 1; k >= 0; --k) {
@@ -373,7 +413,7 @@ static bool split_a_remainder(const DevPiece &d, DevPiece *whole, DevPiece *rest
 }
 
 static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t in_bytes, DevPiece *d) {
-  if (es > 8 || p.src == AMAP_CONST || !p.guards.empty() || !p.domain.empty()) return false;
+  if (es > 8 || p.src == AMAP_CONST || p.qa.on || !p.guards.empty() || !p.domain.empty()) return false;
   const int n = p.n();
   if (n < 2) return false;
   const int ia = n - 1;
@@ -771,7 +811,7 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
               c.placed[q] = 1;
               continue;
             }
-            if (c.o.force_kernel != AMAP_KERNEL_GATHER) make_strip(&d);
+            if (c.o.force_kernel != AMAP_KERNEL_GATHER && d.qa_n == 0) make_strip(&d);
             if (d.kind != kind) continue;
             if (!check_affine_piece(d, in_bytes, out_bytes)) return plan_fail(AMAP_EOVERFLOW, q);
             if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q);
@@ -806,7 +846,7 @@ static void plan_slabs(const Map &m, int device, const amap_plan_opts &o, amap_p
     return lo >= 0 && hi < slab;
   };
   for (const Piece &p : m.pieces) {
-    if (p.n() < 1 || p.ext[0] != N || !p.guards.empty() || !p.domain.empty()) return;
+    if (p.n() < 1 || p.ext[0] != N || !p.guards.empty() || !p.domain.empty() || p.qa.on) return;
     if (p.dst.c[0] != DS || !inside(p.dst, p.ext, DS)) return;
     if (p.src != AMAP_CONST) {
       const int64_t SS = m.in_numel[p.src] / N;
@@ -902,7 +942,8 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
       kind = AMAP_KERNEL_FILL;
     } else {
       reads[p.src] += piece_unique_reads(p, slot_numel[p.src]);
-      const bool contiguous = p.n() > 0 && p.srcoff.c[p.n() - 1] == 1 && p.dst.c[p.n() - 1] == 1;
+      const bool contiguous = p.n() > 0 && p.dst.c[p.n() - 1] == 1 &&
+                              (p.qa.on ? unit_of[q] > es : p.srcoff.c[p.n() - 1] == 1);
       if (!contiguous && allow_transpose && build_transpose_piece(p, es, align, slot_numel[p.src] * es, &tr[q])) {
         is_tr[q] = 1;
         kind = AMAP_KERNEL_TRANSPOSE;

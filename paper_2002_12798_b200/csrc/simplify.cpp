@@ -33,6 +33,7 @@ template <class F>
 static void for_each_aff(Piece &p, F f) {
   f(p.dst);
   if (p.src != AMAP_CONST) f(p.srcoff);
+  if (p.src != AMAP_CONST && p.qa.on) f(p.qa.f);
   for (auto &g : p.guards) f(g.e);
   for (auto &g : p.domain) f(g.e);
 }
@@ -135,6 +136,7 @@ bool tighten(Piece &p) {
         p.src = AMAP_CONST;
         p.srcoff = Aff();
         p.srcoff.c.assign(p.ext.size(), 0);
+        p.qa = QuasiSrc();
         p.guards.clear();
         break;
       }
@@ -196,6 +198,7 @@ static bool mergeable(const Piece &p, int k) {  // loops k and k+1
   auto fits = [&](const Aff &a) { return a.c[k] == e * a.c[k + 1]; };
   if (!fits(p.dst)) return false;
   if (p.src != AMAP_CONST && !fits(p.srcoff)) return false;
+  if (p.src != AMAP_CONST && p.qa.on && !fits(p.qa.f)) return false;
   for (auto &g : p.guards)
     if (!fits(g.e)) return false;
   for (auto &g : p.domain)
@@ -261,6 +264,38 @@ static void merge_fill_pieces(std::vector<Piece> &pieces) {
   }
 }
 
+int64_t piece_run_elems(const Piece &p, int in, int64_t cap) {
+  if (in < 0 || in >= p.n() || p.dst.c[in] != 1) return 1;
+  for (auto &g : p.guards)
+    if (g.e.c[in] != 0) return 1;
+  for (auto &g : p.domain)
+    if (g.e.c[in] != 0) return 1;
+  if (p.src == AMAP_CONST) return 1;
+  auto divides = [](int64_t q, int64_t v) { return v % q == 0; };
+  int64_t q = 1;
+  while (q * 2 <= cap) q *= 2;
+  for (; q > 1; q /= 2) {
+    bool ok = divides(q, p.ext[in]) && divides(q, p.dst.c0);
+    for (int k = 0; k < p.n() && ok; ++k)
+      if (k != in) ok = divides(q, p.dst.c[k]);
+    if (!p.qa.on) {
+      ok = ok && p.srcoff.c[in] == 1 && divides(q, p.srcoff.c0);
+      for (int k = 0; k < p.n() && ok; ++k)
+        if (k != in) ok = divides(q, p.srcoff.c[k]);
+    } else {
+      // the run walks f by one; it stays inside one innermost digit and that digit is contiguous in the source
+      const size_t K = p.qa.radix.size();
+      ok = ok && K > 0 && p.qa.f.c[in] == 1 && divides(q, p.qa.f.c0) && p.qa.stride[K - 1] == 1 &&
+           divides(q, p.qa.radix[K - 1]) && divides(q, p.srcoff.c0);
+      for (int k = 0; k < p.n() && ok; ++k)
+        if (k != in) ok = divides(q, p.qa.f.c[k]);
+      for (size_t d = 0; d + 1 < K && ok; ++d) ok = divides(q, p.qa.stride[d]);
+    }
+    if (ok) return q;
+  }
+  return 1;
+}
+
 Status canonicalise(std::vector<Piece> &pieces) {
   std::vector<Piece> work;
   work.swap(pieces);
@@ -291,6 +326,7 @@ Status canonicalise(std::vector<Piece> &pieces) {
       f.src = AMAP_CONST;
       f.srcoff = Aff();
       f.srcoff.c.assign(f.ext.size(), 0);
+      f.qa = QuasiSrc();
       f.guards.clear();
       clip_loop(f, gk, from, len);
       work.push_back(std::move(f));

@@ -59,7 +59,16 @@ def _eval_pieces(pieces, numel, flat, dtype):
                 g &= (v >= 0) & (v < e)
             d = aff(p["C_s"], p["b_s"])[dom]
             if p["input"] >= 0:
-                s = aff(p["C_l"], p["b_l"])[dom]
+                s = aff(p["C_l"], p["b_l"])
+                if p["quasi"]:  # b_l + sum_k stride_k * digit_k(f0 + F i), digits in the mixed radix, innermost last
+                    f = aff(p["quasi"]["F"], p["quasi"]["f0"])
+                    f = np.where(dom & g, f, 0)
+                    for radix, stride in zip(reversed(p["quasi"]["radix"][1:]), reversed(p["quasi"]["stride"][1:])):
+                        s += stride * (f % radix)
+                        f = f // radix
+                    assert ((f >= 0) & (f < p["quasi"]["radix"][0])).all()
+                    s += p["quasi"]["stride"][0] * f
+                s = s[dom]
                 gg = g[dom]
                 vals = np.where(gg, flat[p["input"]][np.where(gg, s, 0)], p["fill_bits"]).astype(out.dtype)
             else:
@@ -533,3 +542,99 @@ def test_device_view_refuses_what_it_cannot_hold():
     with pytest.raises(B.AmapError) as e:
         B.compose_chain(chain, outputs=outs).device_view()  # several outputs
     assert e.value.code == -9
+
+
+# ---------------------------------------------------------------------------
+# quasi-affine pieces: reshapes whose factors do not line up with the loops around them
+# ---------------------------------------------------------------------------
+def _run_preserving_chain(a=100, b=81, c=90, d=90, inner=8, dtype="bf16"):
+    """[a, b, inner] -> transpose(1,0,2) -> reshape [c, d, inner] (a*b == c*d, the factors do not line up) ->
+    transpose(1,0,2): rows of `inner` elements stay contiguous on both sides."""
+    assert a * b == c * d
+    return W.Chain(
+        name="quasi_runs", dtype=dtype, inputs=[[a, b, inner]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0, 2]},
+            {"kind": "reshape", "src": 1, "shape": [c, d, inner]},
+            {"kind": "transpose", "src": 2, "perm": [1, 0, 2]},
+        ],
+        values="normal",
+    )
+
+
+def _scattered_chain(m=128, n=90, r=160):
+    """[m, n] -> transpose -> reshape [r, m*n/r] -> transpose: no contiguous run survives."""
+    return W.Chain(
+        name="quasi_scattered", dtype="bf16", inputs=[[m, n]],
+        ops=[
+            {"kind": "transpose", "src": 0, "perm": [1, 0]},
+            {"kind": "reshape", "src": 1, "shape": [r, m * n // r]},
+            {"kind": "transpose", "src": 2, "perm": [1, 0]},
+        ],
+        values="normal",
+    )
+
+
+def test_runs_that_survive_a_misaligned_reshape_compose_into_one_quasi_affine_piece():
+    chain = _run_preserving_chain()
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    m = B.compose_chain(chain)
+    assert len(m.stages()) == 1  # no temporary
+    quasi = [p for p in m.pieces() if p["quasi"]]
+    assert len(quasi) == 1 and quasi[0]["quasi"]["radix"][-1] == 8 and quasi[0]["quasi"]["stride"][-1] == 1
+    assert np.array_equal(eval_map(m, xs), want.reshape(-1))
+    st = m.plan(device=-1).stats()
+    assert st["n_stages"] == 1 and st["kernels"]["copy"] == 1  # 16-byte units: one division chain per unit
+    # switched off, the pair keeps its temporary
+    m2 = B.compose_chain(chain, B.COMPOSE_NO_QUASI_AFFINE)
+    assert len(m2.stages()) == 2 and not any(p["quasi"] for p in m2.pieces())
+    assert np.array_equal(eval_map(m2, xs), want.reshape(-1))
+
+
+def test_scattered_quasi_affine_pairs_keep_their_temporary_unless_forced():
+    chain = _scattered_chain()
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    m = B.compose_chain(chain)
+    assert len(m.stages()) == 2 and not any(p["quasi"] for p in m.pieces())
+    forced = B.compose_chain(chain, B.COMPOSE_QUASI_AFFINE)
+    assert len(forced.stages()) == 1 and any(p["quasi"] for p in forced.pieces())
+    assert np.array_equal(eval_map(forced, xs), want.reshape(-1))
+    assert forced.plan(device=-1).stats()["kernels"]["gather"] == 1
+
+
+def test_readers_of_a_quasi_affine_tensor_and_guards_compose_on():
+    """pad and slice behind the misaligned reshape: the reader's guards stay affine in its own loops, and a reader
+    that lines up with the quasi-affine writer inherits its digits."""
+    chain = _run_preserving_chain(dtype="fp32")
+    chain.ops += [
+        {"kind": "pad", "src": 3, "lo": [1, 0, 0], "hi": [0, 2, 0]},
+        {"kind": "slice", "src": 4, "start": [0, 1, 0], "stop": [91, 90, 8], "step": [3, 2, 1]},
+    ]
+    chain.values = "raw"
+    xs = W.make_index_tagged_inputs(chain)
+    xs = [x + np.uint32(1) for x in xs]
+    want = oracle.run_chain(chain, xs)
+    for flags in (0, B.COMPOSE_QUASI_AFFINE):
+        m = B.compose_chain(chain, flags)
+        assert np.array_equal(eval_map(m, xs), want.reshape(-1))
+    assert len(B.compose_chain(chain).stages()) == 1
+
+
+def test_random_chains_with_quasi_affine_composition_forced():
+    r = np.random.default_rng(1279800)
+    quasi = 0
+    for trial in range(300):
+        chain = random_chain(r)
+        xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
+        try:
+            m = B.compose_chain(chain, B.COMPOSE_QUASI_AFFINE)
+        except B.AmapError as e:
+            assert e.code == -9
+            continue
+        quasi += any(p["quasi"] for p in m.pieces())
+        want = oracle.run_chain(chain, xs)
+        assert np.array_equal(eval_map(m, xs), want.reshape(-1)), (trial, chain.ops)
+        m.plan(device=-1)  # the planner's host replay of every address
+    assert quasi >= 10

@@ -275,6 +275,60 @@ def test_consumer_reads_through_the_map(B, name, rows):
     assert np.array_equal(sums.cpu().numpy().view(np.uint32), want_sums)
 
 
+def test_quasi_affine_pieces_bit_exact(B):
+    """Reshapes whose factors do not line up with the transposes around them: one quasi-affine piece (digits by
+    multiply-and-shift division inside the affine kernel) instead of a temporary -- with 16-byte units where runs
+    survive, element by element where forced, with guards and a further reader behind it."""
+    from test_compose import _run_preserving_chain, _scattered_chain
+
+    runs = _run_preserving_chain()
+    xs = W.make_inputs(runs)
+    want = oracle.run_chain(runs, xs)
+    got, plan = run_gpu(B, runs, xs)
+    assert plan.stats()["n_stages"] == 1 and plan.stats()["kernels"]["copy"] == 1
+    assert np.array_equal(got, want.reshape(-1))
+    got, plan = run_gpu(B, runs, xs, compose_flags=B.COMPOSE_NO_QUASI_AFFINE)  # the two-pass form of the same chain
+    assert plan.stats()["n_stages"] == 2 and np.array_equal(got, want.reshape(-1))
+
+    scattered = _scattered_chain()
+    xs = W.make_inputs(scattered)
+    want = oracle.run_chain(scattered, xs)
+    got, plan = run_gpu(B, scattered, xs, compose_flags=B.COMPOSE_QUASI_AFFINE)
+    assert plan.stats()["n_stages"] == 1 and plan.stats()["kernels"]["gather"] == 1
+    assert np.array_equal(got, want.reshape(-1))
+
+    guarded = _run_preserving_chain(dtype="fp32")
+    guarded.ops += [
+        {"kind": "pad", "src": 3, "lo": [1, 0, 0], "hi": [0, 2, 0]},
+        {"kind": "slice", "src": 4, "start": [0, 1, 0], "stop": [91, 90, 8], "step": [3, 2, 1]},
+    ]
+    guarded.values = "raw"
+    xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(guarded)]
+    want = oracle.run_chain(guarded, xs)
+    for flags in (0, B.COMPOSE_QUASI_AFFINE):
+        got, plan = run_gpu(B, guarded, xs, compose_flags=flags)
+        assert plan.stats()["n_stages"] == 1 and np.array_equal(got, want.reshape(-1))
+
+
+def test_random_chains_with_quasi_affine_pieces(B):
+    r = np.random.default_rng(1279800)
+    quasi = 0
+    for trial in range(120):
+        chain = random_chain(r)
+        xs = [x + np.uint32(1) for x in W.make_index_tagged_inputs(chain)]
+        try:
+            m = B.compose_chain(chain, B.COMPOSE_QUASI_AFFINE)
+        except B.AmapError as e:
+            assert e.code == -9
+            continue
+        quasi += any(p["quasi"] for p in m.pieces())
+        want = oracle.run_chain(chain, xs)
+        for force in (0, 1):
+            got, _ = run_gpu(B, chain, xs, force=force, compose_flags=B.COMPOSE_QUASI_AFFINE)
+            assert np.array_equal(got, want.reshape(-1)), (trial, force, chain.ops)
+    assert quasi >= 4
+
+
 def test_dag_with_a_shared_intermediate(B):
     """One transposed tensor feeds a slice and a pad that are joined again: two readers of one intermediate."""
     chain = W.Chain(
