@@ -506,6 +506,7 @@ static Status compose_reader_affine(const Piece &R, const TensorState &ts, const
 // piece pays divisions per access, so it is only worth having where whole runs share them (a contiguous run of at
 // least 16 bytes on both sides); otherwise the caller keeps t_s as a temporary -- unless `force`.
 static const int kMaxQuasiDigits = 6;
+static const int kQuasiPreferredOverPieces = 8;
 
 static Status compose_reader_quasi(const Piece &R, const TensorState &ts, const TensorInfo &ti, int es, bool force,
                                    std::vector<Piece> *out) {
@@ -566,10 +567,16 @@ static Status compose_reader(const Piece &R, const TensorState &ts, const Tensor
     out->resize(before);
   }
   Status s = compose_reader_affine(R, ts, ti, out);
-  if (s.code != AMAP_EUNSUPPORTED || quasi != 0) return s;
+  if (quasi != 0) return s;
+  // no affine composition, or one that shatters the reader into many pieces (one descriptor and one set of
+  // constraints each; measured: 64 pieces of 16 KiB runs ran at a fortieth of the one quasi-affine piece's rate)
+  const bool shattered = s.ok() && out->size() - before > (size_t)kQuasiPreferredOverPieces;
+  if (s.code != AMAP_EUNSUPPORTED && !shattered) return s;
+  std::vector<Piece> affine(out->begin() + before, out->end());
   out->resize(before);
   if (compose_reader_quasi(R, ts, ti, es, false, out).ok()) return Status();
   out->resize(before);
+  out->insert(out->end(), affine.begin(), affine.end());
   return s;
 }
 

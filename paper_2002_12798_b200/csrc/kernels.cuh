@@ -82,9 +82,14 @@ __device__ __forceinline__ void store_unit(char *p, typename Unit<V>::T v) {
 // find the piece a block belongs to and copy its descriptor to shared memory
 __device__ __forceinline__ void fetch_piece(const DevPiece *__restrict__ table, int first_piece, int n_pieces,
                                             DevPiece *sp) {
-  int p = first_piece;
-  const int last = first_piece + n_pieces - 1;
-  while (p < last && blockIdx.x >= table[p + 1].first_block) ++p;
+  // the last piece whose first block is at or below this block's index: a binary search, since every probe is a
+  // dependent load from global memory (a linear walk over 64 descriptors cost tens of microseconds per block)
+  int p = first_piece, hi = first_piece + n_pieces - 1;
+  while (p < hi) {
+    const int mid = (p + hi + 1) >> 1;
+    if (blockIdx.x >= table[mid].first_block) p = mid;
+    else hi = mid - 1;
+  }
   const uint32_t *src = reinterpret_cast<const uint32_t *>(table + p);
   uint32_t *dst = reinterpret_cast<uint32_t *>(sp);
   for (int w = threadIdx.x; w < (int)(sizeof(DevPiece) / 4); w += blockDim.x) dst[w] = src[w];
