@@ -104,7 +104,15 @@ struct DevPiece {
 
 struct PtrTable {
   const char *src[kMaxInputs];
-  char *dst[kMaxOutputs];
+  char *dst0;                       // output 0: read at a fixed offset of the kernel parameters (the common case)
+  char *dst_more[kMaxOutputs - 1];  // outputs 1.. of a map with several outputs
+#ifdef __CUDACC__
+  __host__ __device__ __forceinline__ char *dst(int out) const { return out == 0 ? dst0 : dst_more[out - 1]; }
+#endif
+  void set_dst(int out, char *p) {
+    if (out == 0) dst0 = p;
+    else dst_more[out - 1] = p;
+  }
 };
 
 }  // namespace amap

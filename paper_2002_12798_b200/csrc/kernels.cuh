@@ -120,7 +120,7 @@ __device__ __forceinline__ void affine_body(const DevPiece &sp, const PtrTable &
   const int n = sp.n_loops;
   const uint64_t item0 = (uint64_t)(blockIdx.x - sp.first_block) * (uint64_t)(kAffineThreads * U) + threadIdx.x;
   const char *src = (sp.input >= 0) ? ptrs.src[sp.input] : nullptr;
-  char *dst = ptrs.dst[sp.out];
+  char *dst = ptrs.dst(sp.out);
 
   uint32_t rem[U], fu[U];
   OffT so[U], doff[U];
@@ -226,7 +226,7 @@ __device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &p
   const uint64_t item = (uint64_t)(blockIdx.x - sp.first_block) * kAffineThreads + threadIdx.x;
   if (item >= sp.n_items) return;
   const char *src = (sp.input >= 0) ? ptrs.src[sp.input] : nullptr;
-  char *dst = ptrs.dst[sp.out];
+  char *dst = ptrs.dst(sp.out);
   uint32_t rem = (uint32_t)item;
   OffT so = (OffT)sp.soff, dof = (OffT)sp.doff;
   int32_t acc[NC > 0 ? NC : 1];
@@ -422,7 +422,7 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
     dbase += (int64_t)i * sp.dstride[k];
   }
   const char *src = ptrs.src[sp.input] + sbase;
-  char *dst = ptrs.dst[sp.out] + dbase;
+  char *dst = ptrs.dst(sp.out) + dbase;
   const uint32_t ext_a = sp.ext_a;
   const uint32_t end_b = min(sp.ext_b, b0 + step_b);  // the tile's own end along b
   // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
@@ -547,7 +547,7 @@ __device__ __forceinline__ void transpose_body(const DevPiece &sp, const PtrTabl
   __shared__ __align__(128) unsigned char tile[kTileBytes];
   if (sp.kind != kDevTranspose) {  // block-uniform
     pdl_wait();
-    fill_block(sp, ptrs.dst[sp.out]);
+    fill_block(sp, ptrs.dst(sp.out));
     return;
   }
   if (sp.tile_ca == 4) {
@@ -613,7 +613,7 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
     dbase += (int64_t)i * sp.dstride[k];
   }
   const char *src = ptrs.src[sp.input] + sbase;
-  char *dst = ptrs.dst[sp.out] + dbase;
+  char *dst = ptrs.dst(sp.out) + dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
   const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1], db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
@@ -708,7 +708,7 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
     dbase += (int64_t)i * sp.dstride[k];
   }
   const char *src = ptrs.src[sp.input] + sbase;
-  char *dst = ptrs.dst[sp.out];  // dbase stays a byte offset: the slots are aligned relative to the tensor's start
+  char *dst = ptrs.dst(sp.out);  // dbase stays a byte offset: the slots are aligned relative to the tensor's start
   const uint32_t ext_a = sp.ext_a;
   const uint32_t end_b = min(sp.ext_b, b0 + kTileB);
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
@@ -863,7 +863,7 @@ __device__ __forceinline__ void transpose_realign_body(const DevPiece &sp, const
     dbase += (int64_t)i * sp.dstride[k];
   }
   const char *src = ptrs.src[sp.input];
-  char *dst = ptrs.dst[sp.out] + dbase;
+  char *dst = ptrs.dst(sp.out) + dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
   const int nb = (int)min((uint32_t)TBR, ext_b - b0);

@@ -1197,7 +1197,7 @@ static int bind_buffers(const amap_plan_t *plan, const void *const *src_dev_ptrs
       const uintptr_t e0 = (uintptr_t)dst_dev_ptrs[j], e1 = e0 + (uintptr_t)plan->out_numels[j] * plan->elem_size;
       if (d0 < e1 && e0 < d1) return AMAP_EINVAL;
     }
-    pt->dst[k] = (char *)dst_dev_ptrs[k];
+    pt->set_dst((int)k, (char *)dst_dev_ptrs[k]);
   }
   for (size_t q = 0; q < plan->in_numel.size(); ++q) {
     if (!src_dev_ptrs[q]) {  // allowed for an input that no piece of this map reads
@@ -1243,7 +1243,7 @@ extern "C" int amap_execute_multi(const amap_plan_t *plan, const void *const *sr
     const LaunchDesc &ld = plan->launch_desc[li];
     const int t = plan->stage_dst[L.stage];
     PtrTable stage_pt = pt;  // stages run in stream order; a stage that writes a temporary has one destination
-    if (t >= 0) stage_pt.dst[0] = (char *)plan->temps[t];
+    if (t >= 0) stage_pt.set_dst(0, (char *)plan->temps[t]);
     const DescSource ds{ld.n_pieces > 0 ? &ld : nullptr, plan->dev_table};
     const cudaError_t e = enqueue(ds, L, stage_pt, s, plan->pdl);
     if (e != cudaSuccess) return cuda_fail(e, "amap_execute: kernel launch");
