@@ -48,9 +48,10 @@ SIGNED = {1: np.int8, 2: np.int16, 4: np.int32, 8: np.int64}
 # previous launch leaves them).  Valid only for the kernel source it was taken on: the digest below is that of the
 # kernel sources at capture time, and the line reports traffic = null when they have changed since.
 STEADY_STATE_TRAFFIC = {
-    "bytes_per_launch": None,
-    "kernel_digest": None,
-    "note": "no steady-state capture for the present kernel sources",
+    "bytes_per_launch": 101_530_960,
+    "kernel_digest": "56814d7913a635ed",
+    "note": "ncu counters over 16 consecutive launches of the timed loop, caches as the previous launch leaves them: "
+            "51.41 MB read + 50.12 MB written per launch, 0.988 of the algorithmic bytes",
 }
 KERNEL_SOURCES = ("kernels.cuh", "device_table.hpp", "plan_execute.cu")
 
