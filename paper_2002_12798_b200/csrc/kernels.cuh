@@ -413,38 +413,153 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
   q = fast_div(t, sp.fd_tiles_a);
   const uint32_t a0 = (t - q * sp.tiles_a) * TA;
   t = q;
-  int64_t sbase = sp.soff, dbase = sp.doff;
+  // Offsets are kept relative to the TENSORS' first bytes: with 32-bit OffT the arithmetic wraps around, which is
+  // exact as long as the final offset fits 32 bits -- it does (the planner checks), whatever the signs of the
+  // strides on the way.
+  OffT sbase = (OffT)sp.soff, dbase = (OffT)sp.doff;
   for (int k = sp.n_loops - 1; k >= 0; --k) {
     q = fast_div(t, sp.fd[k]);
     const uint32_t i = t - q * sp.ext[k];
     t = q;
-    sbase += (int64_t)i * sp.sstride[k];
-    dbase += (int64_t)i * sp.dstride[k];
+    sbase += (OffT)i * (OffT)sp.sstride[k];
+    dbase += (OffT)i * (OffT)sp.dstride[k];
   }
-  const char *src = ptrs.src[sp.input] + sbase;
-  char *dst = ptrs.dst(sp.out) + dbase;
+  const char *src = ptrs.src[sp.input];
+  char *dst = ptrs.dst(sp.out);
   const uint32_t ext_a = sp.ext_a;
   const uint32_t end_b = min(sp.ext_b, b0 + step_b);  // the tile's own end along b
+  const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
+  const bool split = fa.d < ext_a;       // a merges two loops
+  const bool split_b = fb.d < sp.ext_b;  // b merges two loops
+  const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1], db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
   // While the kernel before this one on the stream drains, ask L2 for this tile's source rows (a hint: it
   // reads nothing into the SM and is harmless whatever that kernel still writes); the loads after the wait
-  // then start from L2 instead of paying a DRAM round trip with the memory system idle.
-  auto prefetch_rows = [&](const char *base, uint32_t pa0, uint32_t pb0) {
+  // then start from L2 instead of paying a DRAM round trip with the memory system idle.  One bulk prefetch per
+  // row; the instruction is issued lane by lane (some 500 instructions for the 64 rows), which is free here: the
+  // block has nothing else to do until the wait returns.
+  auto prefetch_rows_bulk = [&](OffT base, uint32_t pa0, uint32_t pb0) {
     const uint32_t a = pa0 + threadIdx.x;
-    if (a < ext_a && pb0 < sp.ext_b) {
-      const uint32_t a_hi = fast_div(a, sp.fd_a_in);
-      const char *row = base + (int64_t)(a - a_hi * sp.fd_a_in.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1] + (int64_t)pb0 * ES;
+    if (threadIdx.x < TA && a < ext_a && pb0 < sp.ext_b) {
+      const uint32_t a_hi = fast_div(a, fa);
+      const OffT off = base + (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1 + (OffT)(pb0 * ES);
       const uint32_t bytes = min(step_b, sp.ext_b - pb0) * ES;
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src + off), "r"(bytes) : "memory");
     }
   };
-  if (sp.prefetch && threadIdx.x < TA) prefetch_rows(src, a0, b0);
+  // The same hint line by line with the per-thread prefetch instruction (one warp instruction covers 32 lines; a
+  // tile is 128 lines of 128 bytes: thread i < 128 asks for line i % LPR of row i / LPR): used between the loads and
+  // the shared-memory stores, where instructions are not free.
+  auto prefetch_rows = [&](OffT base, uint32_t pa0, uint32_t pb0) {
+    constexpr int LPR = RB / 128;  // lines per tile row
+    const uint32_t a = pa0 + threadIdx.x / LPR, line = threadIdx.x % LPR;
+    if (threadIdx.x < TA * LPR && a < ext_a && pb0 < sp.ext_b) {
+      const uint32_t bytes = min(step_b, sp.ext_b - pb0) * ES;
+      if (line * 128 < bytes) {
+        const uint32_t a_hi = fast_div(a, fa);
+        const OffT off = base + (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1 + (OffT)(pb0 * ES);
+        const char *row = src + off;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(row + line * 128));
+        // a row that does not start on a line boundary ends in one line more
+        if ((line + 1) * 128 >= bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(row + bytes - 1));
+      }
+    }
+  };
+  // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
+  // blocks further on in the grid): its loads will find their lines in L2.  Only within this piece: on a
+  // launch of several small pieces (measured on configuration 4) hints for another piece's tiles cost more
+  // than they save.
+  auto prefetch_ahead = [&]() {
+    if (sp.prefetch > 1 && threadIdx.x < 128) {
+      uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
+      if (t2 < sp.n_blocks) {
+        uint32_t q2 = fast_div(t2, sp.fd_tiles_b);
+        const uint32_t nb0 = (t2 - q2 * sp.tiles_b) * step_b;
+        t2 = q2;
+        q2 = fast_div(t2, sp.fd_tiles_a);
+        const uint32_t na0 = (t2 - q2 * sp.tiles_a) * TA;
+        t2 = q2;
+        OffT nbase = (OffT)sp.soff;
+        for (int k = sp.n_loops - 1; k >= 0; --k) {
+          q2 = fast_div(t2, sp.fd[k]);
+          nbase += (OffT)(t2 - q2 * sp.ext[k]) * (OffT)sp.sstride[k];
+          t2 = q2;
+        }
+        prefetch_rows(nbase, na0, nb0);
+      }
+    }
+  };
+  if (sp.prefetch) prefetch_rows_bulk(sbase, a0, b0);
   pdl_wait();
+
+  // The common case -- the general tile shape, 2- or 4-byte elements, no merged indices, all rows of the tile inside
+  // the piece -- with every address formed once per thread and stepped by constants: a third of the instructions
+  // of the general path below.  (These kernels run against the power limit: instructions not issued are clock
+  // kept.)  Block-uniform.
+  if constexpr (CA == 8 && (ES == 2 || ES == 4)) {
+    if (!split && !split_b && a0 + TA <= ext_a) {
+      constexpr int RPU = kTransposeThreads / CB;  // tile rows between a thread's loads
+      const int a_l0 = threadIdx.x / CB, cb = threadIdx.x % CB;
+      const bool in_b = b0 + cb * EPU < end_b;
+      const OffT first = sbase + (OffT)(a0 + a_l0) * sa0 + (OffT)((b0 + cb * EPU) * ES);
+      const OffT step = (OffT)RPU * sa0;
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        v[u] = make_uint4(0, 0, 0, 0);
+        if (in_b) v[u] = load_16(src + (OffT)(first + (OffT)u * step));
+      }
+      issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
+      prefetch_ahead();
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int a_l = a_l0 + u * RPU;
+        *reinterpret_cast<uint4 *>(tile + a_l * RB + ((cb ^ ((a_l / EPU) & 7)) << 4)) = v[u];
+      }
+      __syncthreads();
+      // phase 2.  Work item idx = thread + 256 u takes chunk ca of a and column (pair) bq + 32 u; 32 columns (pairs)
+      // further on the tile's swizzle repeats, so the shared-memory address moves by a constant 128 bytes (ES = 2:
+      // 64 columns) and the destination by a constant number of rows.
+      const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+      const int ca = lane & 7, bq = (lane >> 3) + 4 * w;
+      constexpr int COLS = ES == 2 ? 2 : 1;       // columns a work item stores
+      constexpr int ROUNDS = ES == 2 ? U / 2 : U;
+      const int b_l0 = bq * COLS;
+      const unsigned char *p = tile + (ca * EPU) * RB + (((b_l0 / EPU) ^ ca) << 4) + (b_l0 % EPU) * ES;
+      const OffT dfirst = dbase + (OffT)((a0 + ca * EPU) * ES) + (OffT)(b0 + b_l0) * db0;
+      const OffT dstep = (OffT)(32 * COLS) * db0;
+#pragma unroll
+      for (int u = 0; u < ROUNDS; ++u) {
+        const uint32_t b = b0 + b_l0 + u * 32 * COLS;
+        if (b >= end_b) continue;  // extents and steps are even: with ES == 2, b + 1 is inside too
+        const unsigned char *pu = p + u * 128;
+        char *d = dst + (OffT)(dfirst + (OffT)u * dstep);
+        if constexpr (ES == 2) {
+          uint32_t r[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) r[j] = *reinterpret_cast<const uint32_t *>(pu + j * RB);
+          uint4 lo, hi;
+          lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
+          lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
+          lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
+          lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
+          __stcs(reinterpret_cast<uint4 *>(d), lo);
+          __stcs(reinterpret_cast<uint4 *>(dst + (OffT)(dfirst + (OffT)u * dstep + db0)), hi);
+        } else {
+          uint4 out;
+          out.x = *reinterpret_cast<const uint32_t *>(pu);
+          out.y = *reinterpret_cast<const uint32_t *>(pu + RB);
+          out.z = *reinterpret_cast<const uint32_t *>(pu + 2 * RB);
+          out.w = *reinterpret_cast<const uint32_t *>(pu + 3 * RB);
+          __stcs(reinterpret_cast<uint4 *>(d), out);
+        }
+      }
+      return;
+    }
+  }
+
   // phase 1: global -> shared, 16 bytes along b
   uint4 v[U];
   {
-    const FastDiv fa = sp.fd_a_in;
-    const bool split = fa.d < ext_a;  // a merges two loops
-    const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
@@ -452,7 +567,7 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
       const uint32_t a = a0 + a_l, b = b0 + cb * EPU;
       v[u] = make_uint4(0, 0, 0, 0);
       if (a < ext_a && b < end_b) {
-        OffT off = (OffT)(b * ES);
+        OffT off = sbase + (OffT)(b * ES);
         if (split) {
           const uint32_t a_hi = fast_div(a, fa);
           off += (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1;
@@ -463,28 +578,7 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
       }
     }
     issue_barrier();  // all loads of the tile are in flight before the first shared-memory store waits for one
-    // The same hint for the tile of the block that will take this block's place once it retires (`prefetch`
-    // blocks further on in the grid): its loads will find their lines in L2.  Only within this piece: on a
-    // launch of several small pieces (measured on configuration 4) hints for another piece's tiles cost more
-    // than they save.
-    if (sp.prefetch > 1 && threadIdx.x < TA) {
-      uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
-      if (t2 < sp.n_blocks) {
-        uint32_t q2 = fast_div(t2, sp.fd_tiles_b);
-        const uint32_t nb0 = (t2 - q2 * sp.tiles_b) * step_b;
-        t2 = q2;
-        q2 = fast_div(t2, sp.fd_tiles_a);
-        const uint32_t na0 = (t2 - q2 * sp.tiles_a) * TA;
-        t2 = q2;
-        int64_t nbase = sp.soff;
-        for (int k = sp.n_loops - 1; k >= 0; --k) {
-          q2 = fast_div(t2, sp.fd[k]);
-          nbase += (int64_t)(t2 - q2 * sp.ext[k]) * sp.sstride[k];
-          t2 = q2;
-        }
-        prefetch_rows(ptrs.src[sp.input] + nbase, na0, nb0);
-      }
-    }
+    prefetch_ahead();
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int idx = threadIdx.x + u * kTransposeThreads;
@@ -494,11 +588,8 @@ __device__ __forceinline__ void transpose_tile(const DevPiece &sp, const PtrTabl
   }
   __syncthreads();
   // phase 2: shared -> global, 16 bytes along a
-  const FastDiv fb = sp.fd_b_in;
-  const bool split_b = fb.d < sp.ext_b;  // b merges two loops
-  const OffT db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
   auto dst_of = [&](uint32_t a, uint32_t b) -> char * {
-    OffT off = (OffT)(a * ES);
+    OffT off = dbase + (OffT)(a * ES);
     if (split_b) {
       const uint32_t b_hi = fast_div(b, fb);
       off += (OffT)(b - b_hi * fb.d) * db0 + (OffT)b_hi * db1;
@@ -612,8 +703,11 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
     sbase += (int64_t)i * sp.sstride[k];
     dbase += (int64_t)i * sp.dstride[k];
   }
-  const char *src = ptrs.src[sp.input] + sbase;
-  char *dst = ptrs.dst(sp.out) + dbase;
+  // offsets relative to the tensors' first bytes: 32-bit wrap-around arithmetic is then exact whatever the signs of
+  // the strides (the final offset fits 32 bits)
+  const char *src = ptrs.src[sp.input];
+  char *dst = ptrs.dst(sp.out);
+  const OffT sb = (OffT)sbase, dbs = (OffT)dbase;
   const uint32_t ext_a = sp.ext_a, ext_b = sp.ext_b;
   const FastDiv fa = sp.fd_a_in, fb = sp.fd_b_in;
   const OffT sa0 = (OffT)sp.sa[0], sa1 = (OffT)sp.sa[1], db0 = (OffT)sp.db[0], db1 = (OffT)sp.db[1];
@@ -630,7 +724,7 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
       ok[g] = a < ext_a && b < ext_b;
       if (ok[g]) {
         const uint32_t a_hi = fast_div(a, fa);
-        v[g] = load_unit<UB>(src + (OffT)((OffT)(b * ES) + (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1));
+        v[g] = load_unit<UB>(src + (OffT)(sb + (OffT)(b * ES) + (OffT)(a - a_hi * fa.d) * sa0 + (OffT)a_hi * sa1));
       }
     }
     issue_barrier();
@@ -653,7 +747,7 @@ __device__ __forceinline__ void transpose_narrow_body(const DevPiece &sp, const 
 #pragma unroll
       for (int j = 0; j < EPN; ++j) pk.e[j] = *reinterpret_cast<const E *>(tile + tile_offset<ES>(ca * EPN + j, b_l * ES));
       const uint32_t b_hi = fast_div(b, fb);
-      store_unit<UB>(dst + (OffT)((OffT)(a * ES) + (OffT)(b - b_hi * fb.d) * db0 + (OffT)b_hi * db1), pk.v);
+      store_unit<UB>(dst + (OffT)(dbs + (OffT)(a * ES) + (OffT)(b - b_hi * fb.d) * db0 + (OffT)b_hi * db1), pk.v);
     }
   }
 }

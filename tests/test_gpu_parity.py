@@ -329,6 +329,27 @@ def test_random_chains_with_quasi_affine_pieces(B):
     assert quasi >= 4
 
 
+@pytest.mark.parametrize("rows,cols,dtype", [(64, 256, "bf16"), (128, 384, "bf16"), (40, 72, "bf16"), (32, 132, "fp32"),
+                                             (56, 28, "bf16"), (24, 40, "u8")])
+def test_transposes_with_negative_source_strides(B, rows, cols, dtype):
+    """Y[j, i] = X[rows - 1 - i, j] and Y[j, i] = X[i, cols - 1 - j] as raw statements: the tiled transpose kernels
+    walk the source backwards along one index (offsets stay relative to the tensor's first byte, so 32-bit
+    arithmetic wraps around harmlessly)."""
+    for load_C, load_b in (([[0, -1], [1, 0]], [rows - 1, 0]), ([[0, 1], [-1, 0]], [0, cols - 1])):
+        chain = W.Chain(
+            name="flip_transpose", dtype=dtype, inputs=[[rows, cols]],
+            ops=[{"kind": "stmts", "shape": [cols, rows],
+                  "stmts": [{"bounds": [cols, rows], "load": (0, load_C, load_b), "store": ([[1, 0], [0, 1]], [0, 0])}]}],
+            values="raw" if dtype == "u8" else "normal",
+        )
+        xs = W.make_inputs(chain)
+        want = oracle.run_chain(chain, xs)
+        ref = xs[0][::-1, :].T if load_b[0] else xs[0][:, ::-1].T
+        assert np.array_equal(want, ref)
+        got, plan = run_gpu(B, chain, xs)
+        assert np.array_equal(got, want.reshape(-1)), (rows, cols, dtype, load_b)
+
+
 def test_dag_with_a_shared_intermediate(B):
     """One transposed tensor feeds a slice and a pad that are joined again: two readers of one intermediate."""
     chain = W.Chain(
