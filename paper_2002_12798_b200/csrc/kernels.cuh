@@ -287,9 +287,11 @@ __device__ __forceinline__ void strip_body(const DevPiece &sp, const PtrTable &p
 //            one b, packs them, and stores 16 bytes along a (full lines of the
 //            destination).
 // The 16-byte chunk index within a row is XOR-ed with (a / (16/ES)) & 7, which
-// makes both the vector stores of phase 1 and the element reads of phase 2
-// bank-conflict-free.  Tiles on the ragged edge are predicated per chunk (the
-// planner only selects this kernel when both extents are multiples of 16/ES).
+// spreads both the vector stores of phase 1 and the element reads of phase 2
+// over all banks (a profiler capture of a full-size transpose still counts
+// 1-2 % conflicting wavefronts, from the rounds of partly filled tiles).  Tiles
+// on the ragged edge are predicated per chunk (the planner only selects this
+// kernel when both extents are multiples of 16/ES).
 // ---------------------------------------------------------------------------
 // the 16-byte chunk index within a tile row is XOR-ed with this function of the row's chunk of a
 template <int CA>
