@@ -308,6 +308,28 @@ int amap_plan_stats(const amap_plan_t *plan, amap_stats *out /* host */);
 /* kernel family chosen for piece k (an amap_kernel_kind) */
 int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind);
 
+/* Launch k of the plan (0 <= k < amap_stats.n_launches), in the order amap_execute enqueues them: which kernel
+ * runs, over how many descriptors and blocks.  For inspection and tests; AMAP_EINVAL for a k out of range. */
+enum {
+  AMAP_LAUNCH_AFFINE = 0,            /* per-unit copy / gather                                         */
+  AMAP_LAUNCH_STRIP = 1,             /* strips of units along one loop                                 */
+  AMAP_LAUNCH_TRANSPOSE = 2,         /* tiled transpose, `access` bytes (16, 8, 4, 2) per global access */
+  AMAP_LAUNCH_TRANSPOSE_SHIFTED = 3, /* tiled transpose onto destination rows that are not 16-byte aligned */
+  AMAP_LAUNCH_TRANSPOSE_REALIGN = 4, /* tiled transpose from source rows that are not 16-byte aligned  */
+  AMAP_LAUNCH_TRANSPOSE_FLAT = 5     /* transpose by panels that are contiguous in the destination     */
+};
+typedef struct amap_launch_info {
+  int32_t kernel;        /* AMAP_LAUNCH_*                                               */
+  int32_t access;        /* bytes per global access (affine / strip: the unit width)    */
+  int32_t n_descriptors; /* descriptors the launch covers                               */
+  int32_t stage;         /* stage of the map the launch belongs to                      */
+  uint32_t n_blocks;
+  int32_t threads;       /* threads per block                                           */
+  int32_t smem_bytes;    /* dynamic shared memory per block (0: the kernel's static tile) */
+  int32_t wide_offsets;  /* 1: 64-bit byte offsets                                      */
+} amap_launch_info;
+int amap_plan_launch_info(const amap_plan_t *plan, int32_t k, amap_launch_info *out /* host */);
+
 /* ---------------------------------------------------------------------------
  * amap_execute: the surviving copy (the data movement Section 2.1 cannot
  * remove and Section 2.2 wants run at full memory bandwidth).

@@ -10,7 +10,7 @@ from __future__ import annotations
 
 import ctypes
 import os
-from ctypes import POINTER, Structure, byref, c_char_p, c_int, c_int32, c_int64, c_uint64, c_void_p
+from ctypes import POINTER, Structure, byref, c_char_p, c_int, c_int32, c_int64, c_uint32, c_uint64, c_void_p
 
 from . import build as _build
 
@@ -22,6 +22,7 @@ COMPOSE_NO_QUASI_AFFINE = 4
 PLAN_NO_PDL = 1
 PLAN_NO_PREFETCH = 2
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
+LAUNCH_NAMES = {0: "affine", 1: "strip", 2: "transpose", 3: "transpose_shifted", 4: "transpose_realign", 5: "transpose_flat"}
 
 EXPORTS = [
     "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",
@@ -30,7 +31,7 @@ EXPORTS = [
     "amap_builder_stmt",
     "amap_builder_opaque", "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_compose_multi",
     "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_device_view", "amap_consume_row_sums", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
-    "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel",
+    "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel", "amap_plan_launch_info",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
 
@@ -96,6 +97,13 @@ class DeviceView(Structure):
 
 class _PlanOpts(Structure):
     _fields_ = [("force_kernel", c_int32), ("pointer_align", c_int32), ("flags", c_int32), ("reserved", c_int32 * 5)]
+
+
+class _LaunchInfo(Structure):
+    _fields_ = [
+        ("kernel", c_int32), ("access", c_int32), ("n_descriptors", c_int32), ("stage", c_int32),
+        ("n_blocks", c_uint32), ("threads", c_int32), ("smem_bytes", c_int32), ("wide_offsets", c_int32),
+    ]
 
 
 class _Stats(Structure):
@@ -411,6 +419,17 @@ class Plan:
             kind = c_int32()
             _check(_lib.amap_plan_piece_kernel(self._h, k, byref(kind)), "amap_plan_piece_kernel")
             out.append(KERNEL_NAMES[kind.value])
+        return out
+
+    def launches(self):
+        """One dict per kernel launch of an execute, in order: kernel name, access width, blocks, threads, ..."""
+        out = []
+        for k in range(self.stats()["n_launches"]):
+            info = _LaunchInfo()
+            _check(_lib.amap_plan_launch_info(self._h, k, byref(info)), "amap_plan_launch_info")
+            d = {name: getattr(info, name) for name, _ in _LaunchInfo._fields_}
+            d["kernel"] = LAUNCH_NAMES[info.kernel]
+            out.append(d)
         return out
 
     def _src_array(self, src_ptrs):

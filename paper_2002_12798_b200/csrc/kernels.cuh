@@ -924,6 +924,95 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
 }
 
 // ---------------------------------------------------------------------------
+// The transpose for pieces whose destination rows follow each other in memory
+// (NHWC -> NCHW: a row is the H*W pixels of one channel), whatever the rows'
+// alignment.  A block takes ALL of a for step_b consecutive b, so that what it
+// writes is ONE contiguous range of the destination; the range starts on a
+// 16-byte boundary because step_b is a multiple of 16/ES.  Dynamic shared
+// memory holds that range as it will lie in memory:
+//   phase 1  16-byte loads along b (step_b * ES contiguous bytes per a),
+//            scattered element by element into the rows of the image;
+//   phase 2  a linear copy of the image, 16 bytes per thread: whole lines,
+//            whatever the length of a row.
+// The lanes that share one a are the first 2^tile_ca of a group (tile_ca holds
+// the logarithm here).
+// ---------------------------------------------------------------------------
+template <int ES, int THREADS>
+__device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const PtrTable &ptrs) {
+  constexpr int EPU = 16 / ES;
+  // loads a thread keeps in flight: four in 32 registers where eight blocks of 256 threads share an SM; eight where
+  // the panel's size leaves room for two to four blocks of 512 threads anyway
+  constexpr int U = THREADS == 256 ? 4 : 8;
+  using E = typename Unit<ES>::T;
+  extern __shared__ __align__(128) unsigned char panel[];
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_b);
+  const uint32_t b0 = (t - q * sp.tiles_b) * sp.step_b;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const uint32_t ext_a = sp.ext_a, nb = min(sp.step_b, sp.ext_b - b0);
+  const uint32_t row_bytes = ext_a * ES;
+  const int lg = sp.tile_ca;
+  const uint32_t cb = threadIdx.x & ((1u << lg) - 1u), a_step = THREADS >> lg;
+  const bool lane_on = cb * EPU < nb;
+  const FastDiv fa = sp.fd_a_in;
+  const bool merged = fa.d < ext_a;
+  const char *src = ptrs.src[sp.input] + sbase + (int64_t)b0 * ES + (int64_t)cb * 16;
+  char *dst = ptrs.dst(sp.out) + dbase + (int64_t)b0 * sp.db[0];
+  unsigned char *column = panel + cb * EPU * row_bytes;  // where this lane's first element of a = 0 goes
+  pdl_wait();
+
+  // rounds of equal length: ten loads are five and five, not eight and two
+  const uint32_t per_thread = (ext_a + a_step - 1) / a_step, rounds = (per_thread + U - 1) / U;
+  const int u_round = (int)((per_thread + rounds - 1) / rounds);
+  for (uint32_t a0 = threadIdx.x >> lg; lane_on && a0 < ext_a; a0 += (uint32_t)u_round * a_step) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t a = a0 + (uint32_t)u * a_step;
+      if (u < u_round && a < ext_a) {
+        int64_t off = (int64_t)a * sp.sa[0];
+        if (merged) {
+          const uint32_t a_hi = fast_div(a, fa);
+          off = (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1];
+        }
+        v[u] = load_16(src + off);
+      }
+    }
+    issue_barrier();
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t a = a0 + (uint32_t)u * a_step;
+      if (u < u_round && a < ext_a) {
+        unsigned char *p = column + a * ES;
+        const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int e = 0; e < EPU; ++e) {
+          E x;
+          if constexpr (ES == 4) x = w[e];
+          else x = (E)((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu));
+          *reinterpret_cast<E *>(p) = x;
+          p += row_bytes;
+        }
+      }
+    }
+  }
+  __syncthreads();
+  const uint32_t n16 = nb / EPU * ext_a;  // nb is a multiple of EPU: the range is a whole number of 16-byte units
+#pragma unroll 4
+  for (uint32_t i = threadIdx.x; i < n16; i += THREADS)
+    __stcs(reinterpret_cast<uint4 *>(dst) + i, reinterpret_cast<const uint4 *>(panel)[i]);
+}
+
+// ---------------------------------------------------------------------------
 // The tiled transpose for pieces whose SOURCE rows are not 16-byte aligned but
 // whose destination rows are (NCHW -> NHWC with an odd H*W: 7x7, 35x35, 55x55
 // maps).  Phase 1 still loads aligned 16-byte chunks: the 16 lanes that share a
@@ -1216,6 +1305,30 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_realign_one(
                                                                                  PtrTable ptrs) {
   pdl_launch_dependents();
   transpose_realign_body<ES>(p, ptrs);
+}
+
+// The flat-destination transpose runs with the dynamic shared memory its launch asks for: small panels with eight
+// blocks of 256 threads per SM (32 registers per thread), large ones with blocks of 512 threads (64 registers).
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_param(const __grid_constant__ LaunchDesc ld,
+                                                                                    PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_flat_body<ES, THREADS>(param_piece(ld), ptrs);
+}
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_table(const DevPiece *__restrict__ table,
+                                                                                    int first_piece, int n_pieces,
+                                                                                    PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_flat_body<ES, THREADS>(sp, ptrs);
+}
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_one(const __grid_constant__ DevPiece p,
+                                                                                  PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_flat_body<ES, THREADS>(p, ptrs);
 }
 
 }  // namespace amap

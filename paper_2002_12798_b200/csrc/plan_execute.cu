@@ -36,12 +36,15 @@ struct Launch {
   int kind;  // DevKind
   int unit;  // bytes per item (affine kernel) / element size (transpose kernel)
   int cons;  // affine / strip kernel: constraint slots evaluated per unit (0, 2 or kDevMaxCons)
-             // transpose kernel: bytes per global access (16, 8, 4, 2) or 0 for the shifted-row kernel
+             // transpose kernel: bytes per global access (16, 8, 4, 2), 0 for the shifted-row kernel, -1 for the
+             // realigning kernel, -2 for the flat-destination kernel
   int wide;  // affine kernel: 1 when a byte offset can reach 4 GiB (64-bit offsets)
   int first_piece;
   int n_pieces;
   uint32_t n_blocks;
   int stage;  // which stage of the map this launch belongs to
+  int threads = 0;  // flat-destination transpose only: block size and dynamic shared memory of the launch
+  int smem = 0;
 };
 
 struct amap_plan_t {
@@ -392,6 +395,93 @@ static bool set_transpose_tiles(DevPiece *d, int ca, bool even) {
   return true;
 }
 
+// The flat-destination kernel for a transpose descriptor built with single elements as units: b is one loop whose
+// rows follow each other in the destination, every source access is an aligned 16-byte chunk along b, and every
+// panel (all of a by step_b of b) starts on a 16-byte boundary of the destination.  Chooses step_b and the lanes
+// per a; returns false when the piece does not qualify.
+constexpr int kFlatMaxPanelBytes = 100 * 1024;  // two blocks per SM
+static bool set_flat_panels(DevPiece *d) {
+  const int es = d->unit_bytes, epu = 16 / es;
+  if (d->fd_b_in.d < d->ext_b || d->db[0] != (int64_t)d->ext_a * es || d->ext_b % epu) return false;
+  if (d->soff % 16 || d->sa[0] % 16 || d->sa[1] % 16 || d->doff % 16) return false;
+  for (int j = 0; j < d->n_loops; ++j)
+    if (d->sstride[j] % 16 || d->dstride[j] % 16) return false;
+  const uint64_t row_bytes = (uint64_t)d->ext_a * es;
+  if (row_bytes * epu > (uint64_t)kFlatMaxPanelBytes) return false;
+  // step_b: 16/es elements times a power of two.  Measured on 2-byte elements: panels near 12-24 KB run best (eight
+  // blocks of 256 threads per SM), but 64 bytes of b per a are worth a larger panel (rows of 1.4-2.4 KB: 47-78 KB
+  // panels, two or four blocks of 512 threads per SM); with 32 bytes of b the shifted kernel is as fast or faster.
+  const uint32_t min_bt = 64u / es, max_bt = 256u / es;
+  if (row_bytes * min_bt > (uint64_t)kFlatMaxPanelBytes || d->ext_b < min_bt) return false;
+  uint32_t bt = min_bt;
+  int lg = 2;
+  while (bt * 2 <= max_bt && bt * 2 <= d->ext_b && row_bytes * bt * 2 <= 24u * 1024u) {
+    bt *= 2;
+    ++lg;
+  }
+  d->tr_unit = -2;
+  d->tile_ca = lg;
+  d->step_b = bt;
+  d->tiles_a = 1;
+  d->tiles_b = (d->ext_b + bt - 1) / bt;
+  d->fd_tiles_a = make_fastdiv(1);
+  d->fd_tiles_b = make_fastdiv(d->tiles_b);
+  unsigned __int128 blocks = d->tiles_b;
+  for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
+  if (blocks > 0x7FFFFFFFull) return false;
+  // a handful of large panels would leave most SMs idle: the tiled kernels cut such a piece finer
+  if (row_bytes * bt > 24u * 1024u && blocks < (unsigned __int128)kDefaultSms) return false;
+  d->n_blocks = (uint32_t)blocks;
+  d->n_items = (uint64_t)blocks;
+  return true;
+}
+static int flat_panel_bytes(const DevPiece &d) { return (int)((uint64_t)d.step_b * d.ext_a * d.unit_bytes); }
+static int flat_threads(int panel_bytes) { return panel_bytes > 24 * 1024 ? 512 : 256; }
+
+// the flat-destination kernel's address arithmetic for one block, replayed on the host
+static bool check_flat_block(const DevPiece &d, uint32_t blk, int threads, int64_t in_bytes, int64_t out_bytes) {
+  const int es = d.unit_bytes, epu = 16 / es;
+  if ((es != 2 && es != 4) || d.step_b == 0 || d.step_b % epu || d.ext_b % epu || d.tiles_b == 0 || d.tile_ca < 0 ||
+      d.tile_ca > 5 || ((uint32_t)epu << d.tile_ca) < d.step_b || (threads != 256 && threads != 512) ||
+      (uint64_t)d.tiles_b * d.step_b < d.ext_b || flat_panel_bytes(d) > kFlatMaxPanelBytes)
+    return false;
+  uint32_t t = blk;
+  uint32_t q = host_fast_div(t, d.fd_tiles_b);
+  if (q != t / d.tiles_b) return false;
+  const uint32_t b0 = (t - q * d.tiles_b) * d.step_b;
+  t = q;
+  int64_t sbase = d.soff, dbase = d.doff;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    q = host_fast_div(t, d.fd[k]);
+    if (q != t / d.ext[k]) return false;
+    const uint32_t i = t - q * d.ext[k];
+    t = q;
+    sbase += (int64_t)i * d.sstride[k];
+    dbase += (int64_t)i * d.dstride[k];
+  }
+  if (t != 0 || b0 >= d.ext_b) return false;
+  const uint32_t nb = std::min<uint32_t>(d.step_b, d.ext_b - b0);
+  const int64_t row_bytes = (int64_t)d.ext_a * es, panel = (int64_t)nb * row_bytes;
+  // phase 2: the panel is one aligned range of the destination, a whole number of 16-byte units
+  const int64_t D0 = dbase + (int64_t)b0 * d.db[0];
+  if (d.db[0] != row_bytes || D0 % 16 || panel % 16 || D0 < 0 || D0 + panel > out_bytes) return false;
+  // phase 1: every lane's loads and the elements it scatters
+  const uint32_t lanes = 1u << d.tile_ca;
+  for (uint32_t a = 0; a < d.ext_a; ++a) {
+    const uint32_t a_hi = host_fast_div(a, d.fd_a_in);
+    if (a_hi != a / d.fd_a_in.d) return false;
+    const int64_t off = d.fd_a_in.d < d.ext_a ? (int64_t)(a - a_hi * d.fd_a_in.d) * d.sa[0] + (int64_t)a_hi * d.sa[1]
+                                               : (int64_t)a * d.sa[0];
+    for (uint32_t cb = 0; cb < lanes && cb * epu < nb; ++cb) {
+      const int64_t g = sbase + (int64_t)b0 * es + (int64_t)cb * 16 + off;
+      if (g % 16 || g < 0 || g + 16 > in_bytes) return false;
+      const int64_t last = ((int64_t)cb * epu + epu - 1) * row_bytes + (int64_t)a * es;  // the lane's last element
+      if (last + es > panel) return false;
+    }
+  }
+  return true;
+}
+
 // A 16-byte transpose piece whose extent along a leaves a remainder of at most half a tile is cut in two: whole
 // tiles, and the remainder as a piece of its own on the narrow tile (64 bytes of a by 256 elements of b), which
 // would otherwise travel in half-empty tiles.  Returns false when the piece stays as it is.
@@ -511,6 +601,11 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
       }
     }
   }
+  // destination rows that follow each other in memory, source rows aligned: the flat-destination kernel
+  // (tr_unit = -2), whatever the alignment of the destination rows
+  if ((es == 2 || es == 4) && ptr_align >= 16 && try_build(ia_hi, -1, es) &&
+      set_flat_panels(d))
+    return true;
   if (try_unit(8)) return true;
   // destination rows misaligned, source rows aligned: the shifted-destination kernel (tr_unit = 0; it stores whole
   // slots of the destination's own 16-byte grid; rows at least one slot long, so that a slot spans two rows at most)
@@ -625,6 +720,7 @@ static bool check_realign_block(const DevPiece &d, uint32_t blk, int64_t in_byte
 
 // the kernel's address arithmetic for one block, replayed on the host
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
+  if (d.tr_unit == -2) return check_flat_block(d, blk, flat_threads(flat_panel_bytes(d)), in_bytes, out_bytes);
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   if (d.tr_unit < 0) return check_realign_block(d, blk, in_bytes, out_bytes);
   const int es = d.unit_bytes, epu = 16 / es, ca = d.tile_ca, ta = ca * epu;
@@ -745,7 +841,7 @@ static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
 static int plan_stage_transposes(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
-  for (int access : {16, 8, 4, 2, 0, -1})
+  for (int access : {16, 8, 4, 2, 0, -1, -2})
     for (int wide = 0; wide < 2; ++wide) {
       Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
       std::vector<DevPiece> transposes, fills;
@@ -783,6 +879,10 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
       for (const DevPiece &d : fills)
         if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
       for (size_t q : taken) c.placed[q] = 1;
+      if (access == -2) {  // the block size and the shared memory of the largest panel serve the whole launch
+        for (const DevPiece &d : transposes) L.smem = std::max(L.smem, flat_panel_bytes(d));
+        L.threads = flat_threads(L.smem);
+      }
       c.pl->launches.push_back(L);
     }
   return AMAP_OK;
@@ -1060,6 +1160,28 @@ extern "C" int amap_plan_stats(const amap_plan_t *plan, amap_stats *out) {
   return AMAP_OK;
 }
 
+extern "C" int amap_plan_launch_info(const amap_plan_t *plan, int32_t k, amap_launch_info *out) {
+  if (!plan || !out || k < 0 || k >= (int32_t)plan->launches.size()) return AMAP_EINVAL;
+  const Launch &L = plan->launches[k];
+  memset(out, 0, sizeof *out);
+  if (L.kind == kDevTranspose) {
+    out->kernel = L.cons == -2 ? AMAP_LAUNCH_TRANSPOSE_FLAT : L.cons == -1 ? AMAP_LAUNCH_TRANSPOSE_REALIGN
+                : L.cons == 0 ? AMAP_LAUNCH_TRANSPOSE_SHIFTED : AMAP_LAUNCH_TRANSPOSE;
+    out->access = L.cons > 0 ? L.cons : 16;
+    out->threads = L.threads ? L.threads : kTransposeThreads;
+  } else {
+    out->kernel = L.kind == kDevStrip ? AMAP_LAUNCH_STRIP : AMAP_LAUNCH_AFFINE;
+    out->access = L.unit;
+    out->threads = kAffineThreads;
+  }
+  out->n_descriptors = L.n_pieces;
+  out->stage = L.stage;
+  out->n_blocks = L.n_blocks;
+  out->smem_bytes = L.smem;
+  out->wide_offsets = L.wide;
+  return AMAP_OK;
+}
+
 extern "C" int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_t *kind) {
   if (!plan || !kind || k < 0 || k >= (int32_t)plan->piece_kernel.size()) return AMAP_EINVAL;
   *kind = plan->piece_kernel[k];
@@ -1070,10 +1192,11 @@ extern "C" int amap_plan_piece_kernel(const amap_plan_t *plan, int32_t k, int32_
 // become resident while the kernel before it on the stream drains; the kernels wait (griddepcontrol.wait) for that
 // kernel's completion before they touch a caller buffer.
 template <typename... P, typename... A>
-static void launch(void (*kernel)(P...), uint32_t blocks, int threads, cudaStream_t s, bool pdl, A... args) {
+static void launch_smem(void (*kernel)(P...), uint32_t blocks, int threads, int smem, cudaStream_t s, bool pdl, A... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(blocks);
   cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = (size_t)smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1081,6 +1204,11 @@ static void launch(void (*kernel)(P...), uint32_t blocks, int threads, cudaStrea
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
   cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+template <typename... P, typename... A>
+static void launch(void (*kernel)(P...), uint32_t blocks, int threads, cudaStream_t s, bool pdl, A... args) {
+  launch_smem(kernel, blocks, threads, 0, s, pdl, args...);
 }
 
 // Where a launch finds its descriptors: by value in the kernel parameters (`ld`), or in a table in global memory.
@@ -1132,9 +1260,30 @@ static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const
   }
 }
 
+// The flat-destination kernel: dynamic shared memory above the default limit has to be allowed per function (a
+// function attribute of the current device's context; setting it again costs a host call and nothing else).
+template <int ES>
+static void launch_transpose_flat(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  if constexpr (ES == 2 || ES == 4) {
+    auto go = [&](auto kernel, auto... args) {
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
+      launch_smem(kernel, L.n_blocks, L.threads, L.smem, s, pdl, args...);
+    };
+    auto pick = [&](auto threads) {
+      constexpr int T = decltype(threads)::value;
+      if (ds.ld && ds.ld->n_pieces == 1) go(amap_transpose_flat_one<ES, T>, ds.ld->piece[0], pt);
+      else if (ds.ld) go(amap_transpose_flat_param<ES, T>, *ds.ld, pt);
+      else go(amap_transpose_flat_table<ES, T>, ds.table, L.first_piece, L.n_pieces, pt);
+    };
+    if (L.threads == 512) pick(std::integral_constant<int, 512>());
+    else pick(std::integral_constant<int, 256>());
+  }
+}
+
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
+    case -2: launch_transpose_flat<ES>(ds, L, pt, s, pdl); return;
     case -1:
       if constexpr (ES <= 4)
         AMAP_LAUNCH(amap_transpose_realign_one, amap_transpose_realign_param, amap_transpose_realign_table, kTransposeThreads, ES);

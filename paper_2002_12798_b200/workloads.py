@@ -339,6 +339,23 @@ def reduced_configs() -> dict:
                  {"kind": "pad", "src": 1, "lo": [0, 0, 0, 0], "hi": [0, 0, 0, 2]}],
             values="normal", seed=BASE_SEED + 2,
         ),
+        # panels that are contiguous in the destination (the flat-destination transpose): large panels on blocks of
+        # 512 threads, a source that is a window of a larger tensor (two strides along the pixels), two batch loops,
+        # a last panel with fewer channels than the others, 4-byte elements
+        "c2_inv_flat_big": c2_nhwc_to_nchw(N=20, C=256, H=27, W=27),
+        "c2_inv_flat_big_f32": c2_nhwc_to_nchw(N=19, C=136, H=19, W=21, dtype="fp32"),
+        "c2_inv_flat_window": Chain(
+            name="c2_inv_flat_window", dtype="bf16", inputs=[[3, 9, 12, 104]],
+            ops=[{"kind": "slice", "src": 0, "start": [0, 1, 2, 0], "stop": [3, 8, 9, 104], "step": [1, 1, 1, 1]},
+                 {"kind": "transpose", "src": 1, "perm": [0, 3, 1, 2]}],
+            values="normal", seed=BASE_SEED + 2,
+        ),
+        "c2_inv_flat_5d": Chain(
+            name="c2_inv_flat_5d", dtype="fp16", inputs=[[2, 4, 5, 7, 168]],
+            ops=[{"kind": "slice", "src": 0, "start": [0, 1, 0, 0, 0], "stop": [2, 4, 5, 7, 168], "step": [1, 1, 1, 1, 1]},
+                 {"kind": "transpose", "src": 1, "perm": [0, 1, 4, 2, 3]}],
+            values="normal", seed=BASE_SEED + 2,
+        ),
         "c2_fwd_odd_u8": c2_nchw_to_nhwc(N=2, C=64, H=11, W=13, dtype="u8"),
         "c2_fwd_odd_f32b": c2_nchw_to_nhwc(N=2, C=36, H=7, W=9, dtype="fp32"),
         "c2_fwd_narrow": c2_nchw_to_nhwc(N=2, C=72, H=14, W=14),

@@ -429,6 +429,23 @@ def test_launch_with_more_pieces_than_fit_the_kernel_parameters(B):
     assert np.array_equal(got, want.reshape(-1))
 
 
+def test_flat_destination_transposes_from_the_descriptor_table(B):
+    """Twenty NHWC operands joined along the batch and taken to NCHW (7x7 maps: rows of 98 bytes): twenty pieces
+    of the flat-destination transpose in one launch, their descriptors read from the plan's table."""
+    n_in = 20
+    chain = W.Chain(
+        name="wide_concat_flat", dtype="bf16", inputs=[[2, 7, 7, 72]] * n_in,
+        ops=[{"kind": "concat", "srcs": list(range(n_in)), "axis": 0}, {"kind": "transpose", "src": n_in, "perm": [0, 3, 1, 2]}],
+        values="normal",
+    )
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    got, plan = run_gpu(B, chain, xs)
+    launches = plan.launches()
+    assert len(launches) == 1 and launches[0]["kernel"] == "transpose_flat" and launches[0]["n_descriptors"] == n_in
+    assert np.array_equal(got, want.reshape(-1))
+
+
 def test_three_guards_in_one_piece(B):
     """A 3-D window gather written as one raw guarded statement: three guards, so the kernels' larger
     constraint variant runs."""

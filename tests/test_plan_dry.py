@@ -51,6 +51,46 @@ def test_shifted_transpose_for_misaligned_destination_rows():
     assert k["gather"] == 1
 
 
+def launch_of(chain):
+    launches = B.compose_chain(chain).plan(device=-1).launches()
+    assert len(launches) == 1
+    return launches[0]
+
+
+def test_transpose_kernel_per_shape():
+    """NHWC -> NCHW: which of the transpose kernels a shape gets (amap_plan_launch_info), with the block size and
+    the shared memory of the flat-destination kernel's panels."""
+    inv = W.c2_nhwc_to_nchw
+    L = launch_of(inv(N=32, C=256, H=56, W=56))  # rows of 6272 bytes, aligned on both sides
+    assert (L["kernel"], L["access"], L["threads"], L["smem_bytes"]) == ("transpose", 16, 256, 0)
+    # 35x35 maps: rows of 2450 bytes; a panel of all 1225 pixels by 32 channels is 78400 bytes, 9 panels per image
+    L = launch_of(inv(N=64, C=288, H=35, W=35))
+    assert (L["kernel"], L["threads"], L["smem_bytes"], L["n_blocks"]) == ("transpose_flat", 512, 78400, 64 * 9)
+    # 14x14 maps: rows of 392 bytes; 32 channels make a panel of 12544 bytes (64 channels would pass 24 KB)
+    L = launch_of(inv(N=64, C=1024, H=14, W=14))
+    assert (L["kernel"], L["threads"], L["smem_bytes"], L["n_blocks"]) == ("transpose_flat", 256, 12544, 64 * 32)
+    # 7x7 maps: rows of 98 bytes; 128 channels (256 bytes per pixel, the most a panel takes) make 12544 bytes
+    L = launch_of(inv(N=64, C=2048, H=7, W=7))
+    assert (L["kernel"], L["threads"], L["smem_bytes"], L["n_blocks"]) == ("transpose_flat", 256, 12544, 64 * 16)
+    # 4-byte elements: 64 bytes of the source run are 16 channels
+    L = launch_of(inv(N=19, C=136, H=19, W=21, dtype="fp32"))
+    assert (L["kernel"], L["threads"], L["smem_bytes"], L["n_blocks"]) == ("transpose_flat", 512, 16 * 399 * 4, 19 * 9)
+    # rows too long for a panel of 64 bytes per pixel (71x71: 10082 bytes): the shifted-destination kernel
+    assert launch_of(inv(N=32, C=192, H=71, W=71))["kernel"] == "transpose_shifted"
+    # a handful of large panels (2 images x 8 panels of 46 KB) would leave most SMs idle: shifted-destination too
+    assert launch_of(inv(N=2, C=256, H=27, W=27))["kernel"] == "transpose_shifted"
+    assert launch_of(inv(N=20, C=256, H=27, W=27))["kernel"] == "transpose_flat"
+    # fewer channels than a panel's 64 bytes, or a channel count that is no multiple of 16 bytes
+    assert launch_of(inv(N=2, C=24, H=5, W=13))["kernel"] == "transpose_shifted"
+    L = launch_of(inv(N=2, C=68, H=14, W=14))
+    assert (L["kernel"], L["access"]) == ("transpose", 8)
+    # the other direction: source rows misaligned, destination rows aligned
+    assert launch_of(W.c2_nchw_to_nhwc(N=4, C=256, H=27, W=27))["kernel"] == "transpose_realign"
+    # other families
+    assert launch_of(W.full_configs()["c5"])["kernel"] == "strip"
+    assert launch_of(W.full_configs()["c3"])["kernel"] in ("affine", "strip")
+
+
 def test_remainders_of_at_most_half_a_tile_become_pieces_of_their_own():
     """The 16-byte transpose kernel's tile spans 128 bytes of the destination run.  An extent that leaves at most
     64 bytes over is cut: whole tiles, plus the remainder on the 64-byte tile."""
