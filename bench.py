@@ -343,6 +343,7 @@ def config_rows(torch, B, device, stream, l2, peak, names, flags=0, extras=False
         row["bytes"] = total
         row["launches"] = case.launches
         row["kernels"] = {k: sum(t["kernels"][k] for t in sts) for k in sts[0]["kernels"]}
+        row["launch_kernels"] = [l["kernel"] for p in case.plans for l in p.launches()]
         row["buffer_sets"] = n_sets
         ours = outs[0][0].clone() if case.single else None
 

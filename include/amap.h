@@ -316,7 +316,8 @@ enum {
   AMAP_LAUNCH_TRANSPOSE = 2,         /* tiled transpose, `access` bytes (16, 8, 4, 2) per global access */
   AMAP_LAUNCH_TRANSPOSE_SHIFTED = 3, /* tiled transpose onto destination rows that are not 16-byte aligned */
   AMAP_LAUNCH_TRANSPOSE_REALIGN = 4, /* tiled transpose from source rows that are not 16-byte aligned  */
-  AMAP_LAUNCH_TRANSPOSE_FLAT = 5     /* transpose by panels that are contiguous in the destination     */
+  AMAP_LAUNCH_TRANSPOSE_FLAT = 5,    /* transpose by panels that are contiguous in the destination     */
+  AMAP_LAUNCH_TRANSPOSE_FLAT_SOURCE = 6 /* transpose by panels that are contiguous in the source       */
 };
 typedef struct amap_launch_info {
   int32_t kernel;        /* AMAP_LAUNCH_*                                               */

@@ -22,7 +22,7 @@ COMPOSE_NO_QUASI_AFFINE = 4
 PLAN_NO_PDL = 1
 PLAN_NO_PREFETCH = 2
 KERNEL_NAMES = {1: "gather", 2: "copy", 3: "transpose", 4: "fill"}
-LAUNCH_NAMES = {0: "affine", 1: "strip", 2: "transpose", 3: "transpose_shifted", 4: "transpose_realign", 5: "transpose_flat"}
+LAUNCH_NAMES = {0: "affine", 1: "strip", 2: "transpose", 3: "transpose_shifted", 4: "transpose_realign", 5: "transpose_flat", 6: "transpose_flat_source"}
 
 EXPORTS = [
     "amap_builder_create", "amap_builder_destroy", "amap_builder_input", "amap_builder_reshape",

@@ -1013,6 +1013,85 @@ __device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const Pt
 }
 
 // ---------------------------------------------------------------------------
+// The mirror image: pieces whose SOURCE rows follow each other in memory
+// (NCHW -> NHWC: a row is the H*W pixels of one channel), whatever the rows'
+// alignment.  A block takes ALL of b for step_b consecutive a (the descriptor's
+// step_b counts elements of a here), so that what it reads is ONE contiguous,
+// 16-byte aligned range of the source:
+//   phase 1  a linear copy of that range into shared memory;
+//   phase 2  per b, the 16/ES elements of consecutive a are gathered from the
+//            rows of the image, packed and stored as 16 bytes along a
+//            (step_b * ES contiguous bytes of the destination per b).
+// ---------------------------------------------------------------------------
+template <int ES, int THREADS>
+__device__ __forceinline__ void transpose_flat_source_body(const DevPiece &sp, const PtrTable &ptrs) {
+  constexpr int EPU = 16 / ES;
+  constexpr int U = THREADS == 256 ? 4 : 8;
+  using E = typename Unit<ES>::T;
+  extern __shared__ __align__(128) unsigned char panel[];
+
+  uint32_t t = blockIdx.x - sp.first_block;
+  uint32_t q = fast_div(t, sp.fd_tiles_a);
+  const uint32_t a0 = (t - q * sp.tiles_a) * sp.step_b;
+  t = q;
+  int64_t sbase = sp.soff, dbase = sp.doff;
+  for (int k = sp.n_loops - 1; k >= 0; --k) {
+    q = fast_div(t, sp.fd[k]);
+    const uint32_t i = t - q * sp.ext[k];
+    t = q;
+    sbase += (int64_t)i * sp.sstride[k];
+    dbase += (int64_t)i * sp.dstride[k];
+  }
+  const uint32_t ext_b = sp.ext_b, na = min(sp.step_b, sp.ext_a - a0);
+  const uint32_t row_bytes = ext_b * ES;
+  const char *src = ptrs.src[sp.input] + sbase + (int64_t)a0 * sp.sa[0];
+  pdl_wait();
+
+  const uint32_t n16 = na / EPU * ext_b;  // na is a multiple of EPU: the range is a whole number of 16-byte units
+  for (uint32_t i0 = threadIdx.x; i0 < n16; i0 += U * THREADS) {
+    uint4 v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (i0 + u * THREADS < n16) v[u] = load_16(src + (size_t)(i0 + u * THREADS) * 16);
+    issue_barrier();
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (i0 + u * THREADS < n16) reinterpret_cast<uint4 *>(panel)[i0 + u * THREADS] = v[u];
+  }
+  __syncthreads();
+
+  const int lg = sp.tile_ca;
+  const uint32_t ca = threadIdx.x & ((1u << lg) - 1u), b_step = THREADS >> lg;
+  const bool lane_on = ca * EPU < na;
+  const FastDiv fb = sp.fd_b_in;
+  const bool merged = fb.d < ext_b;
+  char *dst = ptrs.dst(sp.out) + dbase + (int64_t)a0 * ES + (int64_t)ca * 16;
+  const unsigned char *column = panel + ca * EPU * row_bytes;  // this lane's first row of the image
+#pragma unroll 2
+  for (uint32_t b = threadIdx.x >> lg; lane_on && b < ext_b; b += b_step) {
+    const unsigned char *p = column + b * ES;
+    uint32_t w[4];
+    if constexpr (ES == 4) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) w[e] = *reinterpret_cast<const uint32_t *>(p + e * row_bytes);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t lo = *reinterpret_cast<const uint16_t *>(p + (2 * e) * row_bytes);
+        const uint32_t hi = *reinterpret_cast<const uint16_t *>(p + (2 * e + 1) * row_bytes);
+        w[e] = lo | (hi << 16);
+      }
+    }
+    int64_t off = (int64_t)b * sp.db[0];
+    if (merged) {
+      const uint32_t b_hi = fast_div(b, fb);
+      off = (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1];
+    }
+    __stcs(reinterpret_cast<uint4 *>(dst + off), make_uint4(w[0], w[1], w[2], w[3]));
+  }
+}
+
+// ---------------------------------------------------------------------------
 // The tiled transpose for pieces whose SOURCE rows are not 16-byte aligned but
 // whose destination rows are (NCHW -> NHWC with an odd H*W: 7x7, 35x35, 55x55
 // maps).  Phase 1 still loads aligned 16-byte chunks: the 16 lanes that share a
@@ -1329,6 +1408,27 @@ __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpos
                                                                                   PtrTable ptrs) {
   pdl_launch_dependents();
   transpose_flat_body<ES, THREADS>(p, ptrs);
+}
+
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2)
+    amap_transpose_flat_source_param(const __grid_constant__ LaunchDesc ld, PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_flat_source_body<ES, THREADS>(param_piece(ld), ptrs);
+}
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2)
+    amap_transpose_flat_source_table(const DevPiece *__restrict__ table, int first_piece, int n_pieces, PtrTable ptrs) {
+  __shared__ DevPiece sp;
+  pdl_launch_dependents();
+  fetch_piece(table, first_piece, n_pieces, &sp);
+  transpose_flat_source_body<ES, THREADS>(sp, ptrs);
+}
+template <int ES, int THREADS>
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2)
+    amap_transpose_flat_source_one(const __grid_constant__ DevPiece p, PtrTable ptrs) {
+  pdl_launch_dependents();
+  transpose_flat_source_body<ES, THREADS>(p, ptrs);
 }
 
 }  // namespace amap

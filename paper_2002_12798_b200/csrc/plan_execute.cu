@@ -37,7 +37,7 @@ struct Launch {
   int unit;  // bytes per item (affine kernel) / element size (transpose kernel)
   int cons;  // affine / strip kernel: constraint slots evaluated per unit (0, 2 or kDevMaxCons)
              // transpose kernel: bytes per global access (16, 8, 4, 2), 0 for the shifted-row kernel, -1 for the
-             // realigning kernel, -2 for the flat-destination kernel
+             // realigning kernel, -2 for the flat-destination kernel, -3 for the flat-source kernel
   int wide;  // affine kernel: 1 when a byte offset can reach 4 GiB (64-bit offsets)
   int first_piece;
   int n_pieces;
@@ -435,7 +435,42 @@ static bool set_flat_panels(DevPiece *d) {
   d->n_items = (uint64_t)blocks;
   return true;
 }
-static int flat_panel_bytes(const DevPiece &d) { return (int)((uint64_t)d.step_b * d.ext_a * d.unit_bytes); }
+// The mirror image for the flat-source kernel (tr_unit = -3): a is one loop whose rows follow each other in the
+// SOURCE, every destination access is an aligned 16-byte chunk along a; step_b holds the elements of a per panel.
+static bool set_flat_source_panels(DevPiece *d) {
+  const int es = d->unit_bytes, epu = 16 / es;
+  if (d->fd_a_in.d < d->ext_a || d->sa[0] != (int64_t)d->ext_b * es || d->ext_a % epu) return false;
+  if (d->doff % 16 || d->db[0] % 16 || d->db[1] % 16 || d->soff % 16) return false;
+  for (int j = 0; j < d->n_loops; ++j)
+    if (d->sstride[j] % 16 || d->dstride[j] % 16) return false;
+  const uint64_t row_bytes = (uint64_t)d->ext_b * es;
+  const uint32_t min_at = 64u / es, max_at = 256u / es;
+  if (row_bytes * min_at > (uint64_t)kFlatMaxPanelBytes || d->ext_a < min_at) return false;
+  uint32_t at = min_at;
+  int lg = 2;
+  while (at * 2 <= max_at && at * 2 <= d->ext_a && row_bytes * at * 2 <= 24u * 1024u) {
+    at *= 2;
+    ++lg;
+  }
+  d->tr_unit = -3;
+  d->tile_ca = lg;
+  d->step_b = at;
+  d->tiles_b = 1;
+  d->tiles_a = (d->ext_a + at - 1) / at;
+  d->fd_tiles_b = make_fastdiv(1);
+  d->fd_tiles_a = make_fastdiv(d->tiles_a);
+  unsigned __int128 blocks = d->tiles_a;
+  for (int j = 0; j < d->n_loops; ++j) blocks *= d->ext[j];
+  if (blocks > 0x7FFFFFFFull) return false;
+  if (row_bytes * at > 24u * 1024u && blocks < (unsigned __int128)kDefaultSms) return false;
+  d->n_blocks = (uint32_t)blocks;
+  d->n_items = (uint64_t)blocks;
+  return true;
+}
+// bytes of a panel of either flat kernel: step_b elements of the panelled index by all of the other
+static int flat_panel_bytes(const DevPiece &d) {
+  return (int)((uint64_t)d.step_b * (d.tr_unit == -3 ? d.ext_b : d.ext_a) * d.unit_bytes);
+}
 static int flat_threads(int panel_bytes) { return panel_bytes > 24 * 1024 ? 512 : 256; }
 
 // the flat-destination kernel's address arithmetic for one block, replayed on the host
@@ -476,6 +511,50 @@ static bool check_flat_block(const DevPiece &d, uint32_t blk, int threads, int64
       const int64_t g = sbase + (int64_t)b0 * es + (int64_t)cb * 16 + off;
       if (g % 16 || g < 0 || g + 16 > in_bytes) return false;
       const int64_t last = ((int64_t)cb * epu + epu - 1) * row_bytes + (int64_t)a * es;  // the lane's last element
+      if (last + es > panel) return false;
+    }
+  }
+  return true;
+}
+
+// the flat-source kernel's address arithmetic for one block, replayed on the host
+static bool check_flat_source_block(const DevPiece &d, uint32_t blk, int threads, int64_t in_bytes, int64_t out_bytes) {
+  const int es = d.unit_bytes, epu = 16 / es;
+  if ((es != 2 && es != 4) || d.step_b == 0 || d.step_b % epu || d.ext_a % epu || d.tiles_a == 0 || d.tile_ca < 0 ||
+      d.tile_ca > 5 || ((uint32_t)epu << d.tile_ca) < d.step_b || (threads != 256 && threads != 512) ||
+      (uint64_t)d.tiles_a * d.step_b < d.ext_a || flat_panel_bytes(d) > kFlatMaxPanelBytes)
+    return false;
+  uint32_t t = blk;
+  uint32_t q = host_fast_div(t, d.fd_tiles_a);
+  if (q != t / d.tiles_a) return false;
+  const uint32_t a0 = (t - q * d.tiles_a) * d.step_b;
+  t = q;
+  int64_t sbase = d.soff, dbase = d.doff;
+  for (int k = d.n_loops - 1; k >= 0; --k) {
+    q = host_fast_div(t, d.fd[k]);
+    if (q != t / d.ext[k]) return false;
+    const uint32_t i = t - q * d.ext[k];
+    t = q;
+    sbase += (int64_t)i * d.sstride[k];
+    dbase += (int64_t)i * d.dstride[k];
+  }
+  if (t != 0 || a0 >= d.ext_a) return false;
+  const uint32_t na = std::min<uint32_t>(d.step_b, d.ext_a - a0);
+  const int64_t row_bytes = (int64_t)d.ext_b * es, panel = (int64_t)na * row_bytes;
+  // phase 1: the panel is one aligned range of the source, a whole number of 16-byte units
+  const int64_t S0 = sbase + (int64_t)a0 * d.sa[0];
+  if (d.sa[0] != row_bytes || S0 % 16 || panel % 16 || S0 < 0 || S0 + panel > in_bytes) return false;
+  // phase 2: every lane's stores and the elements it gathers
+  const uint32_t lanes = 1u << d.tile_ca;
+  for (uint32_t b = 0; b < d.ext_b; ++b) {
+    const uint32_t b_hi = host_fast_div(b, d.fd_b_in);
+    if (b_hi != b / d.fd_b_in.d) return false;
+    const int64_t off = d.fd_b_in.d < d.ext_b ? (int64_t)(b - b_hi * d.fd_b_in.d) * d.db[0] + (int64_t)b_hi * d.db[1]
+                                               : (int64_t)b * d.db[0];
+    for (uint32_t ca = 0; ca < lanes && ca * epu < na; ++ca) {
+      const int64_t g = dbase + (int64_t)a0 * es + (int64_t)ca * 16 + off;
+      if (g % 16 || g < 0 || g + 16 > out_bytes) return false;
+      const int64_t last = ((int64_t)ca * epu + epu - 1) * row_bytes + (int64_t)b * es;  // the lane's last element
       if (last + es > panel) return false;
     }
   }
@@ -575,10 +654,16 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
     if (ia_hi >= 0 && ib_hi >= 0 && try_build(-1, -1, ub)) return true;
     return false;
   };
-  // Order of preference, as measured on 2-byte elements (TB/s): 16-byte units on both sides 6.5; one side
-  // misaligned: the realigning kernel 4.0-4.5 for the source, 8-byte units 3.4-4.4 or the shifted-destination
-  // kernel 3.2-4.2 for the destination; 4-byte units 2.9.
+  // Order of preference, as measured on 2-byte elements (TB/s): 16-byte units on both sides 6.5; rows that follow
+  // each other on the misaligned side and are short enough for a panel: the flat kernels 4.4-5.3; otherwise the
+  // realigning kernel 4.0-5.0 for a misaligned source, 8-byte units 3.4-4.4 or the shifted-destination kernel
+  // 3.2-4.2 for a misaligned destination; 4-byte units 2.9.
   if (try_unit(16)) return true;
+  // source rows that follow each other in memory, destination rows aligned: the flat-source kernel (tr_unit = -3),
+  // whatever the alignment of the source rows
+  if ((es == 2 || es == 4) && ptr_align >= 16 && try_build(-1, ib_hi, es) &&
+      set_flat_source_panels(d))
+    return true;
   // source rows misaligned, destination rows aligned: the realigning kernel (tr_unit = -1; tile 8 x 14 chunks)
   if (es <= 4 && ptr_align >= 16 && try_build(ia_hi, ib_hi, es) && d->ext_a % (16 / es) == 0 && d->doff % 16 == 0 &&
       d->db[0] % 16 == 0 && d->db[1] % 16 == 0) {
@@ -721,6 +806,7 @@ static bool check_realign_block(const DevPiece &d, uint32_t blk, int64_t in_byte
 // the kernel's address arithmetic for one block, replayed on the host
 static bool check_transpose_block(const DevPiece &d, uint32_t blk, int64_t in_bytes, int64_t out_bytes) {
   if (d.tr_unit == -2) return check_flat_block(d, blk, flat_threads(flat_panel_bytes(d)), in_bytes, out_bytes);
+  if (d.tr_unit == -3) return check_flat_source_block(d, blk, flat_threads(flat_panel_bytes(d)), in_bytes, out_bytes);
   if (d.tr_unit == 0) return check_shifted_block(d, blk, in_bytes, out_bytes);
   if (d.tr_unit < 0) return check_realign_block(d, blk, in_bytes, out_bytes);
   const int es = d.unit_bytes, epu = 16 / es, ca = d.tile_ca, ta = ca * epu;
@@ -841,7 +927,7 @@ static bool append_piece(amap_plan_t *pl, Launch *L, DevPiece d) {
 static int plan_stage_transposes(PlanCtx &c, int stage) {
   const StageInfo &st = c.m.stages[stage];
   const size_t q_lo = st.first_piece, q_hi = q_lo + st.n_pieces;
-  for (int access : {16, 8, 4, 2, 0, -1, -2})
+  for (int access : {16, 8, 4, 2, 0, -1, -2, -3})
     for (int wide = 0; wide < 2; ++wide) {
       Launch L{kDevTranspose, c.es, access, wide, (int)c.pl->table.size(), 0, 0, stage};
       std::vector<DevPiece> transposes, fills;
@@ -879,7 +965,7 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
       for (const DevPiece &d : fills)
         if (!append_piece(c.pl, &L, d)) return plan_fail(AMAP_EUNSUPPORTED, q_lo);
       for (size_t q : taken) c.placed[q] = 1;
-      if (access == -2) {  // the block size and the shared memory of the largest panel serve the whole launch
+      if (access <= -2) {  // the block size and the shared memory of the largest panel serve the whole launch
         for (const DevPiece &d : transposes) L.smem = std::max(L.smem, flat_panel_bytes(d));
         L.threads = flat_threads(L.smem);
       }
@@ -1165,7 +1251,7 @@ extern "C" int amap_plan_launch_info(const amap_plan_t *plan, int32_t k, amap_la
   const Launch &L = plan->launches[k];
   memset(out, 0, sizeof *out);
   if (L.kind == kDevTranspose) {
-    out->kernel = L.cons == -2 ? AMAP_LAUNCH_TRANSPOSE_FLAT : L.cons == -1 ? AMAP_LAUNCH_TRANSPOSE_REALIGN
+    out->kernel = L.cons == -3 ? AMAP_LAUNCH_TRANSPOSE_FLAT_SOURCE : L.cons == -2 ? AMAP_LAUNCH_TRANSPOSE_FLAT : L.cons == -1 ? AMAP_LAUNCH_TRANSPOSE_REALIGN
                 : L.cons == 0 ? AMAP_LAUNCH_TRANSPOSE_SHIFTED : AMAP_LAUNCH_TRANSPOSE;
     out->access = L.cons > 0 ? L.cons : 16;
     out->threads = L.threads ? L.threads : kTransposeThreads;
@@ -1279,11 +1365,29 @@ static void launch_transpose_flat(const DescSource &ds, const Launch &L, const P
     else pick(std::integral_constant<int, 256>());
   }
 }
+template <int ES>
+static void launch_transpose_flat_source(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+  if constexpr (ES == 2 || ES == 4) {
+    auto go = [&](auto kernel, auto... args) {
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
+      launch_smem(kernel, L.n_blocks, L.threads, L.smem, s, pdl, args...);
+    };
+    auto pick = [&](auto threads) {
+      constexpr int T = decltype(threads)::value;
+      if (ds.ld && ds.ld->n_pieces == 1) go(amap_transpose_flat_source_one<ES, T>, ds.ld->piece[0], pt);
+      else if (ds.ld) go(amap_transpose_flat_source_param<ES, T>, *ds.ld, pt);
+      else go(amap_transpose_flat_source_table<ES, T>, ds.table, L.first_piece, L.n_pieces, pt);
+    };
+    if (L.threads == 512) pick(std::integral_constant<int, 512>());
+    else pick(std::integral_constant<int, 256>());
+  }
+}
 
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
     case -2: launch_transpose_flat<ES>(ds, L, pt, s, pdl); return;
+    case -3: launch_transpose_flat_source<ES>(ds, L, pt, s, pdl); return;
     case -1:
       if constexpr (ES <= 4)
         AMAP_LAUNCH(amap_transpose_realign_one, amap_transpose_realign_param, amap_transpose_realign_table, kTransposeThreads, ES);

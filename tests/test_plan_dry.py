@@ -84,8 +84,15 @@ def test_transpose_kernel_per_shape():
     assert launch_of(inv(N=2, C=24, H=5, W=13))["kernel"] == "transpose_shifted"
     L = launch_of(inv(N=2, C=68, H=14, W=14))
     assert (L["kernel"], L["access"]) == ("transpose", 8)
-    # the other direction: source rows misaligned, destination rows aligned
-    assert launch_of(W.c2_nchw_to_nhwc(N=4, C=256, H=27, W=27))["kernel"] == "transpose_realign"
+    # the other direction (source rows misaligned, destination rows aligned): panels that are contiguous in the
+    # source where the rows are short enough and there are enough panels, else the realigning kernel
+    fwd = W.c2_nchw_to_nhwc
+    L = launch_of(fwd(N=64, C=288, H=35, W=35))
+    assert (L["kernel"], L["threads"], L["smem_bytes"], L["n_blocks"]) == ("transpose_flat_source", 512, 78400, 64 * 9)
+    L = launch_of(fwd(N=64, C=1024, H=14, W=14))
+    assert (L["kernel"], L["threads"], L["smem_bytes"]) == ("transpose_flat_source", 256, 12544)
+    assert launch_of(fwd(N=4, C=256, H=27, W=27))["kernel"] == "transpose_realign"
+    assert launch_of(fwd(N=32, C=192, H=71, W=71))["kernel"] == "transpose_realign"
     # other families
     assert launch_of(W.full_configs()["c5"])["kernel"] == "strip"
     assert launch_of(W.full_configs()["c3"])["kernel"] in ("affine", "strip")
