@@ -973,19 +973,19 @@ __device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const Pt
   // rounds of equal length: ten loads are five and five, not eight and two
   const uint32_t per_thread = (ext_a + a_step - 1) / a_step, rounds = (per_thread + U - 1) / U;
   const int u_round = (int)((per_thread + rounds - 1) / rounds);
+  auto source_offset = [&](uint32_t a) -> int64_t {
+    if (merged) {
+      const uint32_t a_hi = fast_div(a, fa);
+      return (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1];
+    }
+    return (int64_t)a * sp.sa[0];
+  };
   for (uint32_t a0 = threadIdx.x >> lg; lane_on && a0 < ext_a; a0 += (uint32_t)u_round * a_step) {
     uint4 v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const uint32_t a = a0 + (uint32_t)u * a_step;
-      if (u < u_round && a < ext_a) {
-        int64_t off = (int64_t)a * sp.sa[0];
-        if (merged) {
-          const uint32_t a_hi = fast_div(a, fa);
-          off = (int64_t)(a - a_hi * fa.d) * sp.sa[0] + (int64_t)a_hi * sp.sa[1];
-        }
-        v[u] = load_16(src + off);
-      }
+      if (u < u_round && a < ext_a) v[u] = load_16(src + source_offset(a));
     }
     issue_barrier();
 #pragma unroll
@@ -1045,6 +1045,11 @@ __device__ __forceinline__ void transpose_flat_source_body(const DevPiece &sp, c
   const uint32_t ext_b = sp.ext_b, na = min(sp.step_b, sp.ext_a - a0);
   const uint32_t row_bytes = ext_b * ES;
   const char *src = ptrs.src[sp.input] + sbase + (int64_t)a0 * sp.sa[0];
+  // L2 hints (they read nothing into the SM): this block's panel while the kernel before this one drains, and,
+  // once this block's first loads are out, the panel of the block that will take its place (`prefetch` blocks on).
+  // A panel is one aligned range: one bulk prefetch from one thread.
+  if (sp.prefetch && threadIdx.x == 0)
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(na * row_bytes) : "memory");
   pdl_wait();
 
   const uint32_t n16 = na / EPU * ext_b;  // na is a multiple of EPU: the range is a whole number of 16-byte units
@@ -1053,6 +1058,23 @@ __device__ __forceinline__ void transpose_flat_source_body(const DevPiece &sp, c
 #pragma unroll
     for (int u = 0; u < U; ++u)
       if (i0 + u * THREADS < n16) v[u] = load_16(src + (size_t)(i0 + u * THREADS) * 16);
+    if (i0 == 0 && sp.prefetch > 1) {  // thread 0, first round
+      uint32_t t2 = blockIdx.x - sp.first_block + (uint32_t)sp.prefetch;
+      if (t2 < sp.n_blocks) {
+        uint32_t q2 = fast_div(t2, sp.fd_tiles_a);
+        const uint32_t na0 = (t2 - q2 * sp.tiles_a) * sp.step_b;
+        t2 = q2;
+        int64_t nbase = sp.soff + (int64_t)na0 * sp.sa[0];
+        for (int k = sp.n_loops - 1; k >= 0; --k) {
+          q2 = fast_div(t2, sp.fd[k]);
+          nbase += (int64_t)(t2 - q2 * sp.ext[k]) * sp.sstride[k];
+          t2 = q2;
+        }
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(ptrs.src[sp.input] + nbase),
+                     "r"(min(sp.step_b, sp.ext_a - na0) * row_bytes)
+                     : "memory");
+      }
+    }
     issue_barrier();
 #pragma unroll
     for (int u = 0; u < U; ++u)

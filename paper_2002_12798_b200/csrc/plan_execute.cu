@@ -472,6 +472,11 @@ static int flat_panel_bytes(const DevPiece &d) {
   return (int)((uint64_t)d.step_b * (d.tr_unit == -3 ? d.ext_b : d.ext_a) * d.unit_bytes);
 }
 static int flat_threads(int panel_bytes) { return panel_bytes > 24 * 1024 ? 512 : 256; }
+// blocks of a flat kernel resident per SM: eight of 256 threads or two of 512 (registers), as far as 227 KB of shared
+// memory hold their panels (1 KB per block is the system's)
+static int flat_blocks_per_sm(int panel_bytes) {
+  return std::max(1, std::min(flat_threads(panel_bytes) == 256 ? 8 : 2, 227 * 1024 / (panel_bytes + 1024)));
+}
 
 // the flat-destination kernel's address arithmetic for one block, replayed on the host
 static bool check_flat_block(const DevPiece &d, uint32_t blk, int threads, int64_t in_bytes, int64_t out_bytes) {
@@ -1167,6 +1172,10 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
     const int ahead = dist ? atoi(dist) : 8 * sms;
     for (DevPiece &d : pl->table)
       d.prefetch = (o.flags & AMAP_PLAN_NO_PREFETCH) ? 0 : (d.kind == kDevTranspose && ahead > 1) ? ahead : 1;
+    // the flat kernels: as many blocks ahead as are resident with their block size and panel
+    for (DevPiece &d : pl->table)
+      if (d.kind == kDevTranspose && d.tr_unit <= -2 && d.prefetch > 1 && !dist)
+        d.prefetch = sms * flat_blocks_per_sm(flat_panel_bytes(d));
     // plain copies (one loop of 16-byte units): the affine kernel looks one resident wave ahead too, up to 128 MB
     // (measured: 15.8 -> 15.1 us on 49 MB, 30.6 -> 30.2 us on 98 MB, but 154 -> 160 us on 512 MB)
     const uint64_t kCopyAheadMaxBytes = 128ull << 20;
