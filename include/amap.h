@@ -431,9 +431,19 @@ int amap_map_device_view(const amap_map *map, struct amap_device_view *out);
  *   view          host pointer (copied into the kernel's parameters)
  *   src_dev_ptrs  host array of the view's n_inputs DEVICE pointers (16-byte aligned)
  *   sums_dev      DEVICE pointer to rows uint32 values
- * Enqueues one kernel on cuda_stream of the current device and returns without synchronising or allocating. */
+ * Enqueues one kernel on cuda_stream of the current device and returns without synchronising or allocating.
+ * Where every row is a whole number of contiguous source runs of one piece (rows of an im2col matrix, of a head
+ * split, of a plain copy) the kernel decodes the loops outside a row once per row and takes the runs inside it from
+ * a table (amap_device.h: amap_view_rows); otherwise it asks amap_view_locate per 16 bytes. */
 int amap_consume_row_sums(const struct amap_device_view *view, const void *const *src_dev_ptrs, int64_t rows,
                           int64_t cols, uint32_t *sums_dev, void *cuda_stream);
+
+/* The row tables of amap_device.h (amap_view_rows_build, amap_view_row_seek, amap_view_row_run) walked on the HOST:
+ * writes the chain's result, seen as rows of `cols` elements, to dst_host from HOST copies of the inputs.  For
+ * tests of the tables a consumer kernel relies on.  AMAP_EUNSUPPORTED when the rows of the view are not whole runs
+ * of one piece each (a consumer then falls back to amap_view_locate); elem_size up to 8. */
+int amap_view_rows_gather_host(const struct amap_device_view *view, int64_t cols, const void *const *src_host_ptrs,
+                               void *dst_host);
 
 const char *amap_strerror(int code);
 /* text of the last CUDA error seen by this thread in this library ("" if none) */

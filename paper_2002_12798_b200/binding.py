@@ -30,7 +30,7 @@ EXPORTS = [
     "amap_builder_window", "amap_builder_window_ex", "amap_builder_tile", "amap_builder_repeat", "amap_builder_split", "amap_builder_tensor",
     "amap_builder_stmt",
     "amap_builder_opaque", "amap_builder_chain", "amap_compose", "amap_compose_ex", "amap_compose_multi",
-    "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_device_view", "amap_consume_row_sums", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
+    "amap_map_num_outputs", "amap_map_output_numel", "amap_execute_multi", "amap_map_device_view", "amap_consume_row_sums", "amap_view_rows_gather_host", "amap_map_num_stages", "amap_map_get_stage", "amap_map_destroy", "amap_map_num_pieces", "amap_map_get_piece",
     "amap_map_sizes", "amap_plan", "amap_plan_destroy", "amap_plan_stats", "amap_plan_piece_kernel", "amap_plan_launch_info",
     "amap_execute", "amap_execute_host", "amap_execute_static", "amap_strerror", "amap_last_cuda_error",
 ]
@@ -351,6 +351,18 @@ class Map:
         v = DeviceView()
         _check(_lib.amap_map_device_view(self._h, byref(v)), "amap_map_device_view")
         return v
+
+    def rows_gather_host(self, inputs, cols):
+        """amap_view_rows_gather_host: the result as rows of `cols` elements, gathered on the host through the row
+        tables of the device view (numpy inputs; returns a flat numpy array of the inputs' dtype)."""
+        import numpy as np
+
+        v = self.device_view()
+        xs = [np.ascontiguousarray(x) for x in inputs]
+        arr = (c_void_p * max(len(xs), 1))(*[c_void_p(x.ctypes.data) for x in xs])
+        out = np.empty(self.out_numel, dtype=xs[0].dtype)
+        _check(_lib.amap_view_rows_gather_host(byref(v), c_int64(cols), arr, c_void_p(out.ctypes.data)), "amap_view_rows_gather_host")
+        return out
 
     def consume_row_sums(self, srcs, rows, cols, sums, stream=None):
         """amap_consume_row_sums: uint32 sums of the rows of the chain's result, read through the map from the

@@ -531,6 +531,42 @@ def test_device_view_reproduces_the_chain(name):
     assert np.array_equal(eval_view(v, xs), want.reshape(-1))
 
 
+@pytest.mark.parametrize("name,cols,whole_runs", [
+    ("c5", 9 * 128, True), ("c5", 3 * 128, True), ("c5", 128, True), ("c5_odd", 9 * 24, True), ("c5_dil2", None, True),
+    ("c3", 128, True), ("c3", 2 * 128, True), ("c3_odd", 24, True), ("c3_odd", 17 * 24, True),
+    ("c5_crs", None, False),  # columns ordered (c, r, s): the innermost loop strides the source
+    ("c2_inv", 11, False), ("c1", 16, False),  # strided sources
+    ("c4", 320, None), ("c4_odd", 88, None), ("c2_inv", 13 * 11, None), ("c1", 48, None),
+])
+def test_row_tables_reproduce_the_chain(name, cols, whole_runs):
+    """The consumer's row walk (outer loops decoded once per row, the runs inside a row from a table) on the host:
+    rows of one run, of several runs with guards (window gathers), rows that cut a loop in two, rows that span a
+    whole inner nest.  `whole_runs`: whether the rows are known to be whole runs (None: either answer is fine, the
+    result must be right if there is one)."""
+    chain = W.reduced_configs()[name]
+    xs = W.make_inputs(chain)
+    want = oracle.run_chain(chain, xs)
+    m = B.compose_chain(chain)
+    cols = cols or want.shape[-1]
+    try:
+        got = m.rows_gather_host(xs, cols)
+    except B.AmapError as e:
+        assert e.code == -9 and not whole_runs, e  # the functor's job
+        return
+    assert whole_runs is not False
+    assert np.array_equal(got.view(np.uint8), np.ascontiguousarray(want).reshape(-1).view(np.uint8))
+
+
+def test_row_tables_of_a_plain_copy_split_its_one_loop():
+    b = B.Builder(2)
+    m = b.compose(b.reshape(b.input([6, 40]), [240]))
+    x = np.arange(240, dtype=np.uint16)
+    for cols in (240, 40, 8, 1):
+        assert np.array_equal(m.rows_gather_host([x], cols), x)
+    with pytest.raises(B.AmapError):
+        m.rows_gather_host([x], 7)  # does not divide the result
+
+
 def test_device_view_refuses_what_it_cannot_hold():
     b = B.Builder(2)
     ids = [b.input([4, 8]) for _ in range(5)]
