@@ -586,7 +586,8 @@ static bool split_a_remainder(const DevPiece &d, DevPiece *whole, DevPiece *rest
   return set_transpose_tiles(whole, 8, true) && set_transpose_tiles(rest, 4, true);
 }
 
-static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t in_bytes, DevPiece *d) {
+static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t in_bytes, DevPiece *d,
+                                  bool allow_flat = true) {
   if (es > 8 || p.src == AMAP_CONST || p.qa.on || !p.guards.empty() || !p.domain.empty()) return false;
   const int n = p.n();
   if (n < 2) return false;
@@ -666,7 +667,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
   if (try_unit(16)) return true;
   // source rows that follow each other in memory, destination rows aligned: the flat-source kernel (tr_unit = -3),
   // whatever the alignment of the source rows
-  if ((es == 2 || es == 4) && ptr_align >= 16 && try_build(-1, ib_hi, es) &&
+  if (allow_flat && (es == 2 || es == 4) && ptr_align >= 16 && try_build(-1, ib_hi, es) &&
       set_flat_source_panels(d))
     return true;
   // source rows misaligned, destination rows aligned: the realigning kernel (tr_unit = -1; tile 8 x 14 chunks)
@@ -693,7 +694,7 @@ static bool build_transpose_piece(const Piece &p, int es, int ptr_align, int64_t
   }
   // destination rows that follow each other in memory, source rows aligned: the flat-destination kernel
   // (tr_unit = -2), whatever the alignment of the destination rows
-  if ((es == 2 || es == 4) && ptr_align >= 16 && try_build(ia_hi, -1, es) &&
+  if (allow_flat && (es == 2 || es == 4) && ptr_align >= 16 && try_build(ia_hi, -1, es) &&
       set_flat_panels(d))
     return true;
   if (try_unit(8)) return true;
@@ -1021,6 +1022,8 @@ static int plan_stage_strips(PlanCtx &c, int stage) {
 // outside the slab).
 // ---------------------------------------------------------------------------
 static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts, bool allow_slabs, amap_plan_t **out_plan);
+static cudaError_t allow_flat_panels();
+static bool has_flat_launches(const amap_plan_t *plan);
 
 static void plan_slabs(const Map &m, int device, const amap_plan_opts &o, amap_plan_t *pl) {
   if (m.stages.size() != 1 || m.pieces.empty() || m.out_numel == 0 || m.out_numels.size() > 1) return;
@@ -1145,6 +1148,27 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
     pl->piece_kernel.push_back(kind);
   }
   for (size_t q = 0; q < reads.size(); ++q) pl->stats.bytes_read += std::min(reads[q], slot_numel[q]) * es;
+  // A stage whose transposes would split between a flat kernel and the tiled kernel for the same misaligned side
+  // (operands of a concat with enough channels for a panel and others with too few) runs them all on the tiled
+  // kernel: one launch instead of two.
+  for (const StageInfo &st : m.stages) {
+    bool flat_src = false, realign = false, flat_dst = false, other_dst = false;
+    for (size_t q = st.first_piece; q < (size_t)(st.first_piece + st.n_pieces); ++q) {
+      if (!is_tr[q]) continue;
+      flat_src = flat_src || tr[q].tr_unit == -3;
+      realign = realign || tr[q].tr_unit == -1;
+      flat_dst = flat_dst || tr[q].tr_unit == -2;
+      other_dst = other_dst || tr[q].tr_unit == 0 || (tr[q].tr_unit > 0 && tr[q].tr_unit < 16);
+    }
+    for (size_t q = st.first_piece; q < (size_t)(st.first_piece + st.n_pieces); ++q) {
+      if (!is_tr[q]) continue;
+      if ((tr[q].tr_unit == -3 && realign) || (tr[q].tr_unit == -2 && other_dst)) {
+        DevPiece d;
+        const Piece &p = m.pieces[q];
+        if (build_transpose_piece(p, es, align, slot_numel[p.src] * es, &d, false)) tr[q] = d;
+      }
+    }
+  }
 
   PlanCtx ctx{m, o, es, slot_numel, unit_of, tr, is_tr, std::vector<char>(m.pieces.size(), 0), pl};
   for (int stage = 0; stage < (int)m.stages.size(); ++stage) {
@@ -1208,6 +1232,7 @@ static int plan_impl(const amap_map *map, int device, const amap_plan_opts *opts
     if (e == cudaSuccess)
       e = cudaMemcpy(pl->dev_table, pl->table.data(), pl->table.size() * sizeof(DevPiece), cudaMemcpyHostToDevice);
   }
+  if (e == cudaSuccess && has_flat_launches(pl)) e = allow_flat_panels();
   pl->temps.assign(pl->temp_numel.size(), nullptr);
   for (size_t k = 0; k < pl->temps.size() && e == cudaSuccess; ++k)
     if (pl->temp_numel[k] > 0) e = cudaMalloc(&pl->temps[k], (size_t)pl->temp_numel[k] * es);
@@ -1355,37 +1380,52 @@ static void launch_transpose_narrow(const DescSource &ds, const Launch &L, const
   }
 }
 
-// The flat-destination kernel: dynamic shared memory above the default limit has to be allowed per function (a
-// function attribute of the current device's context; setting it again costs a host call and nothing else).
-template <int ES>
-static void launch_transpose_flat(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
-  if constexpr (ES == 2 || ES == 4) {
-    auto go = [&](auto kernel, auto... args) {
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
-      launch_smem(kernel, L.n_blocks, L.threads, L.smem, s, pdl, args...);
-    };
-    auto pick = [&](auto threads) {
-      constexpr int T = decltype(threads)::value;
-      if (ds.ld && ds.ld->n_pieces == 1) go(amap_transpose_flat_one<ES, T>, ds.ld->piece[0], pt);
-      else if (ds.ld) go(amap_transpose_flat_param<ES, T>, *ds.ld, pt);
-      else go(amap_transpose_flat_table<ES, T>, ds.table, L.first_piece, L.n_pieces, pt);
-    };
-    if (L.threads == 512) pick(std::integral_constant<int, 512>());
-    else pick(std::integral_constant<int, 256>());
-  }
+// The flat kernels: dynamic shared memory above the default limit has to be allowed per function (an attribute of
+// the function in the current device's context).  Done when a plan with such launches is made for a device and on
+// the first amap_execute_static on a device, never while launches are enqueued.
+template <int ES, int T>
+static cudaError_t allow_flat_panels_for() {
+  cudaError_t e = cudaSuccess;
+  auto allow = [&](auto kernel) {
+    const cudaError_t r = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
+    if (e == cudaSuccess) e = r;
+  };
+  allow(amap_transpose_flat_one<ES, T>);
+  allow(amap_transpose_flat_param<ES, T>);
+  allow(amap_transpose_flat_table<ES, T>);
+  allow(amap_transpose_flat_source_one<ES, T>);
+  allow(amap_transpose_flat_source_param<ES, T>);
+  allow(amap_transpose_flat_source_table<ES, T>);
+  return e;
 }
+static cudaError_t allow_flat_panels() {
+  cudaError_t e = allow_flat_panels_for<2, 256>();
+  if (e == cudaSuccess) e = allow_flat_panels_for<2, 512>();
+  if (e == cudaSuccess) e = allow_flat_panels_for<4, 256>();
+  if (e == cudaSuccess) e = allow_flat_panels_for<4, 512>();
+  return e;
+}
+static bool has_flat_launches(const amap_plan_t *plan) {
+  for (const Launch &L : plan->launches)
+    if (L.kind == kDevTranspose && L.cons <= -2) return true;
+  return false;
+}
+
 template <int ES>
-static void launch_transpose_flat_source(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
+static void launch_transpose_flat(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl,
+                                  bool source_side) {
   if constexpr (ES == 2 || ES == 4) {
-    auto go = [&](auto kernel, auto... args) {
-      cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
-      launch_smem(kernel, L.n_blocks, L.threads, L.smem, s, pdl, args...);
-    };
     auto pick = [&](auto threads) {
       constexpr int T = decltype(threads)::value;
-      if (ds.ld && ds.ld->n_pieces == 1) go(amap_transpose_flat_source_one<ES, T>, ds.ld->piece[0], pt);
-      else if (ds.ld) go(amap_transpose_flat_source_param<ES, T>, *ds.ld, pt);
-      else go(amap_transpose_flat_source_table<ES, T>, ds.table, L.first_piece, L.n_pieces, pt);
+      if (source_side) {
+        if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_source_one<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
+        else if (ds.ld) launch_smem(amap_transpose_flat_source_param<ES, T>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
+        else launch_smem(amap_transpose_flat_source_table<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
+      } else {
+        if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_one<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
+        else if (ds.ld) launch_smem(amap_transpose_flat_param<ES, T>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
+        else launch_smem(amap_transpose_flat_table<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
+      }
     };
     if (L.threads == 512) pick(std::integral_constant<int, 512>());
     else pick(std::integral_constant<int, 256>());
@@ -1395,8 +1435,8 @@ static void launch_transpose_flat_source(const DescSource &ds, const Launch &L, 
 template <int ES>
 static void launch_transpose(const DescSource &ds, const Launch &L, const PtrTable &pt, cudaStream_t s, bool pdl) {
   switch (L.cons) {  // access width of the launch
-    case -2: launch_transpose_flat<ES>(ds, L, pt, s, pdl); return;
-    case -3: launch_transpose_flat_source<ES>(ds, L, pt, s, pdl); return;
+    case -2: launch_transpose_flat<ES>(ds, L, pt, s, pdl, false); return;
+    case -3: launch_transpose_flat<ES>(ds, L, pt, s, pdl, true); return;
     case -1:
       if constexpr (ES <= 4)
         AMAP_LAUNCH(amap_transpose_realign_one, amap_transpose_realign_param, amap_transpose_realign_table, kTransposeThreads, ES);
@@ -1634,6 +1674,7 @@ static int static_table_address(int device, void **out) {
 
 // multiprocessors of the current device, looked up once per device (the look-ahead distance of a dry plan is
 // set for the device the call runs on)
+static char g_static_flat_allowed[kStaticMaxDevices];  // the flat kernels' shared-memory attribute is set on the device
 static int g_static_sms[kStaticMaxDevices];
 static int static_device_sms(int device) {
   int n = __atomic_load_n(&g_static_sms[device], __ATOMIC_ACQUIRE);
@@ -1666,6 +1707,10 @@ extern "C" int amap_execute_static(const amap_plan_t *plan, const void *const *s
   // knowing the device: its look-ahead distances assume kDefaultSms multiprocessors and are rescaled here.
   const int sms = static_device_sms(device);
   const bool rescale = plan->device < 0 && sms != kDefaultSms;
+  if (has_flat_launches(plan) && device < kStaticMaxDevices && !g_static_flat_allowed[device]) {
+    CUDA_TRY(allow_flat_panels());
+    g_static_flat_allowed[device] = 1;
+  }
   for (size_t first = 0; first < plan->table.size(); first += kParamPieces) {
     LaunchDesc ld;
     memset(&ld, 0, sizeof ld);

@@ -556,11 +556,15 @@ def test_overlapping_buffers_are_refused(B):
     assert e.value.code == -1
 
 
-def test_execute_can_be_captured_in_a_cuda_graph(B):
+@pytest.mark.parametrize("chain", [
+    W.reduced_configs()["c2_fwd_mid"],
+    W.c2_nhwc_to_nchw(N=40, C=128, H=35, W=35),  # flat-destination transpose, panels of 78400 bytes of shared memory
+    W.c2_nchw_to_nhwc(N=40, C=128, H=35, W=35),  # flat-source transpose
+], ids=["aligned", "flat_destination", "flat_source"])
+def test_execute_can_be_captured_in_a_cuda_graph(B, chain):
     """amap_execute neither synchronises nor allocates, so a stream capture can record it; replays must copy."""
     import torch
 
-    chain = W.reduced_configs()["c2_fwd_mid"]
     (x,) = W.make_inputs(chain)
     want = oracle.run_chain(chain, [x]).reshape(-1)
     m = B.compose_chain(chain)

@@ -93,6 +93,10 @@ def test_transpose_kernel_per_shape():
     assert (L["kernel"], L["threads"], L["smem_bytes"]) == ("transpose_flat_source", 256, 12544)
     assert launch_of(fwd(N=4, C=256, H=27, W=27))["kernel"] == "transpose_realign"
     assert launch_of(fwd(N=32, C=192, H=71, W=71))["kernel"] == "transpose_realign"
+    # operands of one concat with enough channels for a panel (40) and with too few (8, 24, 16): all of them on the
+    # tiled kernel, so that the transposes stay one launch (plus the launch of the padding borders)
+    mixed = B.compose_chain(W.reduced_configs()["c4_odd"]).plan(device=-1).launches()
+    assert [l["kernel"] for l in mixed] == ["transpose_realign", "strip"]
     # other families
     assert launch_of(W.full_configs()["c5"])["kernel"] == "strip"
     assert launch_of(W.full_configs()["c3"])["kernel"] in ("affine", "strip")

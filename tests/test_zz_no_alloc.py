@@ -40,9 +40,13 @@ def test_static_table_matches_amap_execute_on_calls_in_a_row():
 
     cfg = W.reduced_configs()
     # different maps one after the other: each call finds the previous call's descriptors in the table
-    # every kernel family reads its descriptors from the fixed table here: copy, aligned / narrow / realigning /
-    # shifted transposes with fills, window gather, element-wise gather
-    for name in ("c3", "c4", "c2_fwd_narrow", "c2_fwd", "c2_inv", "c4_odd", "c5", "c1", "c3"):
+    # every kernel family reads its descriptors from the fixed table here: copy, aligned / narrow / flat
+    # transposes (small panels and panels beyond the default shared-memory limit) with fills, window gather,
+    # element-wise gather
+    cfg["flat_destination_large_panels"] = W.c2_nhwc_to_nchw(N=40, C=128, H=35, W=35)  # 78400 bytes of shared memory
+    cfg["flat_source_large_panels"] = W.c2_nchw_to_nhwc(N=40, C=128, H=35, W=35)
+    for name in ("c3", "c4", "c2_fwd_narrow", "c2_fwd", "c2_inv", "flat_destination_large_panels", "c4_odd",
+                 "flat_source_large_panels", "c5", "c1", "c3"):
         ref, out, dry, dev, stream = _both_ways(B, torch, cfg[name])
         ptrs = [d.data_ptr() for d in dev]
         assert torch.equal(ref, out), name  # pure copies: bit-exact
