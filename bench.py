@@ -48,10 +48,10 @@ SIGNED = {1: np.int8, 2: np.int16, 4: np.int32, 8: np.int64}
 # previous launch leaves them).  Valid only for the kernel source it was taken on: the digest below is that of the
 # kernel sources at capture time, and the line reports traffic = null when they have changed since.
 STEADY_STATE_TRAFFIC = {
-    "bytes_per_launch": 101_530_960,
-    "kernel_digest": "56814d7913a635ed",
+    "bytes_per_launch": 101_910_368,
+    "kernel_digest": "9f27bc68d90fa531",
     "note": "ncu counters over 16 consecutive launches of the timed loop, caches as the previous launch leaves them: "
-            "51.41 MB read + 50.12 MB written per launch, 0.988 of the algorithmic bytes",
+            "51.55 MB read + 50.36 MB written per launch, 0.992 of the algorithmic bytes",
 }
 KERNEL_SOURCES = ("kernels.cuh", "device_table.hpp", "plan_execute.cu")
 
@@ -235,7 +235,8 @@ def rate_fields(row, peak):
 # ---------------------------------------------------------------------------
 # the configurations beside the headline workload
 # ---------------------------------------------------------------------------
-TABLE_CONFIGS = ("c2_fwd", "c2_inv", "c3", "c3_merge", "c4", "c5", "odd35_fwd", "odd35_inv", "map14_inv")
+TABLE_CONFIGS = ("c2_fwd", "c2_inv", "c3", "c3_merge", "c4", "c5", "odd35_fwd", "odd35_inv", "map14_inv", "map7_inv",
+                 "map71_fwd", "map71_inv", "map14_c1020_inv")
 
 
 def bench_configs():
@@ -245,11 +246,17 @@ def bench_configs():
     # operators beyond the five configurations: nearest-neighbour upsampling (repeat on H and W: every input byte
     # is read once and written four times) and a fused QKV tensor cut in three, each part to [B, heads, S, D]
     configs["upsample2x"] = W.upsample_nhwc()
-    # layout changes whose rows are not 16-byte aligned on one side (Inception's 35x35x288 maps, ResNet's 14x14x1024):
-    # the realigning, shifted-destination and narrow-unit transpose kernels
+    # layout changes whose rows are not 16-byte aligned on one side.  Rows short enough for a panel (Inception's
+    # 35x35x288 maps, ResNet's 14x14x1024 and 7x7x2048): the flat-source and flat-destination transposes
     configs["odd35_fwd"] = W.c2_nchw_to_nhwc(N=64, C=288, H=35, W=35)
     configs["odd35_inv"] = W.c2_nhwc_to_nchw(N=64, C=288, H=35, W=35)
     configs["map14_inv"] = W.c2_nhwc_to_nchw(N=64, C=1024, H=14, W=14)
+    configs["map7_inv"] = W.c2_nhwc_to_nchw(N=128, C=2048, H=7, W=7)
+    # longer rows (71x71x192 maps): the realigning and shifted-destination kernels; a channel count that is no
+    # multiple of 16 bytes (14x14x1020): 8-byte units
+    configs["map71_fwd"] = W.c2_nchw_to_nhwc(N=32, C=192, H=71, W=71)
+    configs["map71_inv"] = W.c2_nhwc_to_nchw(N=32, C=192, H=71, W=71)
+    configs["map14_c1020_inv"] = W.c2_nhwc_to_nchw(N=64, C=1020, H=14, W=14)
     configs["qkv_split"] = [W.qkv_split(part=k) for k in range(3)]   # three maps, three launches
     configs["qkv_split_one_launch"] = W.qkv_split_all()               # one map with three outputs, one launch
     return configs
@@ -269,9 +276,9 @@ def torch_view_chain(torch, name, chain):
     """The same result with torch's own operators, views kept as views (reshape / slice / permute cost nothing until
     a copy is forced): the strong library baseline on the same GPU.  Returns fn(list of typed tensors) -> tensor."""
     F = torch.nn.functional
-    if name in ("c2_fwd", "odd35_fwd"):
+    if name in ("c2_fwd", "odd35_fwd", "map71_fwd"):
         return lambda xs: xs[0].permute(0, 2, 3, 1).contiguous()
-    if name in ("c2_inv", "odd35_inv", "map14_inv"):
+    if name in ("c2_inv", "odd35_inv", "map14_inv", "map7_inv", "map71_inv", "map14_c1020_inv"):
         return lambda xs: xs[0].permute(0, 3, 1, 2).contiguous()
     if name == "c3":
         B_, S, HD = chain.inputs[0]
@@ -790,6 +797,17 @@ def run_one_config(args):
             launches = 2
 
         case = _C()
+    elif args.config in ("consumer_c5", "consumer_c3"):
+        # the row-sum consumer reading through the map (nothing is copied)
+        name = args.config.split("_")[1]
+        case = Case(torch, B, bench_configs()[name], device, stream, l2, args.plan_flags)
+        m, n_sets = case.maps[0], case.n_sets
+        cols = {"c5": 9 * 128, "c3": 128}[name]
+        rows = m.out_numel // cols
+        sums = [torch.empty(rows, dtype=torch.int32, device=device) for _ in range(n_sets)]
+        calls = [m.bind_consume_row_sums(case.ins[i], rows, cols, sums[i], stream) for i in range(n_sets)]
+        total = case.stats[0]["bytes_read"] + 4 * rows
+        case.launches = 1
     else:
         case = Case(torch, B, bench_configs()[args.config], device, stream, l2, args.plan_flags)
         calls, n_sets, total = case.calls, case.n_sets, case.total
