@@ -937,7 +937,7 @@ __device__ __forceinline__ void transpose_shifted_body(const DevPiece &sp, const
 // The lanes that share one a are the first 2^tile_ca of a group (tile_ca holds
 // the logarithm here).
 // ---------------------------------------------------------------------------
-template <int ES, int THREADS>
+template <int ES, int THREADS, bool PAIRED>
 __device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const PtrTable &ptrs) {
   constexpr int EPU = 16 / ES;
   // loads a thread keeps in flight: four in 32 registers where eight blocks of 256 threads share an SM; eight where
@@ -980,7 +980,42 @@ __device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const Pt
     }
     return (int64_t)a * sp.sa[0];
   };
-  for (uint32_t a0 = threadIdx.x >> lg; lane_on && a0 < ext_a; a0 += (uint32_t)u_round * a_step) {
+  // 2-byte elements, rows an even number of elements long (so that every row of the image starts on a 4-byte
+  // boundary): a thread takes PAIRS of neighbouring a and stores 32-bit words, half the shared-memory stores
+  // (PAIRED: the launch's pieces all qualify; a kernel of its own, so that neither form carries the other's registers)
+  if constexpr (PAIRED) {
+    constexpr int UP = U / 2;
+    const uint32_t n_pairs = ext_a >> 1;
+    const uint32_t pairs_per_thread = (n_pairs + a_step - 1) / a_step, pair_rounds = (pairs_per_thread + UP - 1) / UP;
+    const int up_round = (int)((pairs_per_thread + pair_rounds - 1) / pair_rounds);
+    for (uint32_t q0 = threadIdx.x >> lg; lane_on && q0 < n_pairs; q0 += (uint32_t)up_round * a_step) {
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < UP; ++u) {
+        const uint32_t pr = q0 + (uint32_t)u * a_step;
+        if (u < up_round && pr < n_pairs) {
+          v[2 * u] = load_16(src + source_offset(2 * pr));
+          v[2 * u + 1] = load_16(src + source_offset(2 * pr + 1));
+        }
+      }
+      issue_barrier();
+#pragma unroll
+      for (int u = 0; u < UP; ++u) {
+        const uint32_t pr = q0 + (uint32_t)u * a_step;
+        if (u < up_round && pr < n_pairs) {
+          unsigned char *p = column + pr * 4;
+          const uint32_t w0[4] = {v[2 * u].x, v[2 * u].y, v[2 * u].z, v[2 * u].w};
+          const uint32_t w1[4] = {v[2 * u + 1].x, v[2 * u + 1].y, v[2 * u + 1].z, v[2 * u + 1].w};
+#pragma unroll
+          for (int e = 0; e < EPU; ++e) {
+            *reinterpret_cast<uint32_t *>(p) = __byte_perm(w0[e >> 1], w1[e >> 1], (e & 1) ? 0x7632 : 0x5410);
+            p += row_bytes;
+          }
+        }
+      }
+    }
+  }
+  for (uint32_t a0 = threadIdx.x >> lg; !PAIRED && lane_on && a0 < ext_a; a0 += (uint32_t)u_round * a_step) {
     uint4 v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -1089,6 +1124,34 @@ __device__ __forceinline__ void transpose_flat_source_body(const DevPiece &sp, c
   const bool merged = fb.d < ext_b;
   char *dst = ptrs.dst(sp.out) + dbase + (int64_t)a0 * ES + (int64_t)ca * 16;
   const unsigned char *column = panel + ca * EPU * row_bytes;  // this lane's first row of the image
+  auto dest_offset = [&](uint32_t b) -> int64_t {
+    if (merged) {
+      const uint32_t b_hi = fast_div(b, fb);
+      return (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1];
+    }
+    return (int64_t)b * sp.db[0];
+  };
+  // 2-byte elements, rows an even number of elements long: a thread takes PAIRS of neighbouring b, reads 32-bit
+  // words (one per a, both b) and stores two vectors: half the shared-memory loads
+  bool paired = false;
+  if constexpr (ES == 2) paired = (ext_b & 1u) == 0;
+  if (paired) {
+#pragma unroll 2
+    for (uint32_t pr = threadIdx.x >> lg; lane_on && pr < (ext_b >> 1); pr += b_step) {
+      const unsigned char *p = column + pr * 4;
+      uint32_t r[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) r[e] = *reinterpret_cast<const uint32_t *>(p + e * row_bytes);
+      uint4 lo, hi;
+      lo.x = __byte_perm(r[0], r[1], 0x5410); hi.x = __byte_perm(r[0], r[1], 0x7632);
+      lo.y = __byte_perm(r[2], r[3], 0x5410); hi.y = __byte_perm(r[2], r[3], 0x7632);
+      lo.z = __byte_perm(r[4], r[5], 0x5410); hi.z = __byte_perm(r[4], r[5], 0x7632);
+      lo.w = __byte_perm(r[6], r[7], 0x5410); hi.w = __byte_perm(r[6], r[7], 0x7632);
+      __stcs(reinterpret_cast<uint4 *>(dst + dest_offset(2 * pr)), lo);
+      __stcs(reinterpret_cast<uint4 *>(dst + dest_offset(2 * pr + 1)), hi);
+    }
+    return;
+  }
 #pragma unroll 2
   for (uint32_t b = threadIdx.x >> lg; lane_on && b < ext_b; b += b_step) {
     const unsigned char *p = column + b * ES;
@@ -1104,12 +1167,7 @@ __device__ __forceinline__ void transpose_flat_source_body(const DevPiece &sp, c
         w[e] = lo | (hi << 16);
       }
     }
-    int64_t off = (int64_t)b * sp.db[0];
-    if (merged) {
-      const uint32_t b_hi = fast_div(b, fb);
-      off = (int64_t)(b - b_hi * fb.d) * sp.db[0] + (int64_t)b_hi * sp.db[1];
-    }
-    __stcs(reinterpret_cast<uint4 *>(dst + off), make_uint4(w[0], w[1], w[2], w[3]));
+    __stcs(reinterpret_cast<uint4 *>(dst + dest_offset(b)), make_uint4(w[0], w[1], w[2], w[3]));
   }
 }
 
@@ -1410,26 +1468,26 @@ __global__ void __launch_bounds__(kTransposeThreads) amap_transpose_realign_one(
 
 // The flat-destination transpose runs with the dynamic shared memory its launch asks for: small panels with eight
 // blocks of 256 threads per SM (32 registers per thread), large ones with blocks of 512 threads (64 registers).
-template <int ES, int THREADS>
+template <int ES, int THREADS, bool PAIRED>
 __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_param(const __grid_constant__ LaunchDesc ld,
                                                                                     PtrTable ptrs) {
   pdl_launch_dependents();
-  transpose_flat_body<ES, THREADS>(param_piece(ld), ptrs);
+  transpose_flat_body<ES, THREADS, PAIRED>(param_piece(ld), ptrs);
 }
-template <int ES, int THREADS>
+template <int ES, int THREADS, bool PAIRED>
 __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_table(const DevPiece *__restrict__ table,
                                                                                     int first_piece, int n_pieces,
                                                                                     PtrTable ptrs) {
   __shared__ DevPiece sp;
   pdl_launch_dependents();
   fetch_piece(table, first_piece, n_pieces, &sp);
-  transpose_flat_body<ES, THREADS>(sp, ptrs);
+  transpose_flat_body<ES, THREADS, PAIRED>(sp, ptrs);
 }
-template <int ES, int THREADS>
+template <int ES, int THREADS, bool PAIRED>
 __global__ void __launch_bounds__(THREADS, THREADS == 256 ? 8 : 2) amap_transpose_flat_one(const __grid_constant__ DevPiece p,
                                                                                   PtrTable ptrs) {
   pdl_launch_dependents();
-  transpose_flat_body<ES, THREADS>(p, ptrs);
+  transpose_flat_body<ES, THREADS, PAIRED>(p, ptrs);
 }
 
 template <int ES, int THREADS>

@@ -43,8 +43,9 @@ struct Launch {
   int n_pieces;
   uint32_t n_blocks;
   int stage;  // which stage of the map this launch belongs to
-  int threads = 0;  // flat-destination transpose only: block size and dynamic shared memory of the launch
+  int threads = 0;  // flat transposes only: block size and dynamic shared memory of the launch
   int smem = 0;
+  int paired = 0;   // flat-destination transpose of 2-byte elements: every piece's rows are an even number of elements long
 };
 
 struct amap_plan_t {
@@ -974,6 +975,9 @@ static int plan_stage_transposes(PlanCtx &c, int stage) {
       if (access <= -2) {  // the block size and the shared memory of the largest panel serve the whole launch
         for (const DevPiece &d : transposes) L.smem = std::max(L.smem, flat_panel_bytes(d));
         L.threads = flat_threads(L.smem);
+        L.paired = (access == -2 && c.es == 2) ? 1 : 0;
+        for (const DevPiece &d : transposes)
+          if (d.ext_a & 1u) L.paired = 0;
       }
       c.pl->launches.push_back(L);
     }
@@ -1390,9 +1394,14 @@ static cudaError_t allow_flat_panels_for() {
     const cudaError_t r = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFlatMaxPanelBytes);
     if (e == cudaSuccess) e = r;
   };
-  allow(amap_transpose_flat_one<ES, T>);
-  allow(amap_transpose_flat_param<ES, T>);
-  allow(amap_transpose_flat_table<ES, T>);
+  allow(amap_transpose_flat_one<ES, T, false>);
+  allow(amap_transpose_flat_param<ES, T, false>);
+  allow(amap_transpose_flat_table<ES, T, false>);
+  if constexpr (ES == 2) {
+    allow(amap_transpose_flat_one<ES, T, true>);
+    allow(amap_transpose_flat_param<ES, T, true>);
+    allow(amap_transpose_flat_table<ES, T, true>);
+  }
   allow(amap_transpose_flat_source_one<ES, T>);
   allow(amap_transpose_flat_source_param<ES, T>);
   allow(amap_transpose_flat_source_table<ES, T>);
@@ -1421,10 +1430,15 @@ static void launch_transpose_flat(const DescSource &ds, const Launch &L, const P
         if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_source_one<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
         else if (ds.ld) launch_smem(amap_transpose_flat_source_param<ES, T>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
         else launch_smem(amap_transpose_flat_source_table<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
+      } else if (ES == 2 && L.paired) {
+        constexpr bool P = ES == 2;
+        if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_one<ES, T, P>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
+        else if (ds.ld) launch_smem(amap_transpose_flat_param<ES, T, P>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
+        else launch_smem(amap_transpose_flat_table<ES, T, P>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
       } else {
-        if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_one<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
-        else if (ds.ld) launch_smem(amap_transpose_flat_param<ES, T>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
-        else launch_smem(amap_transpose_flat_table<ES, T>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
+        if (ds.ld && ds.ld->n_pieces == 1) launch_smem(amap_transpose_flat_one<ES, T, false>, L.n_blocks, T, L.smem, s, pdl, ds.ld->piece[0], pt);
+        else if (ds.ld) launch_smem(amap_transpose_flat_param<ES, T, false>, L.n_blocks, T, L.smem, s, pdl, *ds.ld, pt);
+        else launch_smem(amap_transpose_flat_table<ES, T, false>, L.n_blocks, T, L.smem, s, pdl, ds.table, L.first_piece, L.n_pieces, pt);
       }
     };
     if (L.threads == 512) pick(std::integral_constant<int, 512>());
