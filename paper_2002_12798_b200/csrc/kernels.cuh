@@ -968,6 +968,17 @@ __device__ __forceinline__ void transpose_flat_body(const DevPiece &sp, const Pt
   const char *src = ptrs.src[sp.input] + sbase + (int64_t)b0 * ES + (int64_t)cb * 16;
   char *dst = ptrs.dst(sp.out) + dbase + (int64_t)b0 * sp.db[0];
   unsigned char *column = panel + cb * EPU * row_bytes;  // where this lane's first element of a = 0 goes
+  // An L2 hint for this block's own segments, one line per a from the lanes with cb = 0, ahead of the dependency
+  // wait: free for the blocks that sit in that wait while the kernel before this one drains.
+  if (sp.prefetch && cb == 0) {
+    const uint32_t seg = nb * ES;
+    for (uint32_t a = threadIdx.x >> lg; a < ext_a; a += a_step) {
+      const char *p = src + (merged ? (int64_t)(a - fast_div(a, fa) * fa.d) * sp.sa[0] + (int64_t)fast_div(a, fa) * sp.sa[1]
+                                    : (int64_t)a * sp.sa[0]);
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+      if (seg > 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + 128));
+    }
+  }
   pdl_wait();
 
   // rounds of equal length: ten loads are five and five, not eight and two
