@@ -429,6 +429,33 @@ def test_launch_with_more_pieces_than_fit_the_kernel_parameters(B):
     assert np.array_equal(got, want.reshape(-1))
 
 
+def test_random_layout_changes_on_every_transpose_kernel(B):
+    """Seeded random NCHW <-> NHWC shapes (odd and even maps, channel counts around the kernels' thresholds, 2- and
+    4-byte elements): whichever transpose kernel the planner picks, the bytes are the oracle's; every kernel of the
+    family is met at least once."""
+    rng = np.random.default_rng(12798)
+    seen = {}
+    for _ in range(70):
+        es = int(rng.choice([2, 2, 2, 4]))
+        n, h, w = int(rng.integers(1, 25)), int(rng.integers(1, 40)), int(rng.integers(1, 40))
+        c = int(rng.choice([8, 16, 24, 32, 40, 48, 64, 72, 96, 128, 136, 200, 256])) if rng.random() < 0.8 else int(rng.integers(1, 200))
+        n = max(1, min(n, 400_000 // (h * w * c)))
+        fwd = bool(rng.random() < 0.5)
+        chain = W.Chain(
+            name="layout", dtype="bf16" if es == 2 else "fp32", inputs=[[n, c, h, w] if fwd else [n, h, w, c]],
+            ops=[{"kind": "transpose", "src": 0, "perm": [0, 2, 3, 1] if fwd else [0, 3, 1, 2]}], values="normal",
+            seed=int(rng.integers(1 << 30)),
+        )
+        xs = W.make_inputs(chain)
+        want = oracle.run_chain(chain, xs)
+        got, plan = run_gpu(B, chain, xs)
+        for launch in plan.launches():
+            seen[launch["kernel"]] = seen.get(launch["kernel"], 0) + 1
+        assert np.array_equal(got.view(SIGNED[es]), np.ascontiguousarray(want).reshape(-1).view(SIGNED[es])), (chain.inputs, fwd)
+    for kernel in ("transpose", "transpose_flat", "transpose_flat_source", "transpose_shifted", "transpose_realign"):
+        assert seen.get(kernel, 0) > 0, seen
+
+
 def test_flat_destination_transposes_from_the_descriptor_table(B):
     """Twenty NHWC operands joined along the batch and taken to NCHW (7x7 maps: rows of 98 bytes): twenty pieces
     of the flat-destination transpose in one launch, their descriptors read from the plan's table."""
