@@ -102,6 +102,20 @@ def test_transpose_kernel_per_shape():
     assert launch_of(W.full_configs()["c3"])["kernel"] in ("affine", "strip")
 
 
+def test_launch_info_arguments():
+    import ctypes
+
+    plan = B.compose_chain(W.full_configs()["c4"]).plan(device=-1)
+    (L,) = plan.launches()
+    assert L["n_descriptors"] == plan.stats()["n_descriptors"] == 9 and L["stage"] == 0 and L["wide_offsets"] == 0
+    info = B._LaunchInfo()
+    lib = B._lib
+    assert lib.amap_plan_launch_info(plan._h, 1, ctypes.byref(info)) == -1   # one launch only: AMAP_EINVAL
+    assert lib.amap_plan_launch_info(plan._h, -1, ctypes.byref(info)) == -1
+    assert lib.amap_plan_launch_info(plan._h, 0, None) == -1
+    assert lib.amap_plan_launch_info(None, 0, ctypes.byref(info)) == -1
+
+
 def test_remainders_of_at_most_half_a_tile_become_pieces_of_their_own():
     """The 16-byte transpose kernel's tile spans 128 bytes of the destination run.  An extent that leaves at most
     64 bytes over is cut: whole tiles, plus the remainder on the 64-byte tile."""
